@@ -1,0 +1,156 @@
+/*
+ * zqfp — W4A8 quantized linear layer (FP4-E2M1 weights, FP8-E4M3 activations, LoRC) for sm_100a.
+ *
+ * C ABI.  Unless a parameter says "host", every pointer is a DEVICE pointer owned by the caller;
+ * the library never allocates or frees device memory.  Every call enqueues its work on `stream`
+ * (a cudaStream_t passed as void*, NULL = the default stream) and returns without synchronizing,
+ * except where stated.  Return value: ZQ_OK, or a negative ZQ_ERR_* found by host-side validation
+ * before anything was launched.  No exception crosses the boundary.  Calls on distinct streams with
+ * distinct workspaces are independent; two calls that share a workspace must not overlap on the GPU.
+ *
+ * Notation (follows the paper): x[M,K] activations (tokens x input features), W[N,K] weight
+ * (output x input features, as nn.Linear stores it), group = number of consecutive input features
+ * of one output row that share a weight scale, G = K / group, r = LoRC rank.
+ */
+#ifndef ZQFP_H_
+#define ZQFP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ZQ_OK 0
+#define ZQ_ERR_NULL (-1)           /* a required pointer is NULL */
+#define ZQ_ERR_SHAPE (-2)          /* a size is negative, not a supported multiple, or too large */
+#define ZQ_ERR_ALIGN (-3)          /* a pointer or a leading dimension breaks its alignment rule */
+#define ZQ_ERR_MODE (-4)           /* unknown scale mode or output type */
+#define ZQ_ERR_WORKSPACE (-5)      /* workspace missing or smaller than *_workspace_bytes() says */
+#define ZQ_ERR_ARCH (-6)           /* the current device is not compute capability 10.x */
+#define ZQ_ERR_CUDA (-7)           /* a CUDA runtime / driver call failed (launch, tensor map) */
+#define ZQ_ERR_DEVICE_TIMEOUT (-8) /* a kernel gave up on a bounded wait; see zq_device_status */
+
+/* Weight-scale constraint, Section 3 "Casting the FP4 to FP8". */
+typedef enum {
+  ZQ_SCALE_NONE = 0, /* unconstrained FP32 scale per group */
+  ZQ_SCALE_M1 = 1,   /* (M1) every group scale is rounded up to a power of two */
+  ZQ_SCALE_M2 = 2    /* (M2) group scale = per-channel S_max divided by a power of two */
+} zq_scale_mode;
+
+typedef enum { ZQ_OUT_F32 = 0, ZQ_OUT_BF16 = 1 } zq_out_dtype;
+
+const char* zq_status_string(int status);
+
+/*
+ * Token-wise FP8 activation quantization (Section 3: "token-wise quantization for activation";
+ * Appendix A; symmetric, i.e. Eq. 1 with Z = 0, in the E4M3 format of Section 2 / 4).
+ *
+ *   a_m = max_k |x[m,k]| ;  sx[m] = a_m / 448 ;  q[m,k] = RNE_E4M3( fl32( x[m,k] * fl32(448 / a_m) ) )
+ *   saturating at +-448; a token whose elements are all zero gets sx = 1 and codes 0.
+ * If V != NULL it also computes the LoRC down-projection (Section 3, LoRC) with the raw x:
+ *   t[m,j] = sum_k V[j,k] * x[m,k],  j < r, accumulated in FP32.
+ *
+ * x    : bf16 [M, ldx] row-major, ldx >= K in elements; 16-byte aligned, ldx % 8 == 0
+ * q    : out, E4M3 bytes [M, K] dense; 16-byte aligned
+ * sx   : out, FP32 [M]
+ * V    : fp16 [r, K] dense or NULL; 16-byte aligned;  t: out, FP32 [M, r] (required iff V != NULL)
+ * K % 16 == 0, 16 <= K; 0 <= M; 0 < r <= 64 when V is given.  M == 0 is a no-op.
+ */
+int zq_quantize_act_fp8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, uint8_t* q,
+                        float* sx, const void* V_f16, int r, float* t, void* stream);
+
+/*
+ * Sizes in bytes of the three buffers zq_pack_weight_fp4 writes:
+ *   codes: N*K/2 ; shift: N*G (M1, M2) or 0 (none) ; scale: 4*N (M1, M2) or 4*N*G (none).
+ */
+int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, size_t* codes_bytes,
+                           size_t* shift_bytes, size_t* scale_bytes);
+
+/*
+ * Fine-grained FP4 weight quantization (Section 3: FGQ; Appendix A: group size) with the scale
+ * constraints of Section 3 "Casting the FP4 to FP8".
+ *
+ *   per (n, group j):  S_j = max|W| / 6  (FP32 division);
+ *   none: S^_j = S_j                                  -> scale[n,j] = S_j
+ *   M1  : S^_j = 2^ceil(log2 S_j)                     -> scale[n] = 2^P, P = max_j ceil(log2 S_j),
+ *                                                        shift[n,j] = P - ceil(log2 S_j)
+ *   M2  : S^_j = S_max / 2^ceil(log2(S_max / S_j))    -> scale[n] = S_max = max_j S_j,
+ *                                                        shift[n,j] = ceil(log2(S_max / S_j))
+ *   code = RNE_E2M1( fl32( W[n,k] / S^_j ) ), saturating at +-6.
+ * Shifts are stored clamped to [0, 5] (the range in which the cast to E4M3 is a subtraction in the
+ * exponent field); a clamped group is quantized with scale[n] * 2^-5.  A group of all zeros takes no
+ * part in the row maximum, gets shift 0 (and scale 1 in mode none).
+ *
+ * W     : FP32 [N, K] dense row-major; 16-byte aligned
+ * codes : out, [N, K/2]; byte b of a row = element 2b in bits 0..3, element 2b+1 in bits 4..7
+ * shift : out, u8 [N, G] (M1, M2); ignored (may be NULL) in mode none
+ * scale : out, FP32 [N] (M1, M2) or [N, G] (none)
+ * group in {64, 128, 256}; K % group == 0; N >= 0.
+ */
+int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale_mode mode,
+                       uint8_t* codes, uint8_t* shift, float* scale, void* stream);
+
+/*
+ * Workspace for zq_w4a8_linear: a status word, split-K tile counters and partial sums, and (when the
+ * call quantizes x itself) q, sx and t.  Zero it ONCE with zq_workspace_init before its first use;
+ * the kernels leave the counters zero again.  The size depends only on (M, N, K, r); a workspace
+ * sized for M tokens serves every smaller token count at the same (N, K, r).
+ */
+size_t zq_w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int r);
+int zq_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The quantized linear layer (Section 3):
+ *   y[m,n] = sx[m] * sum_k dec_E4M3(q[m,k]) * ( dec_E2M1(code[n,k]) * S^[n, k/group] )
+ *            + sum_{j<r} U[n,j] * t[m,j]
+ * For M1 / M2 the weight is cast to E4M3 inside the kernel by subtracting shift[n, k/group] from the
+ * exponent field (Section 3, "Casting the FP4 to FP8"), the FP8 x FP8 products are accumulated in
+ * FP32 over all of K, and sx[m] * scale[n] multiplies the sum once.  In mode none the FP32
+ * group scale multiplies each group's partial sum.
+ *
+ * Activations come either pre-quantized (q, sx, and t when r > 0; x_bf16 = NULL) or raw
+ * (x_bf16 [M, ldx] given, q = sx = t = NULL): then the call first runs zq_quantize_act_fp8 into the
+ * workspace (with V when r > 0).
+ *
+ * codes / shift / scale : as written by zq_pack_weight_fp4 for the same (N, K, group, mode)
+ * U : fp16 [N, r] dense or NULL (r = 0);  V : fp16 [r, K], only read when x_bf16 is given and r > 0
+ * y : out, [M, ldy] FP32 or bf16 (ydt), ldy >= N in elements
+ * K % 128 == 0; group in {64, 128, 256}; r in {0, 8, 16, ..., 64}; q, codes 16-byte aligned.
+ * M == 0 or N == 0 is a no-op.  Summation order over K depends on the launch shape (split-K), so
+ * FP32 results are reproducible for a fixed (M, N, K) but not bit-identical across token counts.
+ */
+int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M,
+                   int64_t N, int64_t K, int group, zq_scale_mode mode, const uint8_t* codes,
+                   const uint8_t* shift, const float* scale, const void* U_f16, const void* V_f16,
+                   const float* t, int r, void* y, zq_out_dtype ydt, int64_t ldy, void* workspace,
+                   size_t workspace_bytes, void* stream);
+
+/*
+ * The same layer for callers whose activations live in HOST memory: copies x (bf16 [M, K] dense,
+ * host, ideally pinned) to the device, runs quantizer + linear, copies y (FP32 [M, N] dense, host)
+ * back and synchronizes the stream before returning.  Weights, U, V and the workspace stay on the
+ * device.  The workspace must have zq_w4a8_linear_host_workspace_bytes(M, N, K, r) bytes and must
+ * have been zeroed once with zq_workspace_init.
+ */
+size_t zq_w4a8_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int r);
+int zq_w4a8_linear_host(const void* x_bf16_host, int64_t M, int64_t N, int64_t K, int group,
+                        zq_scale_mode mode, const uint8_t* codes, const uint8_t* shift,
+                        const float* scale, const void* U_f16, const void* V_f16, int r,
+                        float* y_host, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Synchronizes `stream`, reads the workspace's status word and clears it.  Returns ZQ_OK or
+ * ZQ_ERR_DEVICE_TIMEOUT (a kernel's bounded wait on a barrier ran out; its output is invalid and the
+ * workspace must be re-initialized).  `detail` (host, may be NULL) receives a code naming the wait.
+ */
+int zq_device_status(void* workspace, int* detail, void* stream);
+
+/* Number of kernels of this library launched by the calling process so far (all entry points). */
+int64_t zq_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZQFP_H_ */

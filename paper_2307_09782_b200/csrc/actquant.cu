@@ -1,0 +1,201 @@
+// Token-wise FP8-E4M3 activation quantizer with the optional LoRC down-projection t = V x.
+// Section 3 (token-wise activation quantization; LoRC), Appendix A, Eq. 1 with Z = 0.
+//
+// One CTA per token.  The row is read once from HBM with 16-byte loads and kept in registers
+// between the absmax reduction and the cast (rows longer than the register budget are re-read).
+// A thread's unit is 16 consecutive elements: two 16-byte loads in, one 16-byte store out.
+#include <cuda_fp16.h>
+
+#include "zq_common.cuh"
+
+namespace zq {
+namespace {
+
+constexpr int kUnit = 16;   // elements per thread-unit
+constexpr int kVpt = 8;     // units a thread keeps in registers
+constexpr int kMaxThreads = 256;
+constexpr int kRChunk = 8;  // LoRC rows of V handled per pass over the registers
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// Two FP32 values -> two E4M3 bytes (round to nearest even, saturate to +-448); `lo` lands in bits 0..7.
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
+  uint16_t r;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ float absmax8(uint4 v, float a) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    a = fmaxf(a, fabsf(bf16_lo(w[i])));  // fmaxf drops a NaN operand
+    a = fmaxf(a, fabsf(bf16_hi(w[i])));
+  }
+  return a;
+}
+
+__device__ __forceinline__ uint2 cast8(uint4 v, float inv) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+  uint32_t p[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    p[i] = cvt_e4m3x2(__fmul_rn(bf16_lo(w[i]), inv), __fmul_rn(bf16_hi(w[i]), inv));
+  return make_uint2(p[0] | (p[1] << 16), p[2] | (p[3] << 16));
+}
+
+// acc + sum over 8 elements of x (bf16 pairs in xv) times V (fp16 pairs in vv)
+__device__ __forceinline__ float dot8(uint4 xv, uint4 vv, float acc) {
+  const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+  const uint32_t vw[4] = {vv.x, vv.y, vv.z, vv.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    __half2 h;
+    *reinterpret_cast<uint32_t*>(&h) = vw[i];
+    const float2 vf = __half22float2(h);
+    acc = fmaf(bf16_lo(xw[i]), vf.x, acc);
+    acc = fmaf(bf16_hi(xw[i]), vf.y, acc);
+  }
+  return acc;
+}
+
+template <bool CACHED>
+__global__ void __launch_bounds__(kMaxThreads)
+act_quant_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, uint8_t* __restrict__ q,
+                 float* __restrict__ sx, const uint4* __restrict__ V, int r, float* __restrict__ t) {
+  const int64_t m = blockIdx.x;
+  const int nunits = K / kUnit;
+  const uint4* row = x + m * ldx_vec;  // 8 bf16 per uint4
+  uint4* qrow = reinterpret_cast<uint4*>(q + m * static_cast<int64_t>(K));
+  const int T = blockDim.x, tid = threadIdx.x;
+  __shared__ float red[kMaxThreads / 32];
+  __shared__ float red_t[kMaxThreads / 32][kRChunk];
+
+  uint4 c0[kVpt], c1[kVpt];
+  float a = 0.0f;
+  if (CACHED) {
+#pragma unroll
+    for (int i = 0; i < kVpt; ++i) {
+      const int u = tid + i * T;
+      if (u < nunits) {
+        c0[i] = __ldg(row + 2 * u);
+        c1[i] = __ldg(row + 2 * u + 1);
+      } else {
+        c0[i] = make_uint4(0, 0, 0, 0);
+        c1[i] = make_uint4(0, 0, 0, 0);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kVpt; ++i) a = absmax8(c1[i], absmax8(c0[i], a));
+  } else {
+    for (int u = tid; u < nunits; u += T) a = absmax8(__ldg(row + 2 * u + 1), absmax8(__ldg(row + 2 * u), a));
+  }
+  a = warp_max(a);
+  if ((tid & 31) == 0) red[tid >> 5] = a;
+  __syncthreads();
+  a = red[0];
+  for (int w = 1; w < (T >> 5); ++w) a = fmaxf(a, red[w]);
+
+  float s = 1.0f, inv = 1.0f;
+  if (a != 0.0f) {
+    s = __fdiv_rn(a, 448.0f);
+    inv = __fdiv_rn(448.0f, a);
+  }
+  if (tid == 0) sx[m] = s;
+
+  if (CACHED) {
+#pragma unroll
+    for (int i = 0; i < kVpt; ++i) {
+      const int u = tid + i * T;
+      if (u < nunits) {
+        const uint2 lo = cast8(c0[i], inv), hi = cast8(c1[i], inv);
+        qrow[u] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+      }
+    }
+  } else {
+    for (int u = tid; u < nunits; u += T) {
+      const uint2 lo = cast8(__ldg(row + 2 * u), inv), hi = cast8(__ldg(row + 2 * u + 1), inv);
+      qrow[u] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+    }
+  }
+
+  // LoRC down-projection with the raw row (Section 3): t[m, j] = sum_k V[j, k] x[m, k]
+  if (V != nullptr) {
+    const int kvec = K / 8;  // uint4 per row of V
+    for (int j0 = 0; j0 < r; j0 += kRChunk) {
+      float acc[kRChunk];
+#pragma unroll
+      for (int j = 0; j < kRChunk; ++j) acc[j] = 0.0f;
+      if (CACHED) {
+#pragma unroll
+        for (int i = 0; i < kVpt; ++i) {
+          const int u = tid + i * T;
+          if (u < nunits) {
+#pragma unroll
+            for (int j = 0; j < kRChunk; ++j)
+              if (j0 + j < r) {
+                const uint4* vr = V + static_cast<int64_t>(j0 + j) * kvec;
+                acc[j] = dot8(c1[i], __ldg(vr + 2 * u + 1), dot8(c0[i], __ldg(vr + 2 * u), acc[j]));
+              }
+          }
+        }
+      } else {
+        for (int u = tid; u < nunits; u += T) {
+          const uint4 a0 = __ldg(row + 2 * u), a1 = __ldg(row + 2 * u + 1);
+#pragma unroll
+          for (int j = 0; j < kRChunk; ++j)
+            if (j0 + j < r) {
+              const uint4* vr = V + static_cast<int64_t>(j0 + j) * kvec;
+              acc[j] = dot8(a1, __ldg(vr + 2 * u + 1), dot8(a0, __ldg(vr + 2 * u), acc[j]));
+            }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < kRChunk; ++j) {
+        const float v = warp_sum(acc[j]);
+        if ((tid & 31) == 0) red_t[tid >> 5][j] = v;
+      }
+      __syncthreads();
+      if (tid < kRChunk && j0 + tid < r) {
+        float v = 0.0f;
+        for (int w = 0; w < (T >> 5); ++w) v += red_t[w][tid];
+        t[m * r + j0 + tid] = v;
+      }
+      __syncthreads();
+    }
+  }
+}
+
+}  // namespace
+
+int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
+                     const void* V, int r, float* t, cudaStream_t st) {
+  if (M == 0) return ZQ_OK;
+  const int nunits = static_cast<int>(K / kUnit);
+  int threads = ((nunits + 31) / 32) * 32;
+  if (threads > kMaxThreads) threads = kMaxThreads;
+  const bool cached = nunits <= threads * kVpt;
+  dim3 grid(static_cast<unsigned>(M));
+  if (cached)
+    act_quant_kernel<true><<<grid, threads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(K), ldx / 8, q,
+                                                     sx, static_cast<const uint4*>(V), r, t);
+  else
+    act_quant_kernel<false><<<grid, threads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(K), ldx / 8, q,
+                                                      sx, static_cast<const uint4*>(V), r, t);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+}
+
+}  // namespace zq

@@ -1,0 +1,181 @@
+// Shared helpers for the zqfp kernels: thin wrappers over the sm_100a PTX this library uses
+// (mbarrier, TMA bulk tensor loads, tcgen05 MMA / TMEM) and the host-side launch bookkeeping.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/zqfp.h"
+
+namespace zq {
+
+// ---- host-side bookkeeping ---------------------------------------------------------------------
+void count_launch(int n = 1);  // adds to the process-wide launch counter
+
+// Workspace head: status words the kernels may write (256 bytes), then the split-K tile counters.
+constexpr size_t kWsStatusBytes = 256;
+constexpr int kWsMaxTiles = 16384;  // counters: one int per output tile
+constexpr size_t kWsCounterBytes = size_t(kWsMaxTiles) * 4;
+constexpr size_t kWsHeadBytes = kWsStatusBytes + kWsCounterBytes;
+
+// ---- launchers implemented in the .cu files ------------------------------------------------------
+int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
+                     const void* V, int r, float* t, cudaStream_t st);
+int launch_pack_weight(const float* W, int64_t N, int64_t K, int group, int mode, uint8_t* codes,
+                       uint8_t* shift, float* scale, cudaStream_t st);
+
+struct GemmArgs {
+  const uint8_t* q;      // [M, K] E4M3
+  const float* sx;       // [M]
+  int64_t M, N, K;
+  int group, mode;
+  const uint8_t* codes;  // [N, K/2]
+  const uint8_t* shift;  // [N, G] or NULL
+  const float* scale;    // [N] or [N, G]
+  const void* U;         // fp16 [N, r] or NULL
+  const float* t;        // [M, r] or NULL
+  int r;
+  void* y;
+  int ydt;
+  int64_t ldy;
+  int* status;           // workspace status words
+  int* counters;         // split-K tile counters
+  float* partials;       // split-K partial sums
+  size_t partial_floats; // capacity of `partials`
+};
+// Tile shape chosen for a problem (shared by the workspace-size query and the launcher).
+struct GemmPlan {
+  int bm;      // tokens per tile (the MMA's N extent)
+  int splits;  // split-K factor
+  int m_tiles, n_tiles;
+  size_t partial_floats;
+};
+GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode);
+int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st);
+
+#ifdef __CUDACC__
+// ---- device: bounded waits -----------------------------------------------------------------------
+// Every spin in this library gives up after kSpinLimit polls; the kernel then records an error in the
+// workspace status word and unwinds instead of hanging.
+constexpr uint32_t kSpinLimit = 1u << 24;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void fence_mbar_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Returns false when the wait ran out or another thread of the CTA already raised `abort_flag`.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (spin > 64) {
+      if (*abort_flag) return false;
+      if (spin > 4096) __nanosleep(64);
+    }
+  }
+  return false;
+}
+
+// ---- device: proxies, TMA ------------------------------------------------------------------------
+__device__ __forceinline__ void fence_proxy_async_smem() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
+}
+// 2-D tiled load global -> shared, completion counted in bytes on `bar`.  c0 is the innermost
+// coordinate; c0 * element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m, int c0, int c1,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+// ---- device: tcgen05 / TMEM ----------------------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t ncols) {  // one full warp
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
+               "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {  // one full warp
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after_sync() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc], 8-bit float operands (E4M3 x E4M3), FP32 accumulate.
+__device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrive once on `bar` when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// 16 consecutive FP32 columns of this thread's TMEM lane (lane = 32 * (warp % 4) + lane id).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory operand descriptor: K-major tile whose rows are 128 bytes, stored as 8-row x 128-byte
+// atoms (1024 bytes apart) with the 128-byte swizzle.  Adding (bytes >> 4) to the low word moves the
+// start along K inside the 128-byte row.
+__device__ __forceinline__ uint64_t umma_desc_k128(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= uint64_t((smem_addr >> 4) & 0x3FFF);  // start address, 16-byte units
+  d |= uint64_t(1) << 16;                    // leading byte offset (unused for swizzled K-major)
+  d |= uint64_t(1024 >> 4) << 32;            // stride byte offset: next 8-row atom
+  d |= uint64_t(1) << 46;                    // descriptor version of this architecture
+  d |= uint64_t(2) << 61;                    // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: E4M3 x E4M3 -> FP32, both operands K-major, D is 128 x n.
+__device__ __forceinline__ uint32_t umma_idesc_e4m3(uint32_t n) {
+  return (1u << 4) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+#endif  // __CUDACC__
+
+}  // namespace zq
