@@ -1,0 +1,191 @@
+"""Thin ctypes binding of ``libzqfp.so``: argument marshalling only.
+
+Every function mirrors the C entry point of the same name in ``include/zqfp.h``.  Tensors are torch
+CUDA tensors used purely as device memory; work is enqueued on torch's current stream.  There is no
+CPU or PyTorch fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libzqfp.so")
+
+SCALE_NONE, SCALE_M1, SCALE_M2 = 0, 1, 2
+MODES = {"none": SCALE_NONE, "M1": SCALE_M1, "M2": SCALE_M2}
+OUT_F32, OUT_BF16 = 0, 1
+
+EXPORTS = [
+    "zq_status_string", "zq_quantize_act_fp8", "zq_packed_weight_sizes", "zq_pack_weight_fp4",
+    "zq_w4a8_linear_workspace_bytes", "zq_workspace_init", "zq_w4a8_linear",
+    "zq_w4a8_linear_host_workspace_bytes", "zq_w4a8_linear_host", "zq_device_status", "zq_launch_count",
+]
+
+
+class ZqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads the library (building nothing: run ``__graft_entry__.build()`` first)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} is missing: build it with paper_2307_09782_b200/build.py")
+        L = C.CDLL(LIB_PATH)
+        vp, i64, sz, ci = C.c_void_p, C.c_int64, C.c_size_t, C.c_int
+        L.zq_status_string.restype = C.c_char_p
+        L.zq_status_string.argtypes = [ci]
+        L.zq_quantize_act_fp8.restype = ci
+        L.zq_quantize_act_fp8.argtypes = [vp, i64, i64, i64, vp, vp, vp, ci, vp, vp]
+        L.zq_packed_weight_sizes.restype = ci
+        L.zq_packed_weight_sizes.argtypes = [i64, i64, ci, ci, C.POINTER(sz), C.POINTER(sz), C.POINTER(sz)]
+        L.zq_pack_weight_fp4.restype = ci
+        L.zq_pack_weight_fp4.argtypes = [vp, i64, i64, ci, ci, vp, vp, vp, vp]
+        L.zq_w4a8_linear_workspace_bytes.restype = sz
+        L.zq_w4a8_linear_workspace_bytes.argtypes = [i64, i64, i64, ci]
+        L.zq_w4a8_linear_host_workspace_bytes.restype = sz
+        L.zq_w4a8_linear_host_workspace_bytes.argtypes = [i64, i64, i64, ci]
+        L.zq_workspace_init.restype = ci
+        L.zq_workspace_init.argtypes = [vp, sz, vp]
+        L.zq_w4a8_linear.restype = ci
+        L.zq_w4a8_linear.argtypes = [vp, vp, vp, i64, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, vp, ci, vp, ci,
+                                     i64, vp, sz, vp]
+        L.zq_w4a8_linear_host.restype = ci
+        L.zq_w4a8_linear_host.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, ci, vp, vp, sz, vp]
+        L.zq_device_status.restype = ci
+        L.zq_device_status.argtypes = [vp, C.POINTER(ci), vp]
+        L.zq_launch_count.restype = i64
+        L.zq_launch_count.argtypes = []
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().zq_status_string(int(status)).decode()
+
+
+def launch_count() -> int:
+    return int(lib().zq_launch_count())
+
+
+def _mode(mode) -> int:
+    return MODES[mode] if isinstance(mode, str) else int(mode)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise ZqError(status, where)
+
+
+def packed_weight_sizes(N: int, K: int, group: int, mode):
+    a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    _check(lib().zq_packed_weight_sizes(N, K, group, _mode(mode), C.byref(a), C.byref(b), C.byref(c)),
+           "zq_packed_weight_sizes")
+    return a.value, b.value, c.value
+
+
+def quantize_act_fp8(x: torch.Tensor, V: Optional[torch.Tensor] = None):
+    """x: bf16 [M, K] (row stride allowed).  Returns (q uint8 [M,K], sx float32 [M], t float32 [M,r] | None)."""
+    assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    M, K = x.shape
+    q = torch.empty((M, K), dtype=torch.uint8, device=x.device)
+    sx = torch.empty((M,), dtype=torch.float32, device=x.device)
+    r, t = 0, None
+    if V is not None:
+        assert V.dtype == torch.float16 and V.is_contiguous() and V.shape[1] == K
+        r = V.shape[0]
+        t = torch.empty((M, r), dtype=torch.float32, device=x.device)
+    ldx = x.stride(0) if M > 1 else K
+    _check(lib().zq_quantize_act_fp8(_ptr(x), M, K, ldx, _ptr(q), _ptr(sx), _ptr(V), r, _ptr(t), _stream()),
+           "zq_quantize_act_fp8")
+    return q, sx, t
+
+
+def pack_weight_fp4(W: torch.Tensor, group: int, mode):
+    """W: float32 [N, K] contiguous.  Returns (codes uint8 [N,K/2], shift uint8 [N,G] | None, scale float32)."""
+    assert W.dtype == torch.float32 and W.is_contiguous() and W.dim() == 2
+    N, K = W.shape
+    mode = _mode(mode)
+    cb, sb, fb = packed_weight_sizes(N, K, group, mode)
+    G = K // group
+    codes = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
+    shift = None if mode == SCALE_NONE else torch.empty((N, G), dtype=torch.uint8, device=W.device)
+    scale = torch.empty((N, G) if mode == SCALE_NONE else (N,), dtype=torch.float32, device=W.device)
+    assert codes.numel() == cb and scale.numel() * 4 == fb and (shift is None or shift.numel() == sb)
+    _check(lib().zq_pack_weight_fp4(_ptr(W), N, K, group, mode, _ptr(codes), _ptr(shift), _ptr(scale), _stream()),
+           "zq_pack_weight_fp4")
+    return codes, shift, scale
+
+
+def linear_workspace_bytes(M: int, N: int, K: int, r: int) -> int:
+    return int(lib().zq_w4a8_linear_workspace_bytes(M, N, K, r))
+
+
+def linear_host_workspace_bytes(M: int, N: int, K: int, r: int) -> int:
+    return int(lib().zq_w4a8_linear_host_workspace_bytes(M, N, K, r))
+
+
+def make_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """Allocates (through torch) and zero-initializes a workspace of ``nbytes``."""
+    ws = torch.empty((max(int(nbytes), 1),), dtype=torch.uint8, device=device)
+    _check(lib().zq_workspace_init(_ptr(ws), ws.numel(), _stream()), "zq_workspace_init")
+    return ws
+
+
+def w4a8_linear(codes, shift, scale, group: int, mode, *, q=None, sx=None, t=None, x=None, U=None, V=None,
+                out_dtype=torch.float32, workspace: Optional[torch.Tensor] = None, y=None):
+    """y [M, N] = the quantized linear layer; activations either (q, sx[, t]) or raw bf16 ``x`` (then V when U)."""
+    N, K = codes.shape[0], codes.shape[1] * 2
+    if x is not None:
+        M, ldx = x.shape[0], (x.stride(0) if x.shape[0] > 1 else K)
+    else:
+        M, ldx = q.shape[0], K
+    r = 0 if U is None else U.shape[1]
+    if workspace is None:
+        workspace = make_workspace(linear_workspace_bytes(M, N, K, r), codes.device)
+    if y is None:
+        y = torch.empty((M, N), dtype=out_dtype, device=codes.device)
+    ydt = OUT_F32 if y.dtype == torch.float32 else OUT_BF16
+    ldy = y.stride(0) if M > 1 else N
+    _check(lib().zq_w4a8_linear(_ptr(q), _ptr(sx), _ptr(x), ldx, M, N, K, group, _mode(mode), _ptr(codes), _ptr(shift),
+                                _ptr(scale), _ptr(U), _ptr(V), _ptr(t), r, _ptr(y), ydt, ldy, _ptr(workspace),
+                                workspace.numel(), _stream()), "zq_w4a8_linear")
+    return y
+
+
+def w4a8_linear_host(x_host: torch.Tensor, y_host: torch.Tensor, codes, shift, scale, group: int, mode, *, U=None,
+                     V=None, workspace: torch.Tensor):
+    """Host-buffer variant: x_host bf16 [M,K] and y_host float32 [M,N] are CPU (pinned) tensors; synchronous."""
+    assert not x_host.is_cuda and not y_host.is_cuda and x_host.is_contiguous() and y_host.is_contiguous()
+    M, K = x_host.shape
+    N = codes.shape[0]
+    r = 0 if U is None else U.shape[1]
+    _check(lib().zq_w4a8_linear_host(_ptr(x_host), M, N, K, group, _mode(mode), _ptr(codes), _ptr(shift),
+                                     _ptr(scale), _ptr(U), _ptr(V), r, _ptr(y_host), _ptr(workspace),
+                                     workspace.numel(), _stream()), "zq_w4a8_linear_host")
+    return y_host
+
+
+def device_status(workspace: torch.Tensor):
+    """Synchronizes the current stream; returns (status, detail)."""
+    d = C.c_int(0)
+    st = lib().zq_device_status(_ptr(workspace), C.byref(d), _stream())
+    return int(st), int(d.value)

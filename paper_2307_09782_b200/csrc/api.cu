@@ -1,0 +1,245 @@
+// C-ABI entry points of libzqfp: argument validation, workspace carving, kernel dispatch.
+// The operations themselves are defined in include/zqfp.h next to their citations.
+#include <atomic>
+
+#include "zq_common.cuh"
+
+namespace zq {
+
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int check_device_sm100() {
+  int dev = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ZQ_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ZQ_ERR_CUDA;
+  return major == 10 ? ZQ_OK : ZQ_ERR_ARCH;
+}
+
+bool valid_mode(int mode) { return mode == ZQ_SCALE_NONE || mode == ZQ_SCALE_M1 || mode == ZQ_SCALE_M2; }
+bool valid_group(int g) { return g == 64 || g == 128 || g == 256; }
+
+// Largest split-K scratch any token count up to M can need at this (N, K), over both kernel families.
+size_t max_partial_floats(int64_t M, int64_t N, int64_t K) {
+  size_t best = 0;
+  const int64_t cand[6] = {16, 32, 64, 128, 256, M};
+  for (int mode = 0; mode < 2; ++mode)
+    for (int i = 0; i < 6; ++i) {
+      const int64_t m = cand[i] < M ? cand[i] : M;
+      if (m <= 0) continue;
+      const GemmPlan pl = plan_gemm(m, N, K, mode == 0 ? ZQ_SCALE_NONE : ZQ_SCALE_M1);
+      if (pl.partial_floats > best) best = pl.partial_floats;
+    }
+  return best;
+}
+
+struct WsLayout {
+  size_t off_partials, partial_floats, off_q, off_sx, off_t, off_x, off_y, total;
+};
+WsLayout ws_layout(int64_t M, int64_t N, int64_t K, int r, bool host_io) {
+  WsLayout w{};
+  size_t off = kWsHeadBytes;
+  w.off_partials = off;
+  w.partial_floats = max_partial_floats(M, N, K);
+  off += round_up(w.partial_floats * 4, 256);
+  w.off_q = off;
+  off += round_up(static_cast<size_t>(M) * K, 256);
+  w.off_sx = off;
+  off += round_up(static_cast<size_t>(M) * 4, 256);
+  w.off_t = off;
+  off += round_up(static_cast<size_t>(M) * (r > 0 ? r : 1) * 4, 256);
+  w.off_x = w.off_y = off;
+  if (host_io) {
+    w.off_x = off;
+    off += round_up(static_cast<size_t>(M) * K * 2, 256);
+    w.off_y = off;
+    off += round_up(static_cast<size_t>(M) * N * 4, 256);
+  }
+  w.total = off;
+  return w;
+}
+
+}  // namespace
+}  // namespace zq
+
+using namespace zq;
+
+extern "C" {
+
+const char* zq_status_string(int status) {
+  switch (status) {
+    case ZQ_OK: return "ok";
+    case ZQ_ERR_NULL: return "a required pointer is NULL";
+    case ZQ_ERR_SHAPE: return "unsupported shape";
+    case ZQ_ERR_ALIGN: return "pointer or leading dimension not aligned";
+    case ZQ_ERR_MODE: return "unknown scale mode or output type";
+    case ZQ_ERR_WORKSPACE: return "workspace missing or too small";
+    case ZQ_ERR_ARCH: return "device is not compute capability 10.x";
+    case ZQ_ERR_CUDA: return "CUDA call failed";
+    case ZQ_ERR_DEVICE_TIMEOUT: return "a kernel gave up on a bounded wait";
+  }
+  return "unknown status";
+}
+
+int64_t zq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int zq_quantize_act_fp8(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
+                        const void* V, int r, float* t, void* stream) {
+  if (M < 0 || K < 16 || K % 16 || ldx < K || K > (int64_t(1) << 30) || M > 0x7FFFFFFF) return ZQ_ERR_SHAPE;
+  if (V && (r <= 0 || r > 64)) return ZQ_ERR_SHAPE;
+  if (M == 0) return ZQ_OK;
+  if (!x || !q || !sx || (V && !t)) return ZQ_ERR_NULL;
+  if (!aligned16(x) || !aligned16(q) || ldx % 8 || (V && !aligned16(V))) return ZQ_ERR_ALIGN;
+  if (int e = check_device_sm100()) return e;
+  return launch_act_quant(x, M, K, ldx, q, sx, V, V ? r : 0, t, static_cast<cudaStream_t>(stream));
+}
+
+int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, size_t* codes_bytes,
+                           size_t* shift_bytes, size_t* scale_bytes) {
+  if (!valid_mode(mode)) return ZQ_ERR_MODE;
+  if (N < 0 || K <= 0 || !valid_group(group) || K % group) return ZQ_ERR_SHAPE;
+  const size_t G = static_cast<size_t>(K / group);
+  if (codes_bytes) *codes_bytes = static_cast<size_t>(N) * (K / 2);
+  if (shift_bytes) *shift_bytes = mode == ZQ_SCALE_NONE ? 0 : static_cast<size_t>(N) * G;
+  if (scale_bytes) *scale_bytes = mode == ZQ_SCALE_NONE ? static_cast<size_t>(N) * G * 4 : static_cast<size_t>(N) * 4;
+  return ZQ_OK;
+}
+
+int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale_mode mode, uint8_t* codes,
+                       uint8_t* shift, float* scale, void* stream) {
+  if (!valid_mode(mode)) return ZQ_ERR_MODE;
+  if (N < 0 || K <= 0 || !valid_group(group) || K % group || N > 0x7FFFFFFF || K > (int64_t(1) << 30))
+    return ZQ_ERR_SHAPE;
+  if (N == 0) return ZQ_OK;
+  if (!W || !codes || !scale || (mode != ZQ_SCALE_NONE && !shift)) return ZQ_ERR_NULL;
+  if (!aligned16(W) || (reinterpret_cast<uintptr_t>(codes) & 3u)) return ZQ_ERR_ALIGN;
+  if (int e = check_device_sm100()) return e;
+  return launch_pack_weight(W, N, K, group, mode, codes, shift, scale, static_cast<cudaStream_t>(stream));
+}
+
+size_t zq_w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int r) {
+  if (M < 0 || N < 0 || K <= 0 || r < 0) return 0;
+  return ws_layout(M, N, K, r, false).total;
+}
+
+size_t zq_w4a8_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int r) {
+  if (M < 0 || N < 0 || K <= 0 || r < 0) return 0;
+  return ws_layout(M, N, K, r, true).total;
+}
+
+int zq_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (!workspace) return ZQ_ERR_NULL;
+  if (workspace_bytes < kWsHeadBytes) return ZQ_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return ZQ_ERR_ALIGN;
+  return cudaMemsetAsync(workspace, 0, kWsHeadBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? ZQ_OK
+                                                                                                       : ZQ_ERR_CUDA;
+}
+
+int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M, int64_t N,
+                   int64_t K, int group, zq_scale_mode mode, const uint8_t* codes, const uint8_t* shift,
+                   const float* scale, const void* U, const void* V, const float* t, int r, void* y,
+                   zq_out_dtype ydt, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!valid_mode(mode) || (ydt != ZQ_OUT_F32 && ydt != ZQ_OUT_BF16)) return ZQ_ERR_MODE;
+  if (M < 0 || N < 0 || K <= 0 || K % 128 || !valid_group(group) || K % group || r < 0 || r > 64 || r % 8 ||
+      ldy < N || M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > (int64_t(1) << 30))
+    return ZQ_ERR_SHAPE;
+  if (M == 0 || N == 0) return ZQ_OK;
+  if (!codes || !scale || !y || (mode != ZQ_SCALE_NONE && !shift) || (r > 0 && !U)) return ZQ_ERR_NULL;
+  if (x_bf16) {
+    if (r > 0 && !V) return ZQ_ERR_NULL;
+    if (ldx < K) return ZQ_ERR_SHAPE;
+  } else if (!q || !sx || (r > 0 && !t)) {
+    return ZQ_ERR_NULL;
+  }
+  if (!aligned16(codes) || (q && !aligned16(q)) || (U && !aligned16(U)) || (t && !aligned16(t)) ||
+      (x_bf16 && (!aligned16(x_bf16) || ldx % 8 || (V && !aligned16(V)))))
+    return ZQ_ERR_ALIGN;
+  if (!workspace) return ZQ_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return ZQ_ERR_ALIGN;
+  const WsLayout w = ws_layout(M, N, K, r, false);
+  const size_t need = x_bf16 ? w.total : w.off_q;
+  if (workspace_bytes < need) return ZQ_ERR_WORKSPACE;
+  const GemmPlan pl = plan_gemm(M, N, K, mode);
+  if (pl.m_tiles > 65535 || pl.splits > 65535) return ZQ_ERR_SHAPE;
+  if (int e = check_device_sm100()) return e;
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if (x_bf16) {
+    uint8_t* q_ws = ws + w.off_q;
+    float* sx_ws = reinterpret_cast<float*>(ws + w.off_sx);
+    float* t_ws = reinterpret_cast<float*>(ws + w.off_t);
+    const int e = launch_act_quant(x_bf16, M, K, ldx, q_ws, sx_ws, r > 0 ? V : nullptr, r, t_ws, st);
+    if (e) return e;
+    q = q_ws;
+    sx = sx_ws;
+    t = t_ws;
+  }
+  GemmArgs a{};
+  a.q = q;
+  a.sx = sx;
+  a.M = M;
+  a.N = N;
+  a.K = K;
+  a.group = group;
+  a.mode = mode;
+  a.codes = codes;
+  a.shift = shift;
+  a.scale = scale;
+  a.U = r > 0 ? U : nullptr;
+  a.t = r > 0 ? t : nullptr;
+  a.r = r;
+  a.y = y;
+  a.ydt = ydt;
+  a.ldy = ldy;
+  a.status = reinterpret_cast<int*>(ws);
+  a.counters = reinterpret_cast<int*>(ws + kWsStatusBytes);
+  a.partials = reinterpret_cast<float*>(ws + w.off_partials);
+  a.partial_floats = w.partial_floats;
+  return launch_w4a8_gemm(a, st);
+}
+
+int zq_w4a8_linear_host(const void* x_host, int64_t M, int64_t N, int64_t K, int group, zq_scale_mode mode,
+                        const uint8_t* codes, const uint8_t* shift, const float* scale, const void* U,
+                        const void* V, int r, float* y_host, void* workspace, size_t workspace_bytes,
+                        void* stream) {
+  if (M < 0 || N < 0 || K <= 0 || r < 0) return ZQ_ERR_SHAPE;
+  if (M == 0 || N == 0) return ZQ_OK;
+  if (!x_host || !y_host) return ZQ_ERR_NULL;
+  if (!workspace) return ZQ_ERR_WORKSPACE;
+  const WsLayout w = ws_layout(M, N, K, r, true);
+  if (workspace_bytes < w.total) return ZQ_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  void* x_dev = ws + w.off_x;
+  float* y_dev = reinterpret_cast<float*>(ws + w.off_y);
+  if (cudaMemcpyAsync(x_dev, x_host, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return ZQ_ERR_CUDA;
+  const int e = zq_w4a8_linear(nullptr, nullptr, x_dev, K, M, N, K, group, mode, codes, shift, scale, U, V, nullptr,
+                               r, y_dev, ZQ_OUT_F32, N, workspace, w.off_x, stream);
+  if (e) return e;
+  if (cudaMemcpyAsync(y_host, y_dev, static_cast<size_t>(M) * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return ZQ_ERR_CUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+}
+
+int zq_device_status(void* workspace, int* detail, void* stream) {
+  if (!workspace) return ZQ_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int words[2] = {0, 0};
+  if (cudaMemcpyAsync(words, workspace, sizeof(words), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return ZQ_ERR_CUDA;
+  if (detail) *detail = words[1];
+  if (words[0] != 0) {
+    if (cudaMemsetAsync(workspace, 0, 8, st) != cudaSuccess) return ZQ_ERR_CUDA;
+    return ZQ_ERR_DEVICE_TIMEOUT;
+  }
+  return ZQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,585 @@
+// W4A8 GEMM: y = sx * scale * (Q_fp8(x) . cast_fp8(W_fp4)^T) + t U^T        (Section 3)
+//
+// The cast FP4 -> FP8 (Section 3, "Casting the FP4 to FP8") runs inside the kernel as an exponent
+// shift: TMA stages packed E2M1 tiles, CUDA cores expand each nibble to an E4M3 byte through an
+// 8-entry byte-permute table whose entries already carry the group's shift, and tcgen05 MMAs
+// (kind::f8f6f4, E4M3 x E4M3, FP32 accumulators in TMEM) consume the widened tile.
+//
+// Orientation: the weight tile is the MMA's 128-row operand (D rows = output channels n, one TMEM
+// lane each), the token tile is the N-extent operand (D columns = tokens m, BM of them).  That keeps
+// the widening work per tile fixed at 128 x 128 codes per K block whatever the token count, lets one
+// kernel serve decode (BM = 16) and prefill (BM = 256), and makes every per-channel quantity
+// (scale, shift, U row, group scale) a per-thread scalar in the epilogue.
+//
+// Warp roles (10 warps):
+//   0-3  group A : widen; M1/M2 also epilogue for the first half of the columns
+//   4-7  group B : M1/M2: widen + epilogue for the second half; mode none: per-group promotion
+//                  (TMEM -> registers, times the FP32 group scale) and the epilogue
+//   8            : TMA producer (one lane)
+//   9            : TMEM allocation, MMA issue (one lane)
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <mutex>
+
+#include "zq_common.cuh"
+
+namespace zq {
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kTileN = 128;      // output channels per CTA (MMA M extent)
+constexpr int kBlockK = 128;     // K elements per pipeline step (= one 128-byte swizzled row of E4M3)
+constexpr int kPackedBytes = kTileN * kBlockK / 2;  // 8 KB
+constexpr int kWideBytes = kTileN * kBlockK;        // 16 KB
+
+// error detail codes written to status[1]
+enum { kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6 };
+
+struct Params {
+  int M, N, K;
+  int G;             // groups per row
+  int group;
+  int kb_per_split;  // K blocks handled by one CTA
+  int kblocks;       // total K blocks
+  int splits;
+  const uint8_t* shift;
+  const float* scale;
+  const float* sx;
+  const __half* U;
+  const float* t;
+  int r;
+  void* y;
+  int ydt;
+  int64_t ldy;
+  int* status;
+  int* counters;
+  float* partials;
+};
+
+template <int BM, bool NONE>
+struct Cfg {
+  static constexpr int kTokBytes = BM * kBlockK;
+  static constexpr int NS = BM <= 16 ? 6 : BM <= 32 ? 5 : BM <= 64 ? 4 : BM <= 128 ? 3 : 2;  // TMA stages
+  static constexpr int NW = 2;                                                               // widened stages
+  static constexpr int kTmemCols = (NONE ? 2 * BM : BM) < 32 ? 32 : (NONE ? 2 * BM : BM);
+  static constexpr int kWidenThreads = NONE ? 128 : 256;
+  static constexpr int kEpiThreads = NONE ? 128 : 256;
+  // shared memory map (offsets from a 1024-byte aligned base)
+  static constexpr int offWide = 0;
+  static constexpr int offTok = offWide + NW * kWideBytes;
+  static constexpr int offPacked = offTok + NS * kTokBytes;
+  static constexpr int offBars = offPacked + NS * kPackedBytes;
+  static constexpr int kNumBars = 2 * NS + 2 * NW + 6;
+  static constexpr int offMisc = offBars + kNumBars * 8;
+  static constexpr int kSmemBytes = offMisc + 32;
+};
+
+// Expand 8 packed E2M1 codes (one 32-bit word, element i in nibble i) to 8 E4M3 bytes.
+// lut_lo / lut_hi hold the E4M3 magnitudes of the 8 E2M1 magnitudes with the group's shift already
+// subtracted from their exponent fields; the sign nibble-bit moves to bit 7 of its byte.
+__device__ __forceinline__ void widen8(uint32_t w, uint32_t lut_lo, uint32_t lut_hi, uint32_t& o0, uint32_t& o1) {
+  const uint32_t w4 = w << 4;
+  uint32_t s0, s1, m0, m1;
+  // selector nibbles with bit 3 set replicate the most significant bit of the chosen byte:
+  // byte b of w carries the sign of element 2b+1 in its top bit, byte b of (w << 4) that of element 2b
+  asm("prmt.b32 %0, %1, %2, 0xD9C8;" : "=r"(s0) : "r"(w4), "r"(w));
+  asm("prmt.b32 %0, %1, %2, 0xFBEA;" : "=r"(s1) : "r"(w4), "r"(w));
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(m0) : "r"(lut_lo), "r"(lut_hi), "r"(w & 0x7777u));
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(m1) : "r"(lut_lo), "r"(lut_hi), "r"((w >> 16) & 0x7777u));
+  o0 = m0 | (s0 & 0x80808080u);
+  o1 = m1 | (s1 & 0x80808080u);
+}
+
+// One 16-byte chunk of packed codes (32 elements) -> two 16-byte chunks of E4M3.
+__device__ __forceinline__ void widen32(uint4 p, uint32_t lut_lo, uint32_t lut_hi, uint4& a, uint4& b) {
+  widen8(p.x, lut_lo, lut_hi, a.x, a.y);
+  widen8(p.y, lut_lo, lut_hi, a.z, a.w);
+  widen8(p.z, lut_lo, lut_hi, b.x, b.y);
+  widen8(p.w, lut_lo, lut_hi, b.z, b.w);
+}
+
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void raise_error(const Params& p, volatile int* abort_flag, int detail) {
+  *abort_flag = 1;
+  if (atomicCAS(p.status, 0, ZQ_ERR_DEVICE_TIMEOUT) == 0) p.status[1] = detail;
+}
+
+// Final arithmetic of 16 consecutive tokens of one output channel, and the store.
+//   y[m, n] = sx[m] * cs * acc + sum_j t[m, j] * U[n, j]
+// u8 holds the channel's U row when r == 8 (the common rank); other ranks read U through the cache.
+__device__ __forceinline__ void finalize16(const Params& p, const float* v, int m_base, int n, float cs,
+                                           const float* u8) {
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    const int m = m_base + c;
+    if (m < p.M) {
+      float out = __ldg(p.sx + m) * cs * v[c];
+      if (p.r == 8) {
+        const float4* tr = reinterpret_cast<const float4*>(p.t + static_cast<int64_t>(m) * 8);
+        const float4 t0 = __ldg(tr), t1 = __ldg(tr + 1);
+        out = fmaf(t0.x, u8[0], out);
+        out = fmaf(t0.y, u8[1], out);
+        out = fmaf(t0.z, u8[2], out);
+        out = fmaf(t0.w, u8[3], out);
+        out = fmaf(t1.x, u8[4], out);
+        out = fmaf(t1.y, u8[5], out);
+        out = fmaf(t1.z, u8[6], out);
+        out = fmaf(t1.w, u8[7], out);
+      } else if (p.r > 0) {
+        const float* tr = p.t + static_cast<int64_t>(m) * p.r;
+        const __half* ur = p.U + static_cast<int64_t>(n) * p.r;
+        for (int j = 0; j < p.r; ++j) out = fmaf(__ldg(tr + j), __half2float(__ldg(ur + j)), out);
+      }
+      if (p.ydt == ZQ_OUT_F32)
+        static_cast<float*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = out;
+      else
+        static_cast<__nv_bfloat16*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = __float2bfloat16_rn(out);
+    }
+  }
+}
+
+template <int BM, bool NONE>
+__global__ void __launch_bounds__(kThreads, NONE ? 1 : 2)
+w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_codes, const __grid_constant__ CUtensorMap tm_q,
+                 const Params p) {
+  using C = Cfg<BM, NONE>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint8_t* s_wide = smem + C::offWide;
+  uint8_t* s_tok = smem + C::offTok;
+  uint8_t* s_packed = smem + C::offPacked;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offBars);
+  uint64_t* tma_full = bars;
+  uint64_t* tma_empty = bars + C::NS;
+  uint64_t* wide_full = bars + 2 * C::NS;
+  uint64_t* wide_empty = bars + 2 * C::NS + C::NW;
+  uint64_t* acc_full = bars + 2 * C::NS + 2 * C::NW;      // [2]
+  uint64_t* acc_empty = acc_full + 2;                     // [2]
+  uint64_t* drain_bar = acc_full + 4;                     // [1]
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::offMisc);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::offMisc + 4);
+  int* s_last = reinterpret_cast<int*>(smem + C::offMisc + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * BM;
+  const int kb0 = blockIdx.z * p.kb_per_split;
+  const int nkb = min(p.kb_per_split, p.kblocks - kb0);
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < C::NS; ++i) {
+      mbar_init(&tma_full[i], 1);
+      mbar_init(&tma_empty[i], 1);
+    }
+    for (int i = 0; i < C::NW; ++i) {
+      mbar_init(&wide_full[i], C::kWidenThreads);
+      mbar_init(&wide_empty[i], 1);
+    }
+    mbar_init(&acc_full[0], 1);
+    mbar_init(&acc_full[1], 1);
+    mbar_init(&acc_empty[0], 128);
+    mbar_init(&acc_empty[1], 128);
+    mbar_init(drain_bar, 1);
+    *s_abort = 0;
+    *s_last = 0;
+    fence_mbar_init();
+    if ((smem_u32(smem) & 1023u) != 0) raise_error(p, s_abort, kErrAlign);
+  }
+  if (warp == 8 && lane == 0) {
+    prefetch_tensormap(&tm_codes);
+    prefetch_tensormap(&tm_q);
+  }
+  if (warp == 9) tmem_alloc(s_tmem, C::kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *s_tmem;
+  const bool ok_start = (*s_abort == 0);
+
+  if (warp == 8) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0 && ok_start) {
+      int issued = 0;
+      for (int i = 0; i < nkb; ++i) {
+        const int s = i % C::NS;
+        const uint32_t ph = (i / C::NS) & 1;
+        if (!mbar_wait(&tma_empty[s], ph ^ 1, s_abort)) {
+          raise_error(p, s_abort, kErrProducer);
+          break;
+        }
+        mbar_arrive_expect_tx(&tma_full[s], kPackedBytes + C::kTokBytes);
+        tma_load_2d(s_packed + s * kPackedBytes, &tm_codes, (kb0 + i) * (kBlockK / 2), n0, &tma_full[s]);
+        tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, (kb0 + i) * kBlockK, m0, &tma_full[s]);
+        issued = i + 1;
+      }
+      // never leave with copies still in flight: wait (bounded) for the last phase issued per stage
+      for (int i = max(0, issued - C::NS); i < issued; ++i) {
+        const int s = i % C::NS;
+        uint32_t spin = 0;
+        while (!mbar_try_wait(&tma_full[s], (i / C::NS) & 1) && ++spin < kSpinLimit) {
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0 && ok_start) {
+      const uint32_t idesc = umma_idesc_e4m3(BM);
+      const int mpg = p.group / 32;  // MMAs per weight group (mode none)
+      int mma_count = 0;
+      bool failed = false;
+      for (int i = 0; i < nkb && !failed; ++i) {
+        const int s = i % C::NS, ws = i % C::NW;
+        if (!mbar_wait(&tma_full[s], (i / C::NS) & 1, s_abort) ||
+            !mbar_wait(&wide_full[ws], (i / C::NW) & 1, s_abort)) {
+          failed = true;
+          break;
+        }
+        tc_fence_after_sync();
+        const uint64_t adesc = umma_desc_k128(smem_u32(s_wide + ws * kWideBytes));
+        const uint64_t bdesc = umma_desc_k128(smem_u32(s_tok + s * C::kTokBytes));
+#pragma unroll
+        for (int k = 0; k < kBlockK / 32; ++k) {
+          uint32_t d_tmem = tmem_base;
+          uint32_t accumulate = (i > 0 || k > 0) ? 1u : 0u;
+          if (NONE) {
+            const int grp = mma_count / mpg, within = mma_count % mpg, b = grp & 1;
+            if (within == 0) {
+              if (!mbar_wait(&acc_empty[b], ((grp >> 1) & 1) ^ 1, s_abort)) {
+                failed = true;
+                break;
+              }
+              tc_fence_after_sync();
+            }
+            d_tmem = tmem_base + b * BM;
+            accumulate = within > 0 ? 1u : 0u;
+          }
+          umma_f8(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, accumulate);
+          ++mma_count;
+          if (NONE && (mma_count % mpg) == 0) umma_commit(&acc_full[((mma_count / mpg) - 1) & 1]);
+        }
+        if (failed) break;
+        umma_commit(&tma_empty[s]);
+        umma_commit(&wide_empty[ws]);
+      }
+      if (failed) {
+        raise_error(p, s_abort, kErrMma);
+        umma_commit(drain_bar);  // let the MMAs already issued finish before TMEM is released
+        uint32_t spin = 0;
+        while (!mbar_try_wait(drain_bar, 0) && ++spin < kSpinLimit) {
+        }
+      } else if (!NONE) {
+        umma_commit(&acc_full[0]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ widen / promote / epilogue
+    const int q4 = warp & 3, grpB = warp >> 2;  // TMEM lane quarter; 0 = group A, 1 = group B
+    const int row = q4 * 32 + lane;             // output channel within the tile = TMEM lane
+    const int n = n0 + row;
+    const bool n_ok = n < p.N;
+    const bool widen_role = NONE ? (grpB == 0) : true;
+    bool failed = !ok_start;
+
+    if (widen_role && !failed) {
+      // M1/M2: a thread widens half a row (64 codes); mode none: group A threads widen a whole row.
+      const int half = NONE ? 0 : grpB;
+      constexpr int kChunks = NONE ? 4 : 2;  // 16-byte packed chunks per thread
+      const uint32_t sw64 = (row >> 1) & 3;  // 64-byte swizzle of the packed tile (TMA wrote it)
+      const uint32_t sw128 = row & 7;        // 128-byte swizzle of the widened tile (the MMA reads it)
+      const uint32_t wide_row_off = (row >> 3) * 1024 + (row & 7) * 128;
+      const uint8_t* shift_row = (!NONE && n_ok) ? p.shift + static_cast<int64_t>(n) * p.G : nullptr;
+      uint32_t d_next = 0;
+      if (shift_row && nkb > 0) d_next = __ldg(shift_row + ((kb0 * kBlockK + half * 64) / p.group));
+      for (int i = 0; i < nkb; ++i) {
+        const int s = i % C::NS, ws = i % C::NW;
+        const uint32_t d = d_next;
+        if (shift_row && i + 1 < nkb) d_next = __ldg(shift_row + (((kb0 + i + 1) * kBlockK + half * 64) / p.group));
+        if (!mbar_wait(&tma_full[s], (i / C::NS) & 1, s_abort) ||
+            !mbar_wait(&wide_empty[ws], ((i / C::NW) & 1) ^ 1, s_abort)) {
+          raise_error(p, s_abort, kErrWiden);
+          failed = true;
+          break;
+        }
+        const uint32_t lut_lo = 0x3C383000u - d * 0x08080800u;
+        const uint32_t lut_hi = 0x4C484440u - d * 0x08080808u;
+        const uint8_t* prow = s_packed + s * kPackedBytes + row * 64;
+        uint8_t* wrow = s_wide + ws * kWideBytes + wide_row_off;
+        uint4 pk[kChunks];
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+          const uint32_t lc = half * 2 + c;  // logical 16-byte chunk of the packed row
+          pk[c] = *reinterpret_cast<const uint4*>(prow + ((lc ^ sw64) << 4));
+        }
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+          const uint32_t lc = half * 2 + c;
+          uint4 a, b;
+          widen32(pk[c], lut_lo, lut_hi, a, b);
+          *reinterpret_cast<uint4*>(wrow + (((2 * lc) ^ sw128) << 4)) = a;
+          *reinterpret_cast<uint4*>(wrow + (((2 * lc + 1) ^ sw128) << 4)) = b;
+        }
+        fence_proxy_async_smem();  // generic-proxy stores -> visible to the tensor core's async proxy
+        mbar_arrive(&wide_full[ws]);
+      }
+    }
+
+    // ---- accumulators -> registers -> y
+    const bool epi_role = NONE ? (grpB == 1) : true;
+    if (epi_role) {
+      constexpr int kMyCols = NONE ? BM : (BM >= 32 ? BM / 2 : 16);
+      const int col0 = NONE ? 0 : (BM >= 32 ? grpB * (BM / 2) : 0);
+      const bool has_cols = NONE ? true : (BM >= 32 || grpB == 0);
+      const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
+      const int tile_id = blockIdx.y * gridDim.x + blockIdx.x;
+      float* my_partial = p.partials + (static_cast<size_t>(tile_id) * p.splits + blockIdx.z) * (BM * kTileN);
+
+      float cs = 1.0f;
+      float u[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) u[e] = 0.0f;
+      if (!NONE && n_ok) cs = __ldg(p.scale + n);
+      if (p.r == 8 && n_ok) {
+        const uint4 h = __ldg(reinterpret_cast<const uint4*>(p.U + static_cast<int64_t>(n) * 8));
+        const uint32_t hw[4] = {h.x, h.y, h.z, h.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __half2 h2;
+          *reinterpret_cast<uint32_t*>(&h2) = hw[e];
+          const float2 f = __half22float2(h2);
+          u[2 * e] = f.x;
+          u[2 * e + 1] = f.y;
+        }
+      }
+
+      float run[NONE ? BM : 1];
+      if (NONE) {
+        // per-group promotion: run += S[n, g] * (this group's FP32 partial sum)
+#pragma unroll
+        for (int c = 0; c < BM; ++c) run[c] = 0.0f;
+        const int gpk = p.group / kBlockK > 0 ? p.group / kBlockK : 1;  // K blocks per group (group >= 128)
+        const int groups = (p.group >= kBlockK) ? nkb / gpk : nkb * (kBlockK / p.group);
+        const int g0 = (kb0 * kBlockK) / p.group;
+        const float* srow = n_ok ? p.scale + static_cast<int64_t>(n) * p.G : nullptr;
+        float S_next = (srow && groups > 0) ? __ldg(srow + g0) : 0.0f;
+        for (int g = 0; g < groups && !failed; ++g) {
+          const int b = g & 1;
+          const float S = S_next;
+          if (srow && g + 1 < groups) S_next = __ldg(srow + g0 + g + 1);
+          if (!mbar_wait(&acc_full[b], (g >> 1) & 1, s_abort)) {
+            raise_error(p, s_abort, kErrPromote);
+            failed = true;
+            break;
+          }
+          tc_fence_after_sync();
+#pragma unroll
+          for (int c = 0; c < BM; c += 16) {
+            float v[16];
+            tmem_ld16(t_lane + b * BM + c, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) run[c + e] = fmaf(S, v[e], run[c + e]);
+          }
+          tc_fence_before_sync();
+          mbar_arrive(&acc_empty[b]);
+        }
+      } else if (!failed) {
+        if (!mbar_wait(&acc_full[0], 0, s_abort)) {
+          raise_error(p, s_abort, kErrEpilogue);
+          failed = true;
+        }
+        tc_fence_after_sync();
+      }
+
+      if (p.splits == 1) {
+        if (!failed && has_cols) {
+#pragma unroll
+          for (int c = 0; c < kMyCols; c += 16) {
+            float v[16];
+            if (NONE) {
+#pragma unroll
+              for (int e = 0; e < 16; ++e) v[e] = run[c + e];
+            } else {
+              tmem_ld16(t_lane + col0 + c, v);
+              tmem_ld_wait();
+            }
+            if (n_ok) finalize16(p, v, m0 + col0 + c, n, cs, u);
+          }
+        }
+      } else {
+        // split-K: leave the raw partial sums in the workspace; the CTA that arrives last for this
+        // output tile adds all of them in split order (deterministic) and finishes the tile.
+        if (!failed && has_cols) {
+#pragma unroll
+          for (int c = 0; c < kMyCols; c += 16) {
+            float v[16];
+            if (NONE) {
+#pragma unroll
+              for (int e = 0; e < 16; ++e) v[e] = run[c + e];
+            } else {
+              tmem_ld16(t_lane + col0 + c, v);
+              tmem_ld_wait();
+            }
+#pragma unroll
+            for (int e = 0; e < 16; ++e) my_partial[(col0 + c + e) * kTileN + row] = v[e];
+          }
+        }
+        __threadfence();
+        named_bar_sync(1, C::kEpiThreads);
+        const bool leader = NONE ? (threadIdx.x == 128) : (threadIdx.x == 0);
+        if (leader) {
+          const int ticket = (*s_abort) ? -1 : atomicAdd(p.counters + tile_id, 1);
+          *s_last = (ticket == p.splits - 1) ? 1 : 0;
+          if (ticket == p.splits - 1) p.counters[tile_id] = 0;  // ready for the next call
+        }
+        named_bar_sync(1, C::kEpiThreads);
+        if (*s_last && has_cols) {
+          __threadfence();
+          const float* tile_partials = p.partials + static_cast<size_t>(tile_id) * p.splits * (BM * kTileN);
+#pragma unroll 1
+          for (int c = 0; c < kMyCols; c += 16) {
+            float v[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) v[e] = 0.0f;
+            for (int z = 0; z < p.splits; ++z) {
+              const float* src = tile_partials + static_cast<size_t>(z) * (BM * kTileN) + (col0 + c) * kTileN + row;
+#pragma unroll
+              for (int e = 0; e < 16; ++e) v[e] += __ldcg(src + e * kTileN);
+            }
+            if (n_ok) finalize16(p, v, m0 + col0 + c, n, cs, u);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, C::kTmemCols);
+  }
+}
+
+// ---- host ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(f);
+  });
+  return fn;
+}
+
+// 2-D u8 tensor [rows, row_bytes] -> tiles of box_rows x box_bytes, written to shared memory swizzled.
+bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t rows, uint32_t box_bytes,
+              uint32_t box_rows, CUtensorMapSwizzle sw) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {row_bytes, rows};
+  const cuuint64_t strides[1] = {row_bytes};
+  const cuuint32_t box[2] = {box_bytes, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BM, bool NONE>
+int launch_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStream_t st) {
+  using C = Cfg<BM, NONE>;
+  CUtensorMap tm_codes, tm_q;
+  if (!make_map(&tm_codes, a.codes, static_cast<uint64_t>(a.K / 2), static_cast<uint64_t>(a.N), kBlockK / 2, kTileN,
+                CU_TENSOR_MAP_SWIZZLE_64B) ||
+      !make_map(&tm_q, a.q, static_cast<uint64_t>(a.K), static_cast<uint64_t>(a.M), kBlockK, BM,
+                CU_TENSOR_MAP_SWIZZLE_128B))
+    return ZQ_ERR_CUDA;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] {
+    attr_err = cudaFuncSetAttribute(w4a8_gemm_kernel<BM, NONE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    C::kSmemBytes);
+  });
+  if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
+  dim3 grid(plan.n_tiles, plan.m_tiles, plan.splits);
+  w4a8_gemm_kernel<BM, NONE><<<grid, kThreads, C::kSmemBytes, st>>>(tm_codes, tm_q, p);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+}
+
+}  // namespace
+
+GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
+  GemmPlan pl{};
+  const int bm_max = (mode == ZQ_SCALE_NONE) ? 128 : 256;
+  int bm = 16;
+  while (bm < bm_max && bm < M) bm *= 2;
+  pl.bm = bm;
+  pl.m_tiles = static_cast<int>((M + bm - 1) / bm);
+  pl.n_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
+  const int64_t tiles = static_cast<int64_t>(pl.m_tiles) * pl.n_tiles;
+  const int kblocks = static_cast<int>(K / kBlockK);
+  // split K until about two CTAs per SM are in flight, keeping at least 4 K blocks per CTA and (for
+  // 256-wide groups) whole groups per CTA
+  int splits = 1;
+  const int64_t target = 2 * 148;
+  if (tiles < target && tiles <= kWsMaxTiles) {
+    splits = static_cast<int>((target + tiles - 1) / tiles);
+    const int max_splits = kblocks / 4 > 0 ? kblocks / 4 : 1;
+    if (splits > max_splits) splits = max_splits;
+  }
+  int kbps = (kblocks + splits - 1) / splits;
+  if (kbps % 2) ++kbps;  // whole 256-element groups per split
+  if (kbps > kblocks) kbps = kblocks;
+  splits = (kblocks + kbps - 1) / kbps;
+  pl.splits = splits;
+  pl.kb_per_split = kbps;
+  pl.partial_floats = splits > 1 ? static_cast<size_t>(tiles) * splits * bm * kTileN : 0;
+  return pl;
+}
+
+int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st) {
+  const GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode);
+  if (plan.partial_floats > a.partial_floats) return ZQ_ERR_WORKSPACE;
+  Params p{};
+  p.M = static_cast<int>(a.M);
+  p.N = static_cast<int>(a.N);
+  p.K = static_cast<int>(a.K);
+  p.group = a.group;
+  p.G = static_cast<int>(a.K / a.group);
+  p.kblocks = static_cast<int>(a.K / kBlockK);
+  p.splits = plan.splits;
+  p.kb_per_split = plan.kb_per_split;
+  p.shift = a.shift;
+  p.scale = a.scale;
+  p.sx = a.sx;
+  p.U = static_cast<const __half*>(a.U);
+  p.t = a.t;
+  p.r = a.U ? a.r : 0;
+  p.y = a.y;
+  p.ydt = a.ydt;
+  p.ldy = a.ldy;
+  p.status = a.status;
+  p.counters = a.counters;
+  p.partials = a.partials;
+  const bool none = a.mode == ZQ_SCALE_NONE;
+  switch (plan.bm) {
+    case 16: return none ? launch_cfg<16, true>(a, plan, p, st) : launch_cfg<16, false>(a, plan, p, st);
+    case 32: return none ? launch_cfg<32, true>(a, plan, p, st) : launch_cfg<32, false>(a, plan, p, st);
+    case 64: return none ? launch_cfg<64, true>(a, plan, p, st) : launch_cfg<64, false>(a, plan, p, st);
+    case 128: return none ? launch_cfg<128, true>(a, plan, p, st) : launch_cfg<128, false>(a, plan, p, st);
+    case 256: return none ? ZQ_ERR_SHAPE : launch_cfg<256, false>(a, plan, p, st);
+  }
+  return ZQ_ERR_SHAPE;
+}
+
+}  // namespace zq

@@ -48,6 +48,7 @@ struct GemmArgs {
 struct GemmPlan {
   int bm;      // tokens per tile (the MMA's N extent)
   int splits;  // split-K factor
+  int kb_per_split;  // 128-element K blocks per split
   int m_tiles, n_tiles;
   size_t partial_floats;
 };
