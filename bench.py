@@ -138,10 +138,10 @@ def oracle_sample_step(wl, state=None, M_s=8):
 def cpu_baseline(wl):
     import oracle
 
-    dt, fl, _ = oracle_sample_step(wl)
+    dt, fl, _ = oracle_sample_step(wl, M_s=32)
     shape = wl.shapes[0]
     return {"value": fl / dt / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{wl.name} {shape.K}->{shape.N}: first 8 tokens, all {shape.N} outputs, quantizer + LoRC + "
+            "sample": f"{wl.name} {shape.K}->{shape.N}: first 32 tokens, all {shape.N} outputs, quantizer + LoRC + "
                       f"FP64 linear, {dt:.1f} s"}
 
 
