@@ -147,6 +147,33 @@ int zq_w4a8_linear_host(const void* x_bf16_host, int64_t M, int64_t N, int64_t K
  */
 int zq_device_status(void* workspace, int* detail, void* stream);
 
+/*
+ * (The paper has no counterpart for this entry point; it exists for deployment reasons only.)
+ *
+ * zq_w4a8_linear for callers that cannot allocate device memory and therefore have no workspace to
+ * hand over: a serving loop whose memory plan is fixed at start-up, a plug-in that receives tensors
+ * from a host framework but owns no allocator, a process whose pool already holds the whole device.
+ * The split-K counters and partial sums live in a fixed 32 MiB array inside the library
+ * (zq_w4a8_linear_noalloc_max_scratch_bytes), resident on every GPU that loads the library until the
+ * process exits.  The call allocates and frees nothing.
+ *
+ * Same operation, arguments and limits as zq_w4a8_linear with pre-quantized activations (q, sx, and
+ * t when r > 0; there is no raw-x path, since that would need scratch for q).  The fixed array bounds
+ * the split-K partial sums (4 bytes x splits x padded M x padded N).  A problem that needs more
+ * returns ZQ_ERR_WORKSPACE and launches nothing.  Problems with about 300 or more 128 x 256 output
+ * tiles are not split and always fit; so do the M <= 128 cases of layers up to 28672 x 28672.
+ * The first call on a device looks up the array's device address (once per device, with that device
+ * current); make that first call outside any stream capture.
+ * Every call on a device shares the one array: the call clears the status words and counters it needs
+ * at zero, but two calls that overlap on the GPU race on it, so issue them on one stream or
+ * serialize them yourself.
+ */
+size_t zq_w4a8_linear_noalloc_max_scratch_bytes(void);
+int zq_w4a8_linear_noalloc(const uint8_t* q, const float* sx, int64_t M, int64_t N, int64_t K, int group,
+                           zq_scale_mode mode, const uint8_t* codes, const uint8_t* shift,
+                           const float* scale, const void* U_f16, const float* t, int r, void* y,
+                           zq_out_dtype ydt, int64_t ldy, void* stream);
+
 /* Number of kernels of this library launched by the calling process so far (all entry points). */
 int64_t zq_launch_count(void);
 

@@ -23,6 +23,7 @@ EXPORTS = [
     "zq_status_string", "zq_quantize_act_fp8", "zq_packed_weight_sizes", "zq_pack_weight_fp4",
     "zq_w4a8_linear_workspace_bytes", "zq_workspace_init", "zq_w4a8_linear",
     "zq_w4a8_linear_host_workspace_bytes", "zq_w4a8_linear_host", "zq_device_status", "zq_launch_count",
+    "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc",
 ]
 
 
@@ -66,6 +67,10 @@ def lib() -> C.CDLL:
         L.zq_device_status.argtypes = [vp, C.POINTER(ci), vp]
         L.zq_launch_count.restype = i64
         L.zq_launch_count.argtypes = []
+        L.zq_w4a8_linear_noalloc_max_scratch_bytes.restype = sz
+        L.zq_w4a8_linear_noalloc_max_scratch_bytes.argtypes = []
+        L.zq_w4a8_linear_noalloc.restype = ci
+        L.zq_w4a8_linear_noalloc.argtypes = [vp, vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, ci, vp, ci, i64, vp]
         _lib = L
     return _lib
 
@@ -168,6 +173,23 @@ def w4a8_linear(codes, shift, scale, group: int, mode, *, q=None, sx=None, t=Non
     _check(lib().zq_w4a8_linear(_ptr(q), _ptr(sx), _ptr(x), ldx, M, N, K, group, _mode(mode), _ptr(codes), _ptr(shift),
                                 _ptr(scale), _ptr(U), _ptr(V), _ptr(t), r, _ptr(y), ydt, ldy, _ptr(workspace),
                                 workspace.numel(), _stream()), "zq_w4a8_linear")
+    return y
+
+
+def w4a8_linear_noalloc(codes, shift, scale, group: int, mode, *, q, sx, t=None, U=None, y=None,
+                        out_dtype=torch.float32):
+    """``zq_w4a8_linear_noalloc``: same result as :func:`w4a8_linear` on pre-quantized activations, for
+    callers that cannot allocate a workspace; the scratch is a fixed array inside the library."""
+    N, K = codes.shape[0], codes.shape[1] * 2
+    M = q.shape[0]
+    r = 0 if U is None else U.shape[1]
+    if y is None:
+        y = torch.empty((M, N), dtype=out_dtype, device=codes.device)
+    ydt = OUT_F32 if y.dtype == torch.float32 else OUT_BF16
+    ldy = y.stride(0) if M > 1 else N
+    _check(lib().zq_w4a8_linear_noalloc(_ptr(q), _ptr(sx), M, N, K, group, _mode(mode), _ptr(codes), _ptr(shift),
+                                        _ptr(scale), _ptr(U), _ptr(t), r, _ptr(y), ydt, ldy, _stream()),
+           "zq_w4a8_linear_noalloc")
     return y
 
 
