@@ -211,21 +211,29 @@ def run_ours(args):
 
     wl = synth.WORKLOADS[WORKLOAD]
     Ms = list(wl.Ms)
+    shapes = list(wl.shapes)
+    mode = MODE
+    if args.case:
+        parts = args.case.split(",")
+        shapes = [synth.LayerShape(int(parts[0]), int(parts[1]), "case")]
+        Ms = [int(parts[2])]
+        if len(parts) > 3:
+            mode = parts[3]
     Mmax = max(Ms)
     layers = []
-    for shape in wl.shapes:
+    for shape in shapes:
         K, N = shape.K, shape.N
         # replicas draw their own activations (row_offset = rank); weights are the same model on every rank
         x_bits = synth.make_x(wl.seed, Mmax, K, wl.n_outliers(K), wl.outlier_factor, row_offset=rank)
         x = torch.from_numpy(x_bits.view(np.int16)).to(dev).view(torch.bfloat16)
         W = torch.from_numpy(synth.make_w(wl.seed, N, K, wl.sigma_w)).to(dev)
-        codes, shift, scale = binding.pack_weight_fp4(W, GROUP, MODE)
+        codes, shift, scale = binding.pack_weight_fp4(W, GROUP, mode)
         del W
         U_h, V_h = synth.make_lorc(wl.seed, N, K, RANK)
         U, V = torch.from_numpy(U_h).to(dev), torch.from_numpy(V_h).to(dev)
         copies = [(codes, shift, scale)]
         for _ in range(N_WEIGHT_COPIES - 1):
-            copies.append((codes.clone(), shift.clone(), scale.clone()))
+            copies.append((codes.clone(), None if shift is None else shift.clone(), scale.clone()))
         ws = binding.make_workspace(binding.linear_workspace_bytes(Mmax, N, K, RANK), dev)
         layers.append(dict(K=K, N=N, x=x, x_bits=x_bits, U=U, V=V, copies=copies, ws=ws,
                            q=torch.empty((Mmax, K), dtype=torch.uint8, device=dev),
@@ -238,7 +246,7 @@ def run_ours(args):
     import ctypes as C
 
     def vp(t):
-        return C.c_void_p(t.data_ptr())
+        return None if t is None else C.c_void_p(t.data_ptr())
 
     stream = torch.cuda.current_stream()
     sp = C.c_void_p(stream.cuda_stream)
@@ -253,7 +261,7 @@ def run_ours(args):
         rc = L.zq_quantize_act_fp8(vp(ly["x"]), M, K, K, vp(ly["q"]), vp(ly["sx"]), vp(ly["V"]), RANK, vp(ly["t"]), sp)
         if ev:
             ev[1].record(stream)
-        rc |= L.zq_w4a8_linear(vp(ly["q"]), vp(ly["sx"]), None, 0, M, N, K, GROUP, binding.MODES[MODE], vp(codes),
+        rc |= L.zq_w4a8_linear(vp(ly["q"]), vp(ly["sx"]), None, 0, M, N, K, GROUP, binding.MODES[mode], vp(codes),
                                vp(shift), vp(scale), vp(ly["U"]), None, vp(ly["t"]), RANK, vp(ly["y"]), 0, N,
                                vp(ly["ws"]), ly["ws"].numel(), sp)
         if ev:
@@ -322,13 +330,13 @@ def run_ours(args):
     roofline = {"bound": "tensor", "kernel": "w4a8_gemm_kernel<256,false>", "achieved": round(achieved, 1),
                 "peak": round(fp8_peak, 1), "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4), "traffic": None,
                 "peak_source": f"2 x bf16 sustained cuBLAS peak ({peaks['source']}); nominal dense FP8 4500"}
-    dec = [s for s in sweep if s["M"] <= 16]
+    dec = [s for s in sweep if s["M"] <= 16] or [sweep[0]]
     roofline_decode = {"bound": "hbm", "kernel": "w4a8_gemm_kernel<16,false>",
                        "achieved": round(statistics.mean(s["gemm_gbs"] for s in dec), 1),
                        "peak": peaks["hbm_gbs"], "unit": "GB/s",
                        "frac": round(statistics.mean(s["frac_hbm"] for s in dec), 4), "traffic": None,
                        "peak_source": f"copy bandwidth ({peaks['source']}); nominal 7700-8000"}
-    big_q = [s for s in sweep if s["M"] == Mmax and s["layer"].startswith("28672")]
+    big_q = [s for s in sweep if s["M"] == Mmax and s["layer"].startswith("28672")] or [sweep[-1]]
     roofline_quant = {"bound": "hbm", "kernel": "act_quant_kernel<true>", "achieved": big_q[0]["quant_gbs"],
                       "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(big_q[0]["quant_gbs"] / peaks["hbm_gbs"], 4),
                       "traffic": None}
@@ -350,7 +358,7 @@ def run_ours(args):
                 ly = layers[li]
                 xh, yh, wsh = hosts[li]
                 codes, shift, scale = ly["copies"][(idx + ci // len(layers)) % N_WEIGHT_COPIES]
-                rc = L.zq_w4a8_linear_host(C.c_void_p(xh.data_ptr()), M, ly["N"], ly["K"], GROUP, binding.MODES[MODE],
+                rc = L.zq_w4a8_linear_host(C.c_void_p(xh.data_ptr()), M, ly["N"], ly["K"], GROUP, binding.MODES[mode],
                                            vp(codes), vp(shift), vp(scale), vp(ly["U"]), vp(ly["V"]), RANK,
                                            C.c_void_p(yh.data_ptr()), vp(wsh), wsh.numel(), sp)
                 if rc:
@@ -381,8 +389,8 @@ def run_ours(args):
     line = {"metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms_max / args.steps, 4), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f8e4m3 x f8e4m3 -> f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "layers": [f"{s.K}->{s.N}" for s in wl.shapes], "M": Ms, "group": GROUP,
-                       "mode": MODE, "lorc_rank": RANK, "multi_gpu": "independent replicas",
+            "config": {"workload": WORKLOAD if not args.case else f"case {args.case}",
+                       "layers": [f"{s.K}->{s.N}" for s in shapes], "M": Ms, "group": GROUP, "mode": mode, "lorc_rank": RANK, "multi_gpu": "independent replicas",
                        "l2": f"inputs larger than L2: {N_WEIGHT_COPIES} weight copies per layer rotated, >300 MB "
                              "streamed between two reads of one buffer"},
             "roofline": roofline, "roofline_decode": roofline_decode, "roofline_quant": roofline_quant,
@@ -400,6 +408,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--case", default=None, metavar="K,N,M[,MODE]",
+                    help="time one layer shape at one token count instead of the sweep (profiling aid)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
