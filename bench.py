@@ -227,13 +227,14 @@ def run_ours(args):
         x_bits = synth.make_x(wl.seed, Mmax, K, wl.n_outliers(K), wl.outlier_factor, row_offset=rank)
         x = torch.from_numpy(x_bits.view(np.int16)).to(dev).view(torch.bfloat16)
         W = torch.from_numpy(synth.make_w(wl.seed, N, K, wl.sigma_w)).to(dev)
-        codes, shift, scale = binding.pack_weight_fp4(W, GROUP, mode)
+        pw = binding.pack_weight_fp4(W, GROUP, mode)
         del W
         U_h, V_h = synth.make_lorc(wl.seed, N, K, RANK)
         U, V = torch.from_numpy(U_h).to(dev), torch.from_numpy(V_h).to(dev)
-        copies = [(codes, shift, scale)]
+        copies = [(pw.codes, pw.shift, pw.scale)]
         for _ in range(N_WEIGHT_COPIES - 1):
-            copies.append((codes.clone(), None if shift is None else shift.clone(), scale.clone()))
+            c = pw.clone()
+            copies.append((c.codes, c.shift, c.scale))
         ws = binding.make_workspace(binding.linear_workspace_bytes(Mmax, N, K, RANK), dev)
         layers.append(dict(K=K, N=N, x=x, x_bits=x_bits, U=U, V=V, copies=copies, ws=ws,
                            q=torch.empty((Mmax, K), dtype=torch.uint8, device=dev),

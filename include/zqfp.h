@@ -63,7 +63,8 @@ int zq_quantize_act_fp8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, u
 
 /*
  * Sizes in bytes of the three buffers zq_pack_weight_fp4 writes:
- *   codes: N*K/2 ; shift: N*G (M1, M2) or 0 (none) ; scale: 4*N (M1, M2) or 4*N*G (none).
+ *   codes: ceil(N/128) * (K/128) * 8448 (tiled, see below) ; shift: N*G (M1, M2) or 0 (none) ;
+ *   scale: 4*N (M1, M2) or 4*N*G (none).
  */
 int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, size_t* codes_bytes,
                            size_t* shift_bytes, size_t* scale_bytes);
@@ -84,10 +85,18 @@ int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, 
  * part in the row maximum, gets shift 0 (and scale 1 in mode none).
  *
  * W     : FP32 [N, K] dense row-major; 16-byte aligned
- * codes : out, [N, K/2]; byte b of a row = element 2b in bits 0..3, element 2b+1 in bits 4..7
- * shift : out, u8 [N, G] (M1, M2); ignored (may be NULL) in mode none
+ * codes : out, 16-byte aligned, in the layout the GEMM streams (the paper does not fix one): tiles of
+ *         128 output rows x 128 input features, tile (nt, kb) at byte offset (nt * (K/128) + kb) * 8448.
+ *         A tile is 8192 bytes of codes followed by 256 shift bytes:
+ *           - the 16-byte chunk c (elements 32c .. 32c+31 of the K block) of row r sits at (c*128 + r)*16;
+ *             its 32-bit word j holds elements 8j .. 8j+7: bits 4i .. 4i+2 = the three E2M1 magnitude
+ *             bits (e1 e0 m) of element i, bit 8b+7 = sign of element b, bit 8b+3 = sign of element 4+b
+ *             (b = 0..3);
+ *           - byte 8192 + 2r + h = the shift of row r for elements 64h .. 64h+63 (0 in mode none).
+ *         Rows of the last tile beyond N are zero.
+ * shift : out, u8 [N, G] (M1, M2), the same shifts in plain form; ignored (may be NULL) in mode none
  * scale : out, FP32 [N] (M1, M2) or [N, G] (none)
- * group in {64, 128, 256}; K % group == 0; N >= 0.
+ * group in {64, 128, 256}; K % group == 0 and K % 128 == 0; N >= 0.
  */
 int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale_mode mode,
                        uint8_t* codes, uint8_t* shift, float* scale, void* stream);
@@ -114,7 +123,8 @@ int zq_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  * (x_bf16 [M, ldx] given, q = sx = t = NULL): then the call first runs zq_quantize_act_fp8 into the
  * workspace (with V when r > 0).
  *
- * codes / shift / scale : as written by zq_pack_weight_fp4 for the same (N, K, group, mode)
+ * codes / scale : as written by zq_pack_weight_fp4 for the same (N, K, group, mode); shift is not read
+ *                 (the tiles carry the shifts) and may be NULL
  * U : fp16 [N, r] dense or NULL (r = 0);  V : fp16 [r, K], only read when x_bf16 is given and r > 0
  * y : out, [M, ldy] FP32 or bf16 (ydt), ldy >= N in elements
  * K % 128 == 0; group in {64, 128, 256}; r in {0, 8, 16, ..., 64}; q, codes 16-byte aligned.

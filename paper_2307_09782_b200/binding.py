@@ -8,6 +8,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
+from dataclasses import dataclass
 from typing import Optional
 
 import torch
@@ -124,20 +125,36 @@ def quantize_act_fp8(x: torch.Tensor, V: Optional[torch.Tensor] = None):
     return q, sx, t
 
 
-def pack_weight_fp4(W: torch.Tensor, group: int, mode):
-    """W: float32 [N, K] contiguous.  Returns (codes uint8 [N,K/2], shift uint8 [N,G] | None, scale float32)."""
+@dataclass
+class PackedWeight:
+    """Device buffers written by ``zq_pack_weight_fp4`` plus the shape they were packed for."""
+    codes: torch.Tensor               # uint8, tiled layout (see include/zqfp.h)
+    shift: Optional[torch.Tensor]     # uint8 [N, G] (M1, M2) or None
+    scale: torch.Tensor               # float32 [N] (M1, M2) or [N, G] (none)
+    N: int
+    K: int
+    group: int
+    mode: int
+
+    def clone(self) -> "PackedWeight":
+        return PackedWeight(self.codes.clone(), None if self.shift is None else self.shift.clone(),
+                            self.scale.clone(), self.N, self.K, self.group, self.mode)
+
+
+def pack_weight_fp4(W: torch.Tensor, group: int, mode) -> PackedWeight:
+    """W: float32 [N, K] contiguous."""
     assert W.dtype == torch.float32 and W.is_contiguous() and W.dim() == 2
     N, K = W.shape
     mode = _mode(mode)
     cb, sb, fb = packed_weight_sizes(N, K, group, mode)
     G = K // group
-    codes = torch.empty((N, K // 2), dtype=torch.uint8, device=W.device)
+    codes = torch.empty((cb,), dtype=torch.uint8, device=W.device)
     shift = None if mode == SCALE_NONE else torch.empty((N, G), dtype=torch.uint8, device=W.device)
     scale = torch.empty((N, G) if mode == SCALE_NONE else (N,), dtype=torch.float32, device=W.device)
-    assert codes.numel() == cb and scale.numel() * 4 == fb and (shift is None or shift.numel() == sb)
+    assert scale.numel() * 4 == fb and (shift is None or shift.numel() == sb)
     _check(lib().zq_pack_weight_fp4(_ptr(W), N, K, group, mode, _ptr(codes), _ptr(shift), _ptr(scale), _stream()),
            "zq_pack_weight_fp4")
-    return codes, shift, scale
+    return PackedWeight(codes, shift, scale, N, K, group, mode)
 
 
 def linear_workspace_bytes(M: int, N: int, K: int, r: int) -> int:
@@ -155,10 +172,10 @@ def make_workspace(nbytes: int, device="cuda") -> torch.Tensor:
     return ws
 
 
-def w4a8_linear(codes, shift, scale, group: int, mode, *, q=None, sx=None, t=None, x=None, U=None, V=None,
+def w4a8_linear(w: PackedWeight, *, q=None, sx=None, t=None, x=None, U=None, V=None,
                 out_dtype=torch.float32, workspace: Optional[torch.Tensor] = None, y=None):
     """y [M, N] = the quantized linear layer; activations either (q, sx[, t]) or raw bf16 ``x`` (then V when U)."""
-    N, K = codes.shape[0], codes.shape[1] * 2
+    codes, shift, scale, group, mode, N, K = w.codes, w.shift, w.scale, w.group, w.mode, w.N, w.K
     if x is not None:
         M, ldx = x.shape[0], (x.stride(0) if x.shape[0] > 1 else K)
     else:
@@ -176,11 +193,10 @@ def w4a8_linear(codes, shift, scale, group: int, mode, *, q=None, sx=None, t=Non
     return y
 
 
-def w4a8_linear_noalloc(codes, shift, scale, group: int, mode, *, q, sx, t=None, U=None, y=None,
-                        out_dtype=torch.float32):
+def w4a8_linear_noalloc(w: PackedWeight, *, q, sx, t=None, U=None, y=None, out_dtype=torch.float32):
     """``zq_w4a8_linear_noalloc``: same result as :func:`w4a8_linear` on pre-quantized activations, for
     callers that cannot allocate a workspace; the scratch is a fixed array inside the library."""
-    N, K = codes.shape[0], codes.shape[1] * 2
+    codes, shift, scale, group, mode, N, K = w.codes, w.shift, w.scale, w.group, w.mode, w.N, w.K
     M = q.shape[0]
     r = 0 if U is None else U.shape[1]
     if y is None:
@@ -193,12 +209,13 @@ def w4a8_linear_noalloc(codes, shift, scale, group: int, mode, *, q, sx, t=None,
     return y
 
 
-def w4a8_linear_host(x_host: torch.Tensor, y_host: torch.Tensor, codes, shift, scale, group: int, mode, *, U=None,
-                     V=None, workspace: torch.Tensor):
+def w4a8_linear_host(x_host: torch.Tensor, y_host: torch.Tensor, w: PackedWeight, *, U=None, V=None,
+                     workspace: torch.Tensor):
     """Host-buffer variant: x_host bf16 [M,K] and y_host float32 [M,N] are CPU (pinned) tensors; synchronous."""
     assert not x_host.is_cuda and not y_host.is_cuda and x_host.is_contiguous() and y_host.is_contiguous()
+    codes, shift, scale, group, mode, N = w.codes, w.shift, w.scale, w.group, w.mode, w.N
     M, K = x_host.shape
-    N = codes.shape[0]
+    assert K == w.K
     r = 0 if U is None else U.shape[1]
     _check(lib().zq_w4a8_linear_host(_ptr(x_host), M, N, K, group, _mode(mode), _ptr(codes), _ptr(shift),
                                      _ptr(scale), _ptr(U), _ptr(V), r, _ptr(y_host), _ptr(workspace),

@@ -102,9 +102,10 @@ int zq_quantize_act_fp8(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_
 int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, size_t* codes_bytes,
                            size_t* shift_bytes, size_t* scale_bytes) {
   if (!valid_mode(mode)) return ZQ_ERR_MODE;
-  if (N < 0 || K <= 0 || !valid_group(group) || K % group) return ZQ_ERR_SHAPE;
+  if (N < 0 || K <= 0 || !valid_group(group) || K % group || K % kTileK) return ZQ_ERR_SHAPE;
   const size_t G = static_cast<size_t>(K / group);
-  if (codes_bytes) *codes_bytes = static_cast<size_t>(N) * (K / 2);
+  if (codes_bytes)
+    *codes_bytes = static_cast<size_t>((N + kTileRows - 1) / kTileRows) * static_cast<size_t>(K / kTileK) * kTileBytes;
   if (shift_bytes) *shift_bytes = mode == ZQ_SCALE_NONE ? 0 : static_cast<size_t>(N) * G;
   if (scale_bytes) *scale_bytes = mode == ZQ_SCALE_NONE ? static_cast<size_t>(N) * G * 4 : static_cast<size_t>(N) * 4;
   return ZQ_OK;
@@ -113,11 +114,12 @@ int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, 
 int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale_mode mode, uint8_t* codes,
                        uint8_t* shift, float* scale, void* stream) {
   if (!valid_mode(mode)) return ZQ_ERR_MODE;
-  if (N < 0 || K <= 0 || !valid_group(group) || K % group || N > 0x7FFFFFFF || K > (int64_t(1) << 30))
+  if (N < 0 || K <= 0 || !valid_group(group) || K % group || K % kTileK || N > 0x7FFFFFFF - kTileRows ||
+      K > (int64_t(1) << 30))
     return ZQ_ERR_SHAPE;
   if (N == 0) return ZQ_OK;
   if (!W || !codes || !scale || (mode != ZQ_SCALE_NONE && !shift)) return ZQ_ERR_NULL;
-  if (!aligned16(W) || (reinterpret_cast<uintptr_t>(codes) & 3u)) return ZQ_ERR_ALIGN;
+  if (!aligned16(W) || !aligned16(codes)) return ZQ_ERR_ALIGN;
   if (int e = check_device_sm100()) return e;
   return launch_pack_weight(W, N, K, group, mode, codes, shift, scale, static_cast<cudaStream_t>(stream));
 }
@@ -149,7 +151,7 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
       ldy < N || M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > (int64_t(1) << 30))
     return ZQ_ERR_SHAPE;
   if (M == 0 || N == 0) return ZQ_OK;
-  if (!codes || !scale || !y || (mode != ZQ_SCALE_NONE && !shift) || (r > 0 && !U)) return ZQ_ERR_NULL;
+  if (!codes || !scale || !y || (r > 0 && !U)) return ZQ_ERR_NULL;
   if (x_bf16) {
     if (r > 0 && !V) return ZQ_ERR_NULL;
     if (ldx < K) return ZQ_ERR_SHAPE;

@@ -62,7 +62,7 @@ int zq_w4a8_linear_noalloc(const uint8_t* q, const float* sx, int64_t M, int64_t
       r > 64 || r % 8 || ldy < N || M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > (int64_t(1) << 30))
     return ZQ_ERR_SHAPE;
   if (M == 0 || N == 0) return ZQ_OK;
-  if (!q || !sx || !codes || !scale || !y || (mode != ZQ_SCALE_NONE && !shift) || (r > 0 && (!U || !t)))
+  if (!q || !sx || !codes || !scale || !y || (r > 0 && (!U || !t)))
     return ZQ_ERR_NULL;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(codes) | reinterpret_cast<uintptr_t>(U) |
        reinterpret_cast<uintptr_t>(t)) & 15u)

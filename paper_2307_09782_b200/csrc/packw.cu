@@ -1,11 +1,13 @@
 // Fine-grained FP4-E2M1 weight quantizer and packer with the scale constraints none / M1 / M2.
 // Section 3 (FGQ; "Casting the FP4 to FP8", items M1 and M2), Appendix A (group size).
 //
-// One CTA per output row.  Pass 1: each warp reduces the absmax of its groups and leaves the group
-// scale in shared memory.  Then the row-wide quantity of the constrained modes (largest exponent for
-// M1, largest scale for M2) is reduced.  Pass 2 re-reads the row (it is still in L2), divides,
-// rounds to E2M1 and writes two codes per byte.  All scale decisions use the bits of the FP32 scale,
-// never a logarithm.
+// One CTA per output row (rows of the last, partial tile beyond N are written as zeros).  A lane
+// owns 8 consecutive elements, i.e. one 32-bit word of packed codes.  Pass 1 reduces the absmax of
+// every group (segmented warp shuffle) and leaves the group scales in shared memory; then the
+// row-wide quantity of the constrained modes (largest exponent for M1, largest scale for M2) is
+// reduced; pass 2 re-reads the row (still in L2), divides, rounds to E2M1 and writes the codes in
+// the tiled layout the GEMM streams.  All scale decisions use the bits of the FP32 scale, never a
+// logarithm.
 #include <limits.h>
 
 #include "zq_common.cuh"
@@ -29,36 +31,50 @@ __device__ __forceinline__ void exp_frac(float s, int* e, uint32_t* f) {
   *f = b & 0x7FFFFFu;
 }
 
-// Round to nearest E2M1 magnitude, ties to the code with mantissa bit 0, saturating at 6; sign kept.
-__device__ __forceinline__ uint32_t encode_e2m1(float v) {
+// Round to nearest E2M1 magnitude, ties to the code with mantissa bit 0, saturating at 6.
+// Returns the 3 magnitude bits; the sign is taken from the quotient separately.
+__device__ __forceinline__ uint32_t e2m1_magnitude(float v) {
   const float a = fabsf(v);
-  const uint32_t m = (a > 0.25f) + (a >= 0.75f) + (a > 1.25f) + (a >= 1.75f) + (a > 2.5f) + (a >= 3.5f) + (a > 5.0f);
-  return m | ((__float_as_uint(v) >> 31) << 3);
+  return (a > 0.25f) + (a >= 0.75f) + (a > 1.25f) + (a >= 1.75f) + (a > 2.5f) + (a >= 3.5f) + (a > 5.0f);
 }
 
-template <int EPL>  // elements per lane = group / 32
+template <int GROUP>
 __global__ void __launch_bounds__(kThreads)
-pack_weight_kernel(const float* __restrict__ W, int K, int G, int mode, uint8_t* __restrict__ codes,
+pack_weight_kernel(const float* __restrict__ W, int N, int K, int mode, uint8_t* __restrict__ tiles,
                    uint8_t* __restrict__ shift, float* __restrict__ scale) {
   extern __shared__ float s_S[];  // [G] unconstrained group scales (0 = all-zero group)
   __shared__ int s_red_i[kWarps];
   __shared__ float s_red_f[kWarps];
-  const int64_t n = blockIdx.x;
-  const float* row = W + n * static_cast<int64_t>(K);
+  constexpr int LPG = GROUP / 8;  // lanes per group
+  const int n = blockIdx.x;
+  const int G = K / GROUP;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int group = EPL * 32;
+  const int kblocks = K / kTileK;
+  uint8_t* tile_row = tiles + static_cast<int64_t>(n / kTileRows) * kblocks * kTileBytes;
+  const int r = n % kTileRows;
 
-  for (int j = warp; j < G; j += kWarps) {
-    const float* p = row + static_cast<int64_t>(j) * group + lane * EPL;
-    float a = 0.0f;
-#pragma unroll
-    for (int i = 0; i < EPL; i += 2) {
-      const float2 v = __ldg(reinterpret_cast<const float2*>(p + i));
-      a = fmaxf(a, fmaxf(fabsf(v.x), fabsf(v.y)));
+  if (n >= N) {  // padding row of the last tile: zero codes and shifts
+    for (int k = threadIdx.x * 8; k < K; k += kThreads * 8) {
+      uint8_t* blk = tile_row + static_cast<int64_t>(k / kTileK) * kTileBytes;
+      const int within = k % kTileK;
+      *reinterpret_cast<uint32_t*>(blk + ((within / 32) * kTileRows + r) * 16 + ((within % 32) / 8) * 4) = 0u;
+      if (within % 64 == 0) blk[kTileCodeBytes + 2 * r + within / 64] = 0;
     }
+    return;
+  }
+  const float* row = W + static_cast<int64_t>(n) * K;
+
+  for (int kbase = warp * 256; kbase < K; kbase += kThreads * 8) {  // warp-uniform trip count
+    const int k = kbase + lane * 8;
+    const bool in = k < K;
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4 v0 = in ? __ldg(reinterpret_cast<const float4*>(row + k)) : zero4;
+    const float4 v1 = in ? __ldg(reinterpret_cast<const float4*>(row + k + 4)) : zero4;
+    float a = fmaxf(fmaxf(fmaxf(fabsf(v0.x), fabsf(v0.y)), fmaxf(fabsf(v0.z), fabsf(v0.w))),
+                    fmaxf(fmaxf(fabsf(v1.x), fabsf(v1.y)), fmaxf(fabsf(v1.z), fabsf(v1.w))));
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
-    if (lane == 0) s_S[j] = (a == 0.0f) ? 0.0f : __fdiv_rn(a, 6.0f);
+    for (int o = 1; o < LPG; o <<= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
+    if (in && (lane % LPG) == 0) s_S[k / GROUP] = (a == 0.0f) ? 0.0f : __fdiv_rn(a, 6.0f);
   }
   __syncthreads();
 
@@ -103,14 +119,15 @@ pack_weight_kernel(const float* __restrict__ W, int K, int G, int mode, uint8_t*
   uint32_t f_max = 0;
   if (mode == ZQ_SCALE_M2) exp_frac(Smax, &e_max, &f_max);
 
-  for (int j = warp; j < G; j += kWarps) {
+  for (int k = (warp * 32 + lane) * 8; k < K; k += kThreads * 8) {
+    const int j = k / GROUP;
     const float s = s_S[j];
     float shat;
+    int d = 0;
     if (mode == ZQ_SCALE_NONE) {
       shat = (s == 0.0f) ? 1.0f : s;
-      if (lane == 0) scale[n * G + j] = shat;
+      if ((k % GROUP) == 0) scale[static_cast<int64_t>(n) * G + j] = shat;
     } else {
-      int d = 0;
       if (s != 0.0f) {
         int e;
         uint32_t f;
@@ -120,20 +137,23 @@ pack_weight_kernel(const float* __restrict__ W, int K, int G, int mode, uint8_t*
       }
       d = min(d, kShiftMax);
       shat = (mode == ZQ_SCALE_M1) ? ldexpf(1.0f, P - d) : ldexpf(Smax, -d);
-      if (lane == 0) shift[n * G + j] = static_cast<uint8_t>(d);
+      if ((k % GROUP) == 0) shift[static_cast<int64_t>(n) * G + j] = static_cast<uint8_t>(d);
     }
-    const float* p = row + static_cast<int64_t>(j) * group + lane * EPL;
-    uint32_t packed = 0;
+    const float4 v0 = __ldg(reinterpret_cast<const float4*>(row + k));
+    const float4 v1 = __ldg(reinterpret_cast<const float4*>(row + k + 4));
+    const float q[8] = {__fdiv_rn(v0.x, shat), __fdiv_rn(v0.y, shat), __fdiv_rn(v0.z, shat), __fdiv_rn(v0.w, shat),
+                        __fdiv_rn(v1.x, shat), __fdiv_rn(v1.y, shat), __fdiv_rn(v1.z, shat), __fdiv_rn(v1.w, shat)};
+    uint32_t w = 0;
 #pragma unroll
-    for (int i = 0; i < EPL; i += 2) {
-      const float2 v = __ldg(reinterpret_cast<const float2*>(p + i));
-      packed |= encode_e2m1(__fdiv_rn(v.x, shat)) << (4 * i);
-      packed |= encode_e2m1(__fdiv_rn(v.y, shat)) << (4 * i + 4);
+    for (int i = 0; i < 8; ++i) {
+      w |= e2m1_magnitude(q[i]) << (4 * i);
+      const uint32_t sgn = __float_as_uint(q[i]) >> 31;
+      w |= sgn << (i < 4 ? 8 * i + 7 : 8 * (i - 4) + 3);
     }
-    uint8_t* out = codes + n * static_cast<int64_t>(K / 2) + static_cast<int64_t>(j) * (group / 2) + lane * (EPL / 2);
-    if (EPL == 2) *out = static_cast<uint8_t>(packed);
-    else if (EPL == 4) *reinterpret_cast<uint16_t*>(out) = static_cast<uint16_t>(packed);
-    else *reinterpret_cast<uint32_t*>(out) = packed;
+    uint8_t* blk = tile_row + static_cast<int64_t>(k / kTileK) * kTileBytes;
+    const int within = k % kTileK;
+    *reinterpret_cast<uint32_t*>(blk + ((within / 32) * kTileRows + r) * 16 + ((within % 32) / 8) * 4) = w;
+    if (within % 64 == 0) blk[kTileCodeBytes + 2 * r + within / 64] = static_cast<uint8_t>(d);
   }
 }
 
@@ -144,11 +164,12 @@ int launch_pack_weight(const float* W, int64_t N, int64_t K, int group, int mode
   if (N == 0) return ZQ_OK;
   const int G = static_cast<int>(K / group);
   const size_t smem = static_cast<size_t>(G) * sizeof(float);
-  dim3 grid(static_cast<unsigned>(N));
+  const int rows = static_cast<int>((N + kTileRows - 1) / kTileRows) * kTileRows;
+  dim3 grid(static_cast<unsigned>(rows));
   switch (group) {
-    case 64: pack_weight_kernel<2><<<grid, kThreads, smem, st>>>(W, int(K), G, mode, codes, shift, scale); break;
-    case 128: pack_weight_kernel<4><<<grid, kThreads, smem, st>>>(W, int(K), G, mode, codes, shift, scale); break;
-    case 256: pack_weight_kernel<8><<<grid, kThreads, smem, st>>>(W, int(K), G, mode, codes, shift, scale); break;
+    case 64: pack_weight_kernel<64><<<grid, kThreads, smem, st>>>(W, int(N), int(K), mode, codes, shift, scale); break;
+    case 128: pack_weight_kernel<128><<<grid, kThreads, smem, st>>>(W, int(N), int(K), mode, codes, shift, scale); break;
+    case 256: pack_weight_kernel<256><<<grid, kThreads, smem, st>>>(W, int(N), int(K), mode, codes, shift, scale); break;
     default: return ZQ_ERR_SHAPE;
   }
   count_launch();

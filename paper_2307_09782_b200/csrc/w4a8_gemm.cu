@@ -1,9 +1,10 @@
 // W4A8 GEMM: y = sx * scale * (Q_fp8(x) . cast_fp8(W_fp4)^T) + t U^T        (Section 3)
 //
 // The cast FP4 -> FP8 (Section 3, "Casting the FP4 to FP8") runs inside the kernel as an exponent
-// shift: TMA stages packed E2M1 tiles, CUDA cores expand each nibble to an E4M3 byte through an
-// 8-entry byte-permute table whose entries already carry the group's shift, and tcgen05 MMAs
-// (kind::f8f6f4, E4M3 x E4M3, FP32 accumulators in TMEM) consume the widened tile.
+// shift: one bulk copy per K block stages a packed E2M1 tile (codes + its shift bytes, contiguous in
+// HBM), CUDA cores expand each nibble to an E4M3 byte through an 8-entry byte-permute table whose
+// entries already carry the group's shift, and tcgen05 MMAs (kind::f8f6f4, E4M3 x E4M3, FP32
+// accumulators in TMEM) consume the widened tile.  Token tiles arrive by TMA.
 //
 // Orientation: the weight tile is the MMA's 128-row operand (D rows = output channels n, one TMEM
 // lane each), the token tile is the N-extent operand (D columns = tokens m, BM of them).  That keeps
@@ -30,7 +31,6 @@ namespace {
 constexpr int kThreads = 320;
 constexpr int kTileN = 128;      // output channels per CTA (MMA M extent)
 constexpr int kBlockK = 128;     // K elements per pipeline step (= one 128-byte swizzled row of E4M3)
-constexpr int kPackedBytes = kTileN * kBlockK / 2;  // 8 KB
 constexpr int kWideBytes = kTileN * kBlockK;        // 16 KB
 
 // error detail codes written to status[1]
@@ -43,7 +43,7 @@ struct Params {
   int kb_per_split;  // K blocks handled by one CTA
   int kblocks;       // total K blocks
   int splits;
-  const uint8_t* shift;
+  const uint8_t* codes;  // tiled weight
   const float* scale;
   const float* sx;
   const __half* U;
@@ -60,35 +60,36 @@ struct Params {
 template <int BM, bool NONE>
 struct Cfg {
   static constexpr int kTokBytes = BM * kBlockK;
-  static constexpr int NS = BM <= 16 ? 6 : BM <= 32 ? 5 : BM <= 64 ? 4 : BM <= 128 ? 3 : 2;  // TMA stages
-  static constexpr int NW = 2;                                                               // widened stages
+  // pipeline depth: copy stages (weights + tokens) and widened-tile stages; BM = 256 runs one CTA per SM
+  static constexpr int NS = BM <= 16 ? 6 : BM <= 32 ? 5 : BM <= 64 ? 3 : BM <= 128 ? 3 : 4;
+  static constexpr int NW = BM <= 64 ? 3 : BM <= 128 ? 2 : 3;
+  static constexpr int kMinBlocks = (NONE || BM > 128) ? 1 : 2;
   static constexpr int kTmemCols = (NONE ? 2 * BM : BM) < 32 ? 32 : (NONE ? 2 * BM : BM);
   static constexpr int kWidenThreads = NONE ? 128 : 256;
   static constexpr int kEpiThreads = NONE ? 128 : 256;
   // shared memory map (offsets from a 1024-byte aligned base)
-  static constexpr int offWide = 0;
-  static constexpr int offTok = offWide + NW * kWideBytes;
-  static constexpr int offPacked = offTok + NS * kTokBytes;
-  static constexpr int offBars = offPacked + NS * kPackedBytes;
+  static constexpr int offTok = 0;
+  static constexpr int offWide = offTok + NS * kTokBytes;
+  static constexpr int offPacked = offWide + NW * kWideBytes;
+  static constexpr int offSx = offPacked + NS * kTileBytes;   // [BM] token scales
+  static constexpr int offT = offSx + BM * 4;                 // [BM][8] LoRC down-projection (rank 8)
+  static constexpr int offBars = offT + BM * 32;
   static constexpr int kNumBars = 2 * NS + 2 * NW + 6;
   static constexpr int offMisc = offBars + kNumBars * 8;
   static constexpr int kSmemBytes = offMisc + 32;
 };
 
-// Expand 8 packed E2M1 codes (one 32-bit word, element i in nibble i) to 8 E4M3 bytes.
+// Expand 8 packed E2M1 codes (one 32-bit word of the tile format: magnitude of element i in bits
+// 4i .. 4i+2, sign of element b < 4 in bit 8b+7, sign of element 4+b in bit 8b+3) to 8 E4M3 bytes.
 // lut_lo / lut_hi hold the E4M3 magnitudes of the 8 E2M1 magnitudes with the group's shift already
-// subtracted from their exponent fields; the sign nibble-bit moves to bit 7 of its byte.
+// subtracted from their exponent fields.
 __device__ __forceinline__ void widen8(uint32_t w, uint32_t lut_lo, uint32_t lut_hi, uint32_t& o0, uint32_t& o1) {
-  const uint32_t w4 = w << 4;
-  uint32_t s0, s1, m0, m1;
-  // selector nibbles with bit 3 set replicate the most significant bit of the chosen byte:
-  // byte b of w carries the sign of element 2b+1 in its top bit, byte b of (w << 4) that of element 2b
-  asm("prmt.b32 %0, %1, %2, 0xD9C8;" : "=r"(s0) : "r"(w4), "r"(w));
-  asm("prmt.b32 %0, %1, %2, 0xFBEA;" : "=r"(s1) : "r"(w4), "r"(w));
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(m0) : "r"(lut_lo), "r"(lut_hi), "r"(w & 0x7777u));
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(m1) : "r"(lut_lo), "r"(lut_hi), "r"((w >> 16) & 0x7777u));
-  o0 = m0 | (s0 & 0x80808080u);
-  o1 = m1 | (s1 & 0x80808080u);
+  const uint32_t wm = w & 0x77777777u;
+  uint32_t m0, m1;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(m0) : "r"(lut_lo), "r"(lut_hi), "r"(wm));        // selector: low 16 bits
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(m1) : "r"(lut_lo), "r"(lut_hi), "r"(wm >> 16));
+  o0 = m0 | (w & 0x80808080u);
+  o1 = m1 | ((w << 4) & 0x80808080u);
 }
 
 // One 16-byte chunk of packed codes (32 elements) -> two 16-byte chunks of E4M3.
@@ -108,19 +109,20 @@ __device__ __forceinline__ void raise_error(const Params& p, volatile int* abort
   if (atomicCAS(p.status, 0, ZQ_ERR_DEVICE_TIMEOUT) == 0) p.status[1] = detail;
 }
 
-// Final arithmetic of 16 consecutive tokens of one output channel, and the store.
+// Final arithmetic of 16 consecutive tokens (tile columns c0 .. c0+15) of one output channel, and the store.
 //   y[m, n] = sx[m] * cs * acc + sum_j t[m, j] * U[n, j]
-// u8 holds the channel's U row when r == 8 (the common rank); other ranks read U through the cache.
-__device__ __forceinline__ void finalize16(const Params& p, const float* v, int m_base, int n, float cs,
-                                           const float* u8) {
+// s_sx / s_t are the tile's token scales and rank-8 LoRC rows in shared memory; u8 holds the channel's
+// U row when r == 8 (the common rank); other ranks read t and U through the cache.
+__device__ __forceinline__ void finalize16(const Params& p, const float* v, int m0, int c0, int n, float cs,
+                                           const float* u8, const float* s_sx, const float* s_t) {
 #pragma unroll
   for (int c = 0; c < 16; ++c) {
-    const int m = m_base + c;
+    const int m = m0 + c0 + c;
     if (m < p.M) {
-      float out = __ldg(p.sx + m) * cs * v[c];
+      float out = s_sx[c0 + c] * cs * v[c];
       if (p.r == 8) {
-        const float4* tr = reinterpret_cast<const float4*>(p.t + static_cast<int64_t>(m) * 8);
-        const float4 t0 = __ldg(tr), t1 = __ldg(tr + 1);
+        const float4 t0 = *reinterpret_cast<const float4*>(s_t + (c0 + c) * 8);
+        const float4 t1 = *reinterpret_cast<const float4*>(s_t + (c0 + c) * 8 + 4);
         out = fmaf(t0.x, u8[0], out);
         out = fmaf(t0.y, u8[1], out);
         out = fmaf(t0.z, u8[2], out);
@@ -143,9 +145,8 @@ __device__ __forceinline__ void finalize16(const Params& p, const float* v, int 
 }
 
 template <int BM, bool NONE>
-__global__ void __launch_bounds__(kThreads, NONE ? 1 : 2)
-w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_codes, const __grid_constant__ CUtensorMap tm_q,
-                 const Params p) {
+__global__ void __launch_bounds__(kThreads, Cfg<BM, NONE>::kMinBlocks)
+w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   using C = Cfg<BM, NONE>;
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* s_wide = smem + C::offWide;
@@ -162,6 +163,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_codes, const __grid_cons
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::offMisc);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::offMisc + 4);
   int* s_last = reinterpret_cast<int*>(smem + C::offMisc + 8);
+  float* s_sx = reinterpret_cast<float*>(smem + C::offSx);
+  float* s_t = reinterpret_cast<float*>(smem + C::offT);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * BM;
@@ -187,9 +190,13 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_codes, const __grid_cons
     fence_mbar_init();
     if ((smem_u32(smem) & 1023u) != 0) raise_error(p, s_abort, kErrAlign);
   }
-  if (warp == 8 && lane == 0) {
-    prefetch_tensormap(&tm_codes);
-    prefetch_tensormap(&tm_q);
+  if (warp == 8 && lane == 0) prefetch_tensormap(&tm_q);
+  if (warp < 8) {
+    // token scales and (rank 8) LoRC rows of this tile's tokens, for the epilogue
+    for (int c = threadIdx.x; c < BM; c += 256) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
+    if (p.r == 8)
+      for (int c = threadIdx.x; c < BM * 8; c += 256)
+        s_t[c] = (m0 + (c >> 3) < p.M) ? __ldg(p.t + static_cast<int64_t>(m0) * 8 + c) : 0.0f;
   }
   if (warp == 9) tmem_alloc(s_tmem, C::kTmemCols);
   tc_fence_before_sync();
@@ -201,6 +208,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_codes, const __grid_cons
   if (warp == 8) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0 && ok_start) {
+      const uint8_t* wtiles = p.codes + (static_cast<int64_t>(blockIdx.x) * p.kblocks + kb0) * kTileBytes;
       int issued = 0;
       for (int i = 0; i < nkb; ++i) {
         const int s = i % C::NS;
@@ -209,8 +217,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_codes, const __grid_cons
           raise_error(p, s_abort, kErrProducer);
           break;
         }
-        mbar_arrive_expect_tx(&tma_full[s], kPackedBytes + C::kTokBytes);
-        tma_load_2d(s_packed + s * kPackedBytes, &tm_codes, (kb0 + i) * (kBlockK / 2), n0, &tma_full[s]);
+        mbar_arrive_expect_tx(&tma_full[s], kTileBytes + C::kTokBytes);
+        bulk_load(s_packed + s * kTileBytes, wtiles + static_cast<int64_t>(i) * kTileBytes, kTileBytes, &tma_full[s]);
         tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, (kb0 + i) * kBlockK, m0, &tma_full[s]);
         issued = i + 1;
       }
@@ -286,31 +294,27 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_codes, const __grid_cons
       // M1/M2: a thread widens half a row (64 codes); mode none: group A threads widen a whole row.
       const int half = NONE ? 0 : grpB;
       constexpr int kChunks = NONE ? 4 : 2;  // 16-byte packed chunks per thread
-      const uint32_t sw64 = (row >> 1) & 3;  // 64-byte swizzle of the packed tile (TMA wrote it)
       const uint32_t sw128 = row & 7;        // 128-byte swizzle of the widened tile (the MMA reads it)
       const uint32_t wide_row_off = (row >> 3) * 1024 + (row & 7) * 128;
-      const uint8_t* shift_row = (!NONE && n_ok) ? p.shift + static_cast<int64_t>(n) * p.G : nullptr;
-      uint32_t d_next = 0;
-      if (shift_row && nkb > 0) d_next = __ldg(shift_row + ((kb0 * kBlockK + half * 64) / p.group));
       for (int i = 0; i < nkb; ++i) {
         const int s = i % C::NS, ws = i % C::NW;
-        const uint32_t d = d_next;
-        if (shift_row && i + 1 < nkb) d_next = __ldg(shift_row + (((kb0 + i + 1) * kBlockK + half * 64) / p.group));
         if (!mbar_wait(&tma_full[s], (i / C::NS) & 1, s_abort) ||
             !mbar_wait(&wide_empty[ws], ((i / C::NW) & 1) ^ 1, s_abort)) {
           raise_error(p, s_abort, kErrWiden);
           failed = true;
           break;
         }
+        const uint8_t* tile = s_packed + s * kTileBytes;
+        // the tile carries its shift bytes (zero in mode none): one per row and 64-element half
+        const uint32_t d = NONE ? 0u : tile[kTileCodeBytes + 2 * row + half];
         const uint32_t lut_lo = 0x3C383000u - d * 0x08080800u;
         const uint32_t lut_hi = 0x4C484440u - d * 0x08080808u;
-        const uint8_t* prow = s_packed + s * kPackedBytes + row * 64;
         uint8_t* wrow = s_wide + ws * kWideBytes + wide_row_off;
         uint4 pk[kChunks];
 #pragma unroll
         for (int c = 0; c < kChunks; ++c) {
-          const uint32_t lc = half * 2 + c;  // logical 16-byte chunk of the packed row
-          pk[c] = *reinterpret_cast<const uint4*>(prow + ((lc ^ sw64) << 4));
+          const uint32_t lc = half * 2 + c;  // 16-byte chunk of the packed row; chunk-major in the tile
+          pk[c] = *reinterpret_cast<const uint4*>(tile + (lc * kTileRows + row) * 16);
         }
 #pragma unroll
         for (int c = 0; c < kChunks; ++c) {
@@ -404,7 +408,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_codes, const __grid_cons
               tmem_ld16(t_lane + col0 + c, v);
               tmem_ld_wait();
             }
-            if (n_ok) finalize16(p, v, m0 + col0 + c, n, cs, u);
+            if (n_ok) finalize16(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
           }
         }
       } else {
@@ -447,7 +451,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_codes, const __grid_cons
 #pragma unroll
               for (int e = 0; e < 16; ++e) v[e] += __ldcg(src + e * kTileN);
             }
-            if (n_ok) finalize16(p, v, m0 + col0 + c, n, cs, u);
+            if (n_ok) finalize16(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
           }
         }
       }
@@ -497,10 +501,8 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t row
 template <int BM, bool NONE>
 int launch_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStream_t st) {
   using C = Cfg<BM, NONE>;
-  CUtensorMap tm_codes, tm_q;
-  if (!make_map(&tm_codes, a.codes, static_cast<uint64_t>(a.K / 2), static_cast<uint64_t>(a.N), kBlockK / 2, kTileN,
-                CU_TENSOR_MAP_SWIZZLE_64B) ||
-      !make_map(&tm_q, a.q, static_cast<uint64_t>(a.K), static_cast<uint64_t>(a.M), kBlockK, BM,
+  CUtensorMap tm_q;
+  if (!make_map(&tm_q, a.q, static_cast<uint64_t>(a.K), static_cast<uint64_t>(a.M), kBlockK, BM,
                 CU_TENSOR_MAP_SWIZZLE_128B))
     return ZQ_ERR_CUDA;
   static std::once_flag once;
@@ -511,7 +513,7 @@ int launch_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStr
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
   dim3 grid(plan.n_tiles, plan.m_tiles, plan.splits);
-  w4a8_gemm_kernel<BM, NONE><<<grid, kThreads, C::kSmemBytes, st>>>(tm_codes, tm_q, p);
+  w4a8_gemm_kernel<BM, NONE><<<grid, kThreads, C::kSmemBytes, st>>>(tm_q, p);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
 }
@@ -559,7 +561,7 @@ int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st) {
   p.kblocks = static_cast<int>(a.K / kBlockK);
   p.splits = plan.splits;
   p.kb_per_split = plan.kb_per_split;
-  p.shift = a.shift;
+  p.codes = a.codes;
   p.scale = a.scale;
   p.sx = a.sx;
   p.U = static_cast<const __half*>(a.U);

@@ -19,6 +19,22 @@ constexpr int kWsMaxTiles = 16384;  // counters: one int per output tile
 constexpr size_t kWsCounterBytes = size_t(kWsMaxTiles) * 4;
 constexpr size_t kWsHeadBytes = kWsStatusBytes + kWsCounterBytes;
 
+// ---- packed weight format (written by the packer, streamed by the GEMM) --------------------------
+// The weight is stored as tiles of 128 output rows x 128 input features, tile (nt, kb) at byte offset
+// (nt * (K / 128) + kb) * kTileBytes, so that a CTA walking along K reads one contiguous stream.
+// A tile holds
+//   [0, 8192)    codes: 16-byte chunk c (elements 32c .. 32c+31 of the K block) of row r at (c * 128 + r) * 16;
+//                inside a chunk, 32-bit word j holds elements 8j .. 8j+7: nibble i (bits 4i .. 4i+2) = the
+//                E2M1 magnitude bits of element i, bit 8b+7 = sign of element b, bit 8b+3 = sign of element
+//                4+b (b < 4).  That order lets the cast to E4M3 take signs with one AND per four elements.
+//   [8192, 8448) shifts: byte 2r + h = exponent shift of row r for elements 64h .. 64h+63 (zero in mode none)
+// Rows beyond N in the last tile are zero.
+constexpr int kTileRows = 128;
+constexpr int kTileK = 128;
+constexpr int kTileCodeBytes = kTileRows * kTileK / 2;
+constexpr int kTileShiftBytes = 2 * kTileRows;
+constexpr int kTileBytes = kTileCodeBytes + kTileShiftBytes;
+
 // ---- launchers implemented in the .cu files ------------------------------------------------------
 int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
                      const void* V, int r, float* t, cudaStream_t st);
@@ -30,8 +46,8 @@ struct GemmArgs {
   const float* sx;       // [M]
   int64_t M, N, K;
   int group, mode;
-  const uint8_t* codes;  // [N, K/2]
-  const uint8_t* shift;  // [N, G] or NULL
+  const uint8_t* codes;  // tiled, see above
+  const uint8_t* shift;  // [N, G] or NULL (not read by the GEMM: the tiles carry the shifts)
   const float* scale;    // [N] or [N, G]
   const void* U;         // fp16 [N, r] or NULL
   const float* t;        // [M, r] or NULL
@@ -116,6 +132,13 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
       : "memory");
+}
+
+// Contiguous global -> shared copy of `bytes` (multiple of 16, both addresses 16-byte aligned).
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
 }
 
 // ---- device: tcgen05 / TMEM ----------------------------------------------------------------------

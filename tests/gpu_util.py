@@ -24,6 +24,38 @@ def host(t):
     return None if t is None else t.cpu().numpy()
 
 
+def untile_codes(tiles: np.ndarray, N: int, K: int):
+    """Decodes the library's tiled weight format (include/zqfp.h) back to plain form:
+    returns (codes uint8 [N, K/2] with element 2b in the low nibble of byte b, shifts uint8 [N, K/64])."""
+    nt, kb = (N + 127) // 128, K // 128
+    t = np.ascontiguousarray(tiles, dtype=np.uint8).reshape(nt, kb, 8448)
+    words = t[:, :, :8192].copy().view(np.uint32).reshape(nt, kb, 4, 128, 4)     # [nt, kb, chunk, row, word]
+    el = np.empty((nt, kb, 4, 128, 4, 8), dtype=np.uint8)                         # 4-bit codes per element
+    for i in range(8):
+        mag = (words >> np.uint32(4 * i)) & np.uint32(7)
+        sbit = 8 * i + 7 if i < 4 else 8 * (i - 4) + 3
+        sgn = (words >> np.uint32(sbit)) & np.uint32(1)
+        el[..., i] = (mag | (sgn << np.uint32(3))).astype(np.uint8)
+    # -> [nt, row, kb, chunk, word, i] = [n, k]
+    el = el.transpose(0, 3, 1, 2, 4, 5).reshape(nt * 128, K)
+    codes = (el[:, 0::2] | (el[:, 1::2] << 4)).astype(np.uint8)
+    sh = t[:, :, 8192:].reshape(nt, kb, 128, 2).transpose(0, 2, 1, 3).reshape(nt * 128, kb * 2)
+    assert not codes[N:].any() and not sh[N:].any(), "padding rows must be zero"
+    return codes[:N], sh[:N]
+
+
+def check_packed(pw, c_o, sh_o, sc_o, group):
+    """Bit-exact comparison of a PackedWeight with the oracle's plain codes / shifts / scales."""
+    codes, sh64 = untile_codes(host(pw.codes), pw.N, pw.K)
+    assert np.array_equal(codes, c_o), "FP4 codes"
+    if sh_o is not None:
+        assert np.array_equal(host(pw.shift), sh_o), "shifts"
+        assert np.array_equal(sh64, np.repeat(sh_o, group // 64, axis=1)), "shift bytes inside the tiles"
+    else:
+        assert not sh64.any()
+    assert np.array_equal(host(pw.scale).view(np.uint32), sc_o.view(np.uint32)), "scales"
+
+
 def check_linear(x_bits, W, U, V, group, mode, out_dtype=torch.float32, rows=None, fused_quant=False):
     """Runs oracle and CUDA path on the same inputs; asserts bit-exact codes / scales and y within tolerance."""
     M, K = x_bits.shape
@@ -35,21 +67,18 @@ def check_linear(x_bits, W, U, V, group, mode, out_dtype=torch.float32, rows=Non
 
     x = to_bf16(x_bits)
     Wd, Ud, Vd = up(W), up(U), up(V)
-    codes, shift, scale = binding.pack_weight_fp4(Wd, group, mode)
-    assert np.array_equal(host(codes), c_o), "FP4 codes"
-    if sh_o is not None:
-        assert np.array_equal(host(shift), sh_o), "shifts"
-    assert np.array_equal(host(scale).view(np.uint32), sc_o.view(np.uint32)), "scales"
+    pw = binding.pack_weight_fp4(Wd, group, mode)
+    check_packed(pw, c_o, sh_o, sc_o, group)
     ws = binding.make_workspace(binding.linear_workspace_bytes(M, N, K, r))
     if fused_quant:
-        y = binding.w4a8_linear(codes, shift, scale, group, mode, x=x, U=Ud, V=Vd, out_dtype=out_dtype, workspace=ws)
+        y = binding.w4a8_linear(pw, x=x, U=Ud, V=Vd, out_dtype=out_dtype, workspace=ws)
     else:
         q, sx, t = binding.quantize_act_fp8(x, Vd)
         assert np.array_equal(host(q), q_o), "FP8 codes"
         assert np.array_equal(host(sx).view(np.uint32), sx_o.view(np.uint32)), "token scales"
         if r:
             assert np.abs(host(t) - t_o).max() <= 1e-4 * max(np.abs(t_o).max(), 1e-30), "LoRC down-projection"
-        y = binding.w4a8_linear(codes, shift, scale, group, mode, q=q, sx=sx, t=t, U=Ud, out_dtype=out_dtype,
+        y = binding.w4a8_linear(pw, q=q, sx=sx, t=t, U=Ud, out_dtype=out_dtype,
                                 workspace=ws)
     st, detail = binding.device_status(ws)
     assert st == 0, f"device status {st} detail {detail}"

@@ -34,8 +34,9 @@ def test_status_strings(L):
 
 
 def test_size_queries(L):
-    assert binding.packed_weight_sizes(768, 768, 128, "none") == (768 * 384, 0, 768 * 6 * 4)
-    assert binding.packed_weight_sizes(768, 768, 128, "M2") == (768 * 384, 768 * 6, 768 * 4)
+    assert binding.packed_weight_sizes(768, 768, 128, "none") == (6 * 6 * 8448, 0, 768 * 6 * 4)
+    assert binding.packed_weight_sizes(768, 768, 128, "M2") == (6 * 6 * 8448, 768 * 6, 768 * 4)
+    assert binding.packed_weight_sizes(129, 256, 64, "M1") == (2 * 2 * 8448, 129 * 4, 129 * 4)
     with pytest.raises(binding.ZqError) as e:
         binding.packed_weight_sizes(8, 100, 128, "M1")
     assert e.value.status == -2
@@ -78,7 +79,7 @@ def test_validation_before_launch(L):
     assert call(r=12, U=fake, t=fake) == -2
     assert call(mode=5) == -4
     assert call(ydt=2) == -4
-    assert call(shift=null) == -1
+    assert call(codes=null) == -1
     assert call(q=null) == -1
     assert call(r=8, U=fake) == -1          # t missing
     assert call(ldy=64) == -2

@@ -9,7 +9,7 @@ import torch
 
 import oracle
 from paper_2307_09782_b200 import binding, synth
-from gpu_util import TOL_REL, check_linear, dev, host, to_bf16, up
+from gpu_util import TOL_REL, check_linear, check_packed, dev, host, to_bf16, up
 
 pytestmark = pytest.mark.gpu
 
@@ -55,6 +55,7 @@ def test_act_quant_edge_rows_and_strided_input():
 # ---------------------------------------------------------------------------------------------- packer
 def _special_weights(N, K, seed):
     W = synth.make_w(seed, N, K, 0.02)
+    assert N >= 7
     W[0, :128] = 0.0                                   # all-zero group
     W[1, 128:256] *= np.float32(2.0 ** -9)             # needs a shift beyond the clamp
     W[2, :] = 0.0                                      # all-zero row
@@ -71,22 +72,14 @@ def _special_weights(N, K, seed):
 def test_pack_weight_bit_exact(mode, group):
     W = _special_weights(9, 1024, 31)
     c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, group, mode)
-    codes, shift, scale = binding.pack_weight_fp4(up(W), group, mode)
-    assert np.array_equal(host(codes), c_o)
-    if mode != "none":
-        assert np.array_equal(host(shift), sh_o)
-    assert np.array_equal(host(scale).view(np.uint32), sc_o.view(np.uint32))
+    check_packed(binding.pack_weight_fp4(up(W), group, mode), c_o, sh_o, sc_o, group)
 
 
 @pytest.mark.parametrize("mode", ["none", "M1", "M2"])
 def test_pack_weight_layer_shape(mode):
     W = synth.make_w(2, 1000, 4096, 0.02)
     c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, 128, mode)
-    codes, shift, scale = binding.pack_weight_fp4(up(W), 128, mode)
-    assert np.array_equal(host(codes), c_o)
-    if mode != "none":
-        assert np.array_equal(host(shift), sh_o)
-    assert np.array_equal(host(scale).view(np.uint32), sc_o.view(np.uint32))
+    check_packed(binding.pack_weight_fp4(up(W), 128, mode), c_o, sh_o, sc_o, 128)
 
 
 # ---------------------------------------------------------------------------------------------- linear
@@ -156,12 +149,12 @@ def test_workspace_reuse_across_calls_and_token_counts():
     W = synth.make_w(7, N, K)
     U, V = synth.make_lorc(7, N, K, r)
     c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, 128, "M2")
-    codes, shift, scale = binding.pack_weight_fp4(up(W), 128, "M2")
+    pw = binding.pack_weight_fp4(up(W), 128, "M2")
     for M in (256, 16, 1, 100, 16):
         x_bits = synth.make_x(7 + M, M, K, 20)
         q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
         y_o = oracle.w4a8_linear(q_o, sx_o, c_o, sh_o, sc_o, 128, "M2", U, t_o)
-        y = binding.w4a8_linear(codes, shift, scale, 128, "M2", x=to_bf16(x_bits), U=up(U), V=up(V), workspace=ws)
+        y = binding.w4a8_linear(pw, x=to_bf16(x_bits), U=up(U), V=up(V), workspace=ws)
         assert binding.device_status(ws) == (0, 0)
         assert np.abs(host(y) - y_o).max() <= TOL_REL * np.abs(y_o).max()
 
@@ -169,11 +162,11 @@ def test_workspace_reuse_across_calls_and_token_counts():
 def test_host_buffer_entry_point():
     M, N, K, r = 24, 256, 512, 8
     x_bits, W, U, V = _layer(95, M, N, K, r)
-    codes, shift, scale = binding.pack_weight_fp4(up(W), 128, "M1")
+    pw = binding.pack_weight_fp4(up(W), 128, "M1")
     ws = binding.make_workspace(binding.linear_host_workspace_bytes(M, N, K, r))
     xh = torch.from_numpy(x_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
     yh = torch.empty((M, N), dtype=torch.float32).pin_memory()
-    binding.w4a8_linear_host(xh, yh, codes, shift, scale, 128, "M1", U=up(U), V=up(V), workspace=ws)
+    binding.w4a8_linear_host(xh, yh, pw, U=up(U), V=up(V), workspace=ws)
     q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
     c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, 128, "M1")
     y_o = oracle.w4a8_linear(q_o, sx_o, c_o, sh_o, sc_o, 128, "M1", U, t_o)

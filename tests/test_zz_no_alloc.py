@@ -21,34 +21,33 @@ def _case(seed, M, N, K, r, mode):
     W = synth.make_w(seed, N, K, 0.02)
     U, V = synth.make_lorc(seed, N, K, r)
     q, sx, t = binding.quantize_act_fp8(to_bf16(x_bits), up(V))
-    codes, shift, scale = binding.pack_weight_fp4(up(W), 128, mode)
-    return q, sx, t, up(U), codes, shift, scale
+    return q, sx, t, up(U), binding.pack_weight_fp4(up(W), 128, mode)
 
 
 def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
     # a split-K shape (few output tiles, long K): the scratch array is really used
     M, N, K, r, mode = 16, 256, 8192, 8, "M2"
-    q, sx, t, U, codes, shift, scale = _case(201, M, N, K, r, mode)
+    q, sx, t, U, pw = _case(201, M, N, K, r, mode)
     ws = binding.make_workspace(binding.linear_workspace_bytes(M, N, K, r))
-    y_ref = binding.w4a8_linear(codes, shift, scale, 128, mode, q=q, sx=sx, t=t, U=U, workspace=ws)
+    y_ref = binding.w4a8_linear(pw, q=q, sx=sx, t=t, U=U, workspace=ws)
     assert binding.device_status(ws) == (0, 0)
     ref = host(y_ref).astype(np.float64)
     tol = TOL_REL * np.abs(ref).max()
     for _ in range(2):
-        y = binding.w4a8_linear_noalloc(codes, shift, scale, 128, mode, q=q, sx=sx, t=t, U=U)
+        y = binding.w4a8_linear_noalloc(pw, q=q, sx=sx, t=t, U=U)
         torch.cuda.synchronize()
         assert np.abs(host(y).astype(np.float64) - ref).max() <= tol
     # a different problem right after (other tile shape, mode none, no split) reuses the same array
     M2, N2, K2 = 200, 384, 512
-    q2, sx2, t2, U2, codes2, shift2, scale2 = _case(202, M2, N2, K2, r, "none")
+    q2, sx2, t2, U2, pw2 = _case(202, M2, N2, K2, r, "none")
     ws2 = binding.make_workspace(binding.linear_workspace_bytes(M2, N2, K2, r))
-    ref2 = host(binding.w4a8_linear(codes2, shift2, scale2, 128, "none", q=q2, sx=sx2, t=t2, U=U2, workspace=ws2))
+    ref2 = host(binding.w4a8_linear(pw2, q=q2, sx=sx2, t=t2, U=U2, workspace=ws2))
     for _ in range(2):
-        y2 = binding.w4a8_linear_noalloc(codes2, shift2, scale2, 128, "none", q=q2, sx=sx2, t=t2, U=U2)
+        y2 = binding.w4a8_linear_noalloc(pw2, q=q2, sx=sx2, t=t2, U=U2)
         torch.cuda.synchronize()
         assert np.abs(host(y2).astype(np.float64) - ref2).max() <= TOL_REL * np.abs(ref2).max()
     # and the first problem again
-    y = binding.w4a8_linear_noalloc(codes, shift, scale, 128, mode, q=q, sx=sx, t=t, U=U)
+    y = binding.w4a8_linear_noalloc(pw, q=q, sx=sx, t=t, U=U)
     torch.cuda.synchronize()
     assert np.abs(host(y).astype(np.float64) - ref).max() <= tol
 
@@ -60,9 +59,10 @@ def test_noalloc_rejects_problems_beyond_the_fixed_scratch():
     M, N, K = 256, 4096, 65536
     q = torch.zeros((M, K), dtype=torch.uint8, device="cuda")
     sx = torch.ones((M,), dtype=torch.float32, device="cuda")
-    codes = torch.zeros((N, K // 2), dtype=torch.uint8, device="cuda")
-    shift = torch.zeros((N, K // 128), dtype=torch.uint8, device="cuda")
-    scale = torch.ones((N,), dtype=torch.float32, device="cuda")
+    nbytes = binding.packed_weight_sizes(N, K, 128, "M1")[0]
+    pw = binding.PackedWeight(torch.zeros((nbytes,), dtype=torch.uint8, device="cuda"),
+                              torch.zeros((N, K // 128), dtype=torch.uint8, device="cuda"),
+                              torch.ones((N,), dtype=torch.float32, device="cuda"), N, K, 128, binding.SCALE_M1)
     with pytest.raises(binding.ZqError) as e:
-        binding.w4a8_linear_noalloc(codes, shift, scale, 128, "M1", q=q, sx=sx)
+        binding.w4a8_linear_noalloc(pw, q=q, sx=sx)
     assert e.value.status == -5
