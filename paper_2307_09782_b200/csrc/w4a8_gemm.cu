@@ -1,23 +1,27 @@
 // W4A8 GEMM: y = sx * scale * (Q_fp8(x) . cast_fp8(W_fp4)^T) + t U^T        (Section 3)
 //
 // The cast FP4 -> FP8 (Section 3, "Casting the FP4 to FP8") runs inside the kernel as an exponent
-// shift: one bulk copy per K block stages a packed E2M1 tile (codes + its shift bytes, contiguous in
-// HBM), CUDA cores expand each nibble to an E4M3 byte through an 8-entry byte-permute table whose
-// entries already carry the group's shift, and tcgen05 MMAs (kind::f8f6f4, E4M3 x E4M3, FP32
-// accumulators in TMEM) consume the widened tile.  Token tiles arrive by TMA.
+// shift.  One bulk copy per K block stages a packed E2M1 tile (codes + its shift bytes, contiguous in
+// HBM) in shared memory; CUDA cores expand each nibble to an E4M3 byte through an 8-entry
+// byte-permute table whose entries already carry the group's shift and write the widened row
+// straight into TENSOR MEMORY, from where tcgen05 MMAs (kind::f8f6f4, E4M3 x E4M3, FP32
+// accumulators, also in TMEM) take it as their A operand.  Token tiles arrive by TMA and are the
+// shared-memory B operand.  The widened weights never touch shared memory.
 //
 // Orientation: the weight tile is the MMA's 128-row operand (D rows = output channels n, one TMEM
 // lane each), the token tile is the N-extent operand (D columns = tokens m, BM of them).  That keeps
 // the widening work per tile fixed at 128 x 128 codes per K block whatever the token count, lets one
-// kernel serve decode (BM = 16) and prefill (BM = 256), and makes every per-channel quantity
-// (scale, shift, U row, group scale) a per-thread scalar in the epilogue.
+// kernel serve decode (BM = 16) and prefill (BM = 256), makes "thread = output channel" the natural
+// mapping for widening (a thread writes its own TMEM lane) and turns every per-channel quantity
+// (scale, shift, U row, group scale) into a per-thread scalar in the epilogue.
 //
-// Warp roles (10 warps):
-//   0-3  group A : widen; M1/M2 also epilogue for the first half of the columns
-//   4-7  group B : M1/M2: widen + epilogue for the second half; mode none: per-group promotion
-//                  (TMEM -> registers, times the FP32 group scale) and the epilogue
-//   8            : TMA producer (one lane)
-//   9            : TMEM allocation, MMA issue (one lane)
+// Warp roles:
+//   0-7   two widen groups of four warps (one warp per TMEM lane quarter); group g widens the K blocks
+//         i with i % 2 == g, so two K blocks are in flight and the hand-off latencies overlap.
+//         M1/M2: the same warps run the epilogue (group g takes half of the columns).
+//   8     TMA / bulk-copy producer (one lane)
+//   9     TMEM allocation, MMA issue (one lane)
+//   10-13 mode none only: per-group promotion (TMEM -> registers, times the FP32 group scale), epilogue
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -28,10 +32,10 @@
 namespace zq {
 namespace {
 
-constexpr int kThreads = 320;
-constexpr int kTileN = 128;      // output channels per CTA (MMA M extent)
-constexpr int kBlockK = 128;     // K elements per pipeline step (= one 128-byte swizzled row of E4M3)
-constexpr int kWideBytes = kTileN * kBlockK;        // 16 KB
+constexpr int kTileN = 128;   // output channels per CTA (MMA M extent)
+constexpr int kBlockK = 128;  // K elements per pipeline step
+constexpr int kAStageCols = kBlockK / 4;  // TMEM columns of one widened 128 x 128 tile (4 bytes per column)
+constexpr int kWidenGroups = 2;
 
 // error detail codes written to status[1]
 enum { kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6 };
@@ -59,24 +63,28 @@ struct Params {
 
 template <int BM, bool NONE>
 struct Cfg {
+  static constexpr int kThreads = NONE ? 448 : 320;
   static constexpr int kTokBytes = BM * kBlockK;
-  // pipeline depth: copy stages (weights + tokens) and widened-tile stages; BM = 256 runs one CTA per SM
-  static constexpr int NS = BM <= 16 ? 6 : BM <= 32 ? 5 : BM <= 64 ? 3 : BM <= 128 ? 3 : 4;
-  static constexpr int NW = BM <= 64 ? 3 : BM <= 128 ? 2 : 3;
-  static constexpr int kMinBlocks = (NONE || BM > 128) ? 1 : 2;
-  static constexpr int kTmemCols = (NONE ? 2 * BM : BM) < 32 ? 32 : (NONE ? 2 * BM : BM);
-  static constexpr int kWidenThreads = NONE ? 128 : 256;
+  static constexpr int kDCols = NONE ? 2 * BM : BM;                 // accumulator columns (two buffers in mode none)
+  static constexpr int kDColsPad = kDCols < 32 ? 32 : kDCols;
+  static constexpr int kMinBlocks = (NONE || BM > 128) ? 1 : 2;    // CTAs per SM this configuration is sized for
+  static constexpr int kTmemCols = kMinBlocks == 2 ? 256 : 512;
+  static constexpr int NA = (kTmemCols - kDColsPad) / kAStageCols > 8 ? 8 : (kTmemCols - kDColsPad) / kAStageCols;
+  // copy stages (packed weights + tokens): as many as fit in half (or all) of the SM's shared memory
+  static constexpr int kStageBytes = kTileBytes + kTokBytes;
+  static constexpr int kBudget = kMinBlocks == 2 ? 104 * 1024 : 208 * 1024;
+  static constexpr int NS = kBudget / kStageBytes > 8 ? 8 : kBudget / kStageBytes;
   static constexpr int kEpiThreads = NONE ? 128 : 256;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int offTok = 0;
-  static constexpr int offWide = offTok + NS * kTokBytes;
-  static constexpr int offPacked = offWide + NW * kWideBytes;
+  static constexpr int offPacked = offTok + NS * kTokBytes;
   static constexpr int offSx = offPacked + NS * kTileBytes;   // [BM] token scales
   static constexpr int offT = offSx + BM * 4;                 // [BM][8] LoRC down-projection (rank 8)
   static constexpr int offBars = offT + BM * 32;
-  static constexpr int kNumBars = 2 * NS + 2 * NW + 6;
+  static constexpr int kNumBars = 2 * NS + 2 * NA + 6;
   static constexpr int offMisc = offBars + kNumBars * 8;
   static constexpr int kSmemBytes = offMisc + 32;
+  static_assert(NA >= 4 && NS >= 3, "pipeline too shallow");
 };
 
 // Expand 8 packed E2M1 codes (one 32-bit word of the tile format: magnitude of element i in bits
@@ -90,14 +98,6 @@ __device__ __forceinline__ void widen8(uint32_t w, uint32_t lut_lo, uint32_t lut
   asm("prmt.b32 %0, %1, %2, %3;" : "=r"(m1) : "r"(lut_lo), "r"(lut_hi), "r"(wm >> 16));
   o0 = m0 | (w & 0x80808080u);
   o1 = m1 | ((w << 4) & 0x80808080u);
-}
-
-// One 16-byte chunk of packed codes (32 elements) -> two 16-byte chunks of E4M3.
-__device__ __forceinline__ void widen32(uint4 p, uint32_t lut_lo, uint32_t lut_hi, uint4& a, uint4& b) {
-  widen8(p.x, lut_lo, lut_hi, a.x, a.y);
-  widen8(p.y, lut_lo, lut_hi, a.z, a.w);
-  widen8(p.z, lut_lo, lut_hi, b.x, b.y);
-  widen8(p.w, lut_lo, lut_hi, b.z, b.w);
 }
 
 __device__ __forceinline__ void named_bar_sync(int id, int count) {
@@ -145,21 +145,20 @@ __device__ __forceinline__ void finalize16(const Params& p, const float* v, int 
 }
 
 template <int BM, bool NONE>
-__global__ void __launch_bounds__(kThreads, Cfg<BM, NONE>::kMinBlocks)
+__global__ void __launch_bounds__(Cfg<BM, NONE>::kThreads, Cfg<BM, NONE>::kMinBlocks)
 w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   using C = Cfg<BM, NONE>;
   extern __shared__ __align__(1024) uint8_t smem[];
-  uint8_t* s_wide = smem + C::offWide;
   uint8_t* s_tok = smem + C::offTok;
   uint8_t* s_packed = smem + C::offPacked;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offBars);
-  uint64_t* tma_full = bars;
-  uint64_t* tma_empty = bars + C::NS;
-  uint64_t* wide_full = bars + 2 * C::NS;
-  uint64_t* wide_empty = bars + 2 * C::NS + C::NW;
-  uint64_t* acc_full = bars + 2 * C::NS + 2 * C::NW;      // [2]
-  uint64_t* acc_empty = acc_full + 2;                     // [2]
-  uint64_t* drain_bar = acc_full + 4;                     // [1]
+  uint64_t* tma_full = bars;                   // [NS] copies landed
+  uint64_t* tma_empty = bars + C::NS;          // [NS] stage may be overwritten (MMA of that K block done)
+  uint64_t* a_full = bars + 2 * C::NS;         // [NA] widened tile complete in TMEM (4 warp arrivals)
+  uint64_t* a_empty = a_full + C::NA;          // [NA] MMA that read it done
+  uint64_t* acc_full = a_empty + C::NA;        // [2]
+  uint64_t* acc_empty = acc_full + 2;          // [2]
+  uint64_t* drain_bar = acc_full + 4;          // [1]
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::offMisc);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::offMisc + 4);
   int* s_last = reinterpret_cast<int*>(smem + C::offMisc + 8);
@@ -176,9 +175,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       mbar_init(&tma_full[i], 1);
       mbar_init(&tma_empty[i], 1);
     }
-    for (int i = 0; i < C::NW; ++i) {
-      mbar_init(&wide_full[i], C::kWidenThreads);
-      mbar_init(&wide_empty[i], 1);
+    for (int i = 0; i < C::NA; ++i) {
+      mbar_init(&a_full[i], 4);
+      mbar_init(&a_empty[i], 1);
     }
     mbar_init(&acc_full[0], 1);
     mbar_init(&acc_full[1], 1);
@@ -203,10 +202,11 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *s_tmem;
+  const uint32_t tmem_a = tmem_base + C::kDColsPad;  // widened-weight stages follow the accumulators
   const bool ok_start = (*s_abort == 0);
 
   if (warp == 8) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ copy producer
     if (lane == 0 && ok_start) {
       const uint8_t* wtiles = p.codes + (static_cast<int64_t>(blockIdx.x) * p.kblocks + kb0) * kTileBytes;
       int issued = 0;
@@ -238,14 +238,14 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       int mma_count = 0;
       bool failed = false;
       for (int i = 0; i < nkb && !failed; ++i) {
-        const int s = i % C::NS, ws = i % C::NW;
+        const int s = i % C::NS, a = i % C::NA;
         if (!mbar_wait(&tma_full[s], (i / C::NS) & 1, s_abort) ||
-            !mbar_wait(&wide_full[ws], (i / C::NW) & 1, s_abort)) {
+            !mbar_wait(&a_full[a], (i / C::NA) & 1, s_abort)) {
           failed = true;
           break;
         }
         tc_fence_after_sync();
-        const uint64_t adesc = umma_desc_k128(smem_u32(s_wide + ws * kWideBytes));
+        const uint32_t a_addr = tmem_a + a * kAStageCols;
         const uint64_t bdesc = umma_desc_k128(smem_u32(s_tok + s * C::kTokBytes));
 #pragma unroll
         for (int k = 0; k < kBlockK / 32; ++k) {
@@ -263,13 +263,13 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
             d_tmem = tmem_base + b * BM;
             accumulate = within > 0 ? 1u : 0u;
           }
-          umma_f8(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, accumulate);
+          umma_f8_tmem_a(d_tmem, a_addr + 8 * k, bdesc + 2 * k, idesc, accumulate);
           ++mma_count;
           if (NONE && (mma_count % mpg) == 0) umma_commit(&acc_full[((mma_count / mpg) - 1) & 1]);
         }
         if (failed) break;
         umma_commit(&tma_empty[s]);
-        umma_commit(&wide_empty[ws]);
+        umma_commit(&a_empty[a]);
       }
       if (failed) {
         raise_error(p, s_abort, kErrMma);
@@ -283,59 +283,65 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     }
   } else {
     // ------------------------------------------------------------------ widen / promote / epilogue
-    const int q4 = warp & 3, grpB = warp >> 2;  // TMEM lane quarter; 0 = group A, 1 = group B
-    const int row = q4 * 32 + lane;             // output channel within the tile = TMEM lane
+    const int q4 = warp & 3;         // TMEM lane quarter of this warp
+    const int row = q4 * 32 + lane;  // output channel within the tile = TMEM lane
     const int n = n0 + row;
     const bool n_ok = n < p.N;
-    const bool widen_role = NONE ? (grpB == 0) : true;
+    const uint32_t lane_base = static_cast<uint32_t>(q4 * 32) << 16;
     bool failed = !ok_start;
 
-    if (widen_role && !failed) {
-      // M1/M2: a thread widens half a row (64 codes); mode none: group A threads widen a whole row.
-      const int half = NONE ? 0 : grpB;
-      constexpr int kChunks = NONE ? 4 : 2;  // 16-byte packed chunks per thread
-      const uint32_t sw128 = row & 7;        // 128-byte swizzle of the widened tile (the MMA reads it)
-      const uint32_t wide_row_off = (row >> 3) * 1024 + (row & 7) * 128;
-      for (int i = 0; i < nkb; ++i) {
-        const int s = i % C::NS, ws = i % C::NW;
+    if (warp < 8 && !failed) {
+      // A lane widens whole rows: 64 packed bytes -> 128 E4M3 bytes = 32 TMEM columns of its own lane.
+      const int grp = warp >> 2;
+      for (int i = grp; i < nkb; i += kWidenGroups) {
+        const int s = i % C::NS, a = i % C::NA;
         if (!mbar_wait(&tma_full[s], (i / C::NS) & 1, s_abort) ||
-            !mbar_wait(&wide_empty[ws], ((i / C::NW) & 1) ^ 1, s_abort)) {
+            !mbar_wait(&a_empty[a], ((i / C::NA) & 1) ^ 1, s_abort)) {
           raise_error(p, s_abort, kErrWiden);
           failed = true;
           break;
         }
+        tc_fence_after_sync();
         const uint8_t* tile = s_packed + s * kTileBytes;
+        uint4 pk[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) pk[c] = *reinterpret_cast<const uint4*>(tile + (c * kTileRows + row) * 16);
         // the tile carries its shift bytes (zero in mode none): one per row and 64-element half
-        const uint32_t d = NONE ? 0u : tile[kTileCodeBytes + 2 * row + half];
-        const uint32_t lut_lo = 0x3C383000u - d * 0x08080800u;
-        const uint32_t lut_hi = 0x4C484440u - d * 0x08080808u;
-        uint8_t* wrow = s_wide + ws * kWideBytes + wide_row_off;
-        uint4 pk[kChunks];
+        const uint32_t d2 = NONE ? 0u : *reinterpret_cast<const uint16_t*>(tile + kTileCodeBytes + 2 * row);
+        uint32_t w[32];
 #pragma unroll
-        for (int c = 0; c < kChunks; ++c) {
-          const uint32_t lc = half * 2 + c;  // 16-byte chunk of the packed row; chunk-major in the tile
-          pk[c] = *reinterpret_cast<const uint4*>(tile + (lc * kTileRows + row) * 16);
-        }
+        for (int h = 0; h < 2; ++h) {
+          const uint32_t d = (d2 >> (8 * h)) & 0xFFu;
+          const uint32_t lut_lo = 0x3C383000u - d * 0x08080800u;
+          const uint32_t lut_hi = 0x4C484440u - d * 0x08080808u;
 #pragma unroll
-        for (int c = 0; c < kChunks; ++c) {
-          const uint32_t lc = half * 2 + c;
-          uint4 a, b;
-          widen32(pk[c], lut_lo, lut_hi, a, b);
-          *reinterpret_cast<uint4*>(wrow + (((2 * lc) ^ sw128) << 4)) = a;
-          *reinterpret_cast<uint4*>(wrow + (((2 * lc + 1) ^ sw128) << 4)) = b;
+          for (int c = 0; c < 2; ++c) {
+            const uint4 v = pk[2 * h + c];
+            uint32_t* o = w + (2 * h + c) * 8;
+            widen8(v.x, lut_lo, lut_hi, o[0], o[1]);
+            widen8(v.y, lut_lo, lut_hi, o[2], o[3]);
+            widen8(v.z, lut_lo, lut_hi, o[4], o[5]);
+            widen8(v.w, lut_lo, lut_hi, o[6], o[7]);
+          }
         }
-        fence_proxy_async_smem();  // generic-proxy stores -> visible to the tensor core's async proxy
-        mbar_arrive(&wide_full[ws]);
+        const uint32_t dst = tmem_a + a * kAStageCols + lane_base;
+        tmem_st16(dst, w);
+        tmem_st16(dst + 16, w + 16);
+        tmem_st_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&a_full[a]);
       }
     }
 
     // ---- accumulators -> registers -> y
-    const bool epi_role = NONE ? (grpB == 1) : true;
+    const bool epi_role = NONE ? (warp >= 10) : true;
     if (epi_role) {
+      const int half = NONE ? 0 : (warp >> 2);
       constexpr int kMyCols = NONE ? BM : (BM >= 32 ? BM / 2 : 16);
-      const int col0 = NONE ? 0 : (BM >= 32 ? grpB * (BM / 2) : 0);
-      const bool has_cols = NONE ? true : (BM >= 32 || grpB == 0);
-      const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
+      const int col0 = NONE ? 0 : (BM >= 32 ? half * (BM / 2) : 0);
+      const bool has_cols = NONE ? true : (BM >= 32 || half == 0);
+      const uint32_t t_lane = tmem_base + lane_base;
       const int tile_id = blockIdx.y * gridDim.x + blockIdx.x;
       float* my_partial = p.partials + (static_cast<size_t>(tile_id) * p.splits + blockIdx.z) * (BM * kTileN);
 
@@ -362,8 +368,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
         // per-group promotion: run += S[n, g] * (this group's FP32 partial sum)
 #pragma unroll
         for (int c = 0; c < BM; ++c) run[c] = 0.0f;
-        const int gpk = p.group / kBlockK > 0 ? p.group / kBlockK : 1;  // K blocks per group (group >= 128)
-        const int groups = (p.group >= kBlockK) ? nkb / gpk : nkb * (kBlockK / p.group);
+        const int groups = (nkb * kBlockK) / p.group;
         const int g0 = (kb0 * kBlockK) / p.group;
         const float* srow = n_ok ? p.scale + static_cast<int64_t>(n) * p.G : nullptr;
         float S_next = (srow && groups > 0) ? __ldg(srow + g0) : 0.0f;
@@ -431,7 +436,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
         }
         __threadfence();
         named_bar_sync(1, C::kEpiThreads);
-        const bool leader = NONE ? (threadIdx.x == 128) : (threadIdx.x == 0);
+        const bool leader = NONE ? (threadIdx.x == 320) : (threadIdx.x == 0);
         if (leader) {
           const int ticket = (*s_abort) ? -1 : atomicAdd(p.counters + tile_id, 1);
           *s_last = (ticket == p.splits - 1) ? 1 : 0;
@@ -513,7 +518,7 @@ int launch_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStr
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
   dim3 grid(plan.n_tiles, plan.m_tiles, plan.splits);
-  w4a8_gemm_kernel<BM, NONE><<<grid, kThreads, C::kSmemBytes, st>>>(tm_q, p);
+  w4a8_gemm_kernel<BM, NONE><<<grid, C::kThreads, C::kSmemBytes, st>>>(tm_q, p);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
 }
@@ -522,7 +527,7 @@ int launch_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStr
 
 GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
   GemmPlan pl{};
-  const int bm_max = (mode == ZQ_SCALE_NONE) ? 128 : 256;
+  const int bm_max = (mode == ZQ_SCALE_NONE) ? 64 : 256;
   int bm = 16;
   while (bm < bm_max && bm < M) bm *= 2;
   pl.bm = bm;
@@ -578,7 +583,7 @@ int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st) {
     case 16: return none ? launch_cfg<16, true>(a, plan, p, st) : launch_cfg<16, false>(a, plan, p, st);
     case 32: return none ? launch_cfg<32, true>(a, plan, p, st) : launch_cfg<32, false>(a, plan, p, st);
     case 64: return none ? launch_cfg<64, true>(a, plan, p, st) : launch_cfg<64, false>(a, plan, p, st);
-    case 128: return none ? launch_cfg<128, true>(a, plan, p, st) : launch_cfg<128, false>(a, plan, p, st);
+    case 128: return none ? ZQ_ERR_SHAPE : launch_cfg<128, false>(a, plan, p, st);
     case 256: return none ? ZQ_ERR_SHAPE : launch_cfg<256, false>(a, plan, p, st);
   }
   return ZQ_ERR_SHAPE;
