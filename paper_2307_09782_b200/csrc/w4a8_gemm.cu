@@ -69,11 +69,13 @@ struct Cfg {
   static constexpr int kDColsPad = kDCols < 32 ? 32 : kDCols;
   static constexpr int kMinBlocks = (NONE || BM > 128) ? 1 : 2;    // CTAs per SM this configuration is sized for
   static constexpr int kTmemCols = kMinBlocks == 2 ? 256 : 512;
-  static constexpr int NA = (kTmemCols - kDColsPad) / kAStageCols > 8 ? 8 : (kTmemCols - kDColsPad) / kAStageCols;
+  static constexpr int kMaxA = (kTmemCols - kDColsPad) / kAStageCols;   // widened stages that fit in TMEM
   // copy stages (packed weights + tokens): as many as fit in half (or all) of the SM's shared memory
   static constexpr int kStageBytes = kTileBytes + kTokBytes;
   static constexpr int kBudget = kMinBlocks == 2 ? 104 * 1024 : 208 * 1024;
-  static constexpr int NS = kBudget / kStageBytes > 8 ? 8 : kBudget / kStageBytes;
+  static constexpr int kMaxS = kBudget / kStageBytes;
+  // one ring: stage s = packed tile + token tile in shared memory and the widened tile in TMEM
+  static constexpr int NS = (kMaxS < kMaxA ? kMaxS : kMaxA) > 8 ? 8 : (kMaxS < kMaxA ? kMaxS : kMaxA);
   static constexpr int kEpiThreads = NONE ? 128 : 256;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int offTok = 0;
@@ -81,10 +83,10 @@ struct Cfg {
   static constexpr int offSx = offPacked + NS * kTileBytes;   // [BM] token scales
   static constexpr int offT = offSx + BM * 4;                 // [BM][8] LoRC down-projection (rank 8)
   static constexpr int offBars = offT + BM * 32;
-  static constexpr int kNumBars = 2 * NS + 2 * NA + 6;
+  static constexpr int kNumBars = 3 * NS + 6;
   static constexpr int offMisc = offBars + kNumBars * 8;
   static constexpr int kSmemBytes = offMisc + 32;
-  static_assert(NA >= 4 && NS >= 3, "pipeline too shallow");
+  static_assert(NS >= 4, "pipeline too shallow");
 };
 
 // Expand 8 packed E2M1 codes (one 32-bit word of the tile format: magnitude of element i in bits
@@ -152,11 +154,10 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   uint8_t* s_tok = smem + C::offTok;
   uint8_t* s_packed = smem + C::offPacked;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offBars);
-  uint64_t* tma_full = bars;                   // [NS] copies landed
-  uint64_t* tma_empty = bars + C::NS;          // [NS] stage may be overwritten (MMA of that K block done)
-  uint64_t* a_full = bars + 2 * C::NS;         // [NA] widened tile complete in TMEM (4 warp arrivals)
-  uint64_t* a_empty = a_full + C::NA;          // [NA] MMA that read it done
-  uint64_t* acc_full = a_empty + C::NA;        // [2]
+  uint64_t* tma_full = bars;                   // [NS] copies landed (waited by the widen warps)
+  uint64_t* a_full = bars + C::NS;             // [NS] widened tile complete in TMEM (4 warp arrivals; waited by the MMA)
+  uint64_t* empty = bars + 2 * C::NS;          // [NS] MMA of the stage's K block done: smem and TMEM stage reusable
+  uint64_t* acc_full = bars + 3 * C::NS;       // [2]
   uint64_t* acc_empty = acc_full + 2;          // [2]
   uint64_t* drain_bar = acc_full + 4;          // [1]
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::offMisc);
@@ -173,11 +174,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   if (threadIdx.x == 0) {
     for (int i = 0; i < C::NS; ++i) {
       mbar_init(&tma_full[i], 1);
-      mbar_init(&tma_empty[i], 1);
-    }
-    for (int i = 0; i < C::NA; ++i) {
       mbar_init(&a_full[i], 4);
-      mbar_init(&a_empty[i], 1);
+      mbar_init(&empty[i], 1);
     }
     mbar_init(&acc_full[0], 1);
     mbar_init(&acc_full[1], 1);
@@ -213,7 +211,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       for (int i = 0; i < nkb; ++i) {
         const int s = i % C::NS;
         const uint32_t ph = (i / C::NS) & 1;
-        if (!mbar_wait(&tma_empty[s], ph ^ 1, s_abort)) {
+        if (!mbar_wait(&empty[s], ph ^ 1, s_abort)) {
           raise_error(p, s_abort, kErrProducer);
           break;
         }
@@ -238,14 +236,15 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       int mma_count = 0;
       bool failed = false;
       for (int i = 0; i < nkb && !failed; ++i) {
-        const int s = i % C::NS, a = i % C::NA;
-        if (!mbar_wait(&tma_full[s], (i / C::NS) & 1, s_abort) ||
-            !mbar_wait(&a_full[a], (i / C::NA) & 1, s_abort)) {
+        const int s = i % C::NS;
+        // the widen warps saw the stage's copies land before they arrived here, so this one wait also
+        // orders the token tile (same barrier as the packed tile) before the MMAs that read it
+        if (!mbar_wait(&a_full[s], (i / C::NS) & 1, s_abort)) {
           failed = true;
           break;
         }
         tc_fence_after_sync();
-        const uint32_t a_addr = tmem_a + a * kAStageCols;
+        const uint32_t a_addr = tmem_a + s * kAStageCols;
         const uint64_t bdesc = umma_desc_k128(smem_u32(s_tok + s * C::kTokBytes));
 #pragma unroll
         for (int k = 0; k < kBlockK / 32; ++k) {
@@ -268,8 +267,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
           if (NONE && (mma_count % mpg) == 0) umma_commit(&acc_full[((mma_count / mpg) - 1) & 1]);
         }
         if (failed) break;
-        umma_commit(&tma_empty[s]);
-        umma_commit(&a_empty[a]);
+        umma_commit(&empty[s]);
       }
       if (failed) {
         raise_error(p, s_abort, kErrMma);
@@ -294,9 +292,10 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       // A lane widens whole rows: 64 packed bytes -> 128 E4M3 bytes = 32 TMEM columns of its own lane.
       const int grp = warp >> 2;
       for (int i = grp; i < nkb; i += kWidenGroups) {
-        const int s = i % C::NS, a = i % C::NA;
-        if (!mbar_wait(&tma_full[s], (i / C::NS) & 1, s_abort) ||
-            !mbar_wait(&a_empty[a], ((i / C::NA) & 1) ^ 1, s_abort)) {
+        const int s = i % C::NS;
+        // tma_full(i) implies empty(i - NS): the producer refilled the stage only after that MMA was done,
+        // so the TMEM stage is free as well
+        if (!mbar_wait_warp(&tma_full[s], (i / C::NS) & 1, s_abort)) {
           raise_error(p, s_abort, kErrWiden);
           failed = true;
           break;
@@ -324,13 +323,13 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
             widen8(v.w, lut_lo, lut_hi, o[6], o[7]);
           }
         }
-        const uint32_t dst = tmem_a + a * kAStageCols + lane_base;
+        const uint32_t dst = tmem_a + s * kAStageCols + lane_base;
         tmem_st16(dst, w);
         tmem_st16(dst + 16, w + 16);
         tmem_st_wait();
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&a_full[a]);
+        if (lane == 0) mbar_arrive(&a_full[s]);
       }
     }
 
@@ -376,7 +375,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
           const int b = g & 1;
           const float S = S_next;
           if (srow && g + 1 < groups) S_next = __ldg(srow + g0 + g + 1);
-          if (!mbar_wait(&acc_full[b], (g >> 1) & 1, s_abort)) {
+          if (!mbar_wait_warp(&acc_full[b], (g >> 1) & 1, s_abort)) {
             raise_error(p, s_abort, kErrPromote);
             failed = true;
             break;
@@ -394,7 +393,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
           mbar_arrive(&acc_empty[b]);
         }
       } else if (!failed) {
-        if (!mbar_wait(&acc_full[0], 0, s_abort)) {
+        if (!mbar_wait_warp(&acc_full[0], 0, s_abort)) {
           raise_error(p, s_abort, kErrEpilogue);
           failed = true;
         }
