@@ -338,6 +338,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     if (epi_role) {
       const int half = NONE ? 0 : (warp >> 2);
       constexpr int kMyCols = NONE ? BM : (BM >= 32 ? BM / 2 : 16);
+      // Mode none keeps its running sums in a register array, which needs the column loop unrolled; the
+      // other modes keep the loop rolled so that its body stays resident in the instruction cache.
+      constexpr int kEpiUnroll = NONE ? kMyCols / 16 : 1;
       const int col0 = NONE ? 0 : (BM >= 32 ? half * (BM / 2) : 0);
       const bool has_cols = NONE ? true : (BM >= 32 || half == 0);
       const uint32_t t_lane = tmem_base + lane_base;
@@ -402,7 +405,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
 
       if (p.splits == 1) {
         if (!failed && has_cols) {
-#pragma unroll
+#pragma unroll(kEpiUnroll)
           for (int c = 0; c < kMyCols; c += 16) {
             float v[16];
             if (NONE) {
@@ -419,7 +422,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
         // split-K: leave the raw partial sums in the workspace; the CTA that arrives last for this
         // output tile adds all of them in split order (deterministic) and finishes the tile.
         if (!failed && has_cols) {
-#pragma unroll
+#pragma unroll(kEpiUnroll)
           for (int c = 0; c < kMyCols; c += 16) {
             float v[16];
             if (NONE) {
