@@ -15,13 +15,14 @@
 // mapping for widening (a thread writes its own TMEM lane) and turns every per-channel quantity
 // (scale, shift, U row, group scale) into a per-thread scalar in the epilogue.
 //
-// Warp roles:
-//   0-7   two widen groups of four warps (one warp per TMEM lane quarter); group g widens the K blocks
-//         i with i % 2 == g, so two K blocks are in flight and the hand-off latencies overlap.
-//         M1/M2: the same warps run the epilogue (group g takes half of the columns).
-//   8     TMA / bulk-copy producer (one lane)
-//   9     TMEM allocation, MMA issue (one lane)
-//   10-13 mode none only: per-group promotion (TMEM -> registers, times the FP32 group scale), epilogue
+// Warp roles (NG = 2 widen groups, 4 for the 256-token tile):
+//   0 .. 4NG-1   widen groups of four warps (one warp per TMEM lane quarter); group g widens the K
+//                blocks i with i % NG == g, so NG K blocks are in flight and the hand-off latencies
+//                overlap.  M1/M2: the same warps run the epilogue (group g takes 1/NG of the columns).
+//   4NG          TMA / bulk-copy producer (one lane)
+//   4NG+1        TMEM allocation, MMA issue (one lane)
+//   4NG+2 .. +5  mode none only: per-group promotion (TMEM -> registers, times the FP32 group scale)
+//                and the epilogue
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -35,7 +36,6 @@ namespace {
 constexpr int kTileN = 128;   // output channels per CTA (MMA M extent)
 constexpr int kBlockK = 128;  // K elements per pipeline step
 constexpr int kAStageCols = kBlockK / 4;  // TMEM columns of one widened 128 x 128 tile (4 bytes per column)
-constexpr int kWidenGroups = 2;
 
 // error detail codes written to status[1]
 enum { kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6 };
@@ -63,7 +63,13 @@ struct Params {
 
 template <int BM, bool NONE>
 struct Cfg {
-  static constexpr int kThreads = NONE ? 448 : 320;
+  // widen groups of four warps each; group g takes the K blocks i with i % NG == g
+  static constexpr int NG = (!NONE && BM > 128) ? 4 : 2;
+  static constexpr int kWidenWarps = 4 * NG;
+  static constexpr int kProducerWarp = kWidenWarps;
+  static constexpr int kMmaWarp = kWidenWarps + 1;
+  static constexpr int kPromoteWarp0 = kWidenWarps + 2;  // mode none: four promotion / epilogue warps
+  static constexpr int kThreads = 32 * (kWidenWarps + 2 + (NONE ? 4 : 0));
   static constexpr int kTokBytes = BM * kBlockK;
   static constexpr int kDCols = NONE ? 2 * BM : BM;                 // accumulator columns (two buffers in mode none)
   static constexpr int kDColsPad = kDCols < 32 ? 32 : kDCols;
@@ -75,8 +81,11 @@ struct Cfg {
   static constexpr int kBudget = kMinBlocks == 2 ? 104 * 1024 : 208 * 1024;
   static constexpr int kMaxS = kBudget / kStageBytes;
   // one ring: stage s = packed tile + token tile in shared memory and the widened tile in TMEM
-  static constexpr int NS = (kMaxS < kMaxA ? kMaxS : kMaxA) > 8 ? 8 : (kMaxS < kMaxA ? kMaxS : kMaxA);
-  static constexpr int kEpiThreads = NONE ? 128 : 256;
+  // The depth is a multiple of NG, so that a stage is always widened by the same group: that group
+  // then sees every round of the stage's barrier in order, which a parity wait needs.
+  static constexpr int kMaxStages = (kMaxS < kMaxA ? kMaxS : kMaxA) > 8 ? 8 : (kMaxS < kMaxA ? kMaxS : kMaxA);
+  static constexpr int NS = kMaxStages / NG * NG;
+  static constexpr int kEpiThreads = NONE ? 128 : 128 * NG;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int offTok = 0;
   static constexpr int offPacked = offTok + NS * kTokBytes;
@@ -86,7 +95,7 @@ struct Cfg {
   static constexpr int kNumBars = 3 * NS + 6;
   static constexpr int offMisc = offBars + kNumBars * 8;
   static constexpr int kSmemBytes = offMisc + 32;
-  static_assert(NS >= 4, "pipeline too shallow");
+  static_assert(NS >= 4 && NS % NG == 0, "pipeline too shallow or not a multiple of the widen groups");
 };
 
 // Expand 8 packed E2M1 codes (one 32-bit word of the tile format: magnitude of element i in bits
@@ -187,15 +196,15 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     fence_mbar_init();
     if ((smem_u32(smem) & 1023u) != 0) raise_error(p, s_abort, kErrAlign);
   }
-  if (warp == 8 && lane == 0) prefetch_tensormap(&tm_q);
-  if (warp < 8) {
+  if (warp == C::kProducerWarp && lane == 0) prefetch_tensormap(&tm_q);
+  if (warp < C::kWidenWarps) {
     // token scales and (rank 8) LoRC rows of this tile's tokens, for the epilogue
-    for (int c = threadIdx.x; c < BM; c += 256) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
+    for (int c = threadIdx.x; c < BM; c += 32 * C::kWidenWarps) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
     if (p.r == 8)
-      for (int c = threadIdx.x; c < BM * 8; c += 256)
+      for (int c = threadIdx.x; c < BM * 8; c += 32 * C::kWidenWarps)
         s_t[c] = (m0 + (c >> 3) < p.M) ? __ldg(p.t + static_cast<int64_t>(m0) * 8 + c) : 0.0f;
   }
-  if (warp == 9) tmem_alloc(s_tmem, C::kTmemCols);
+  if (warp == C::kMmaWarp) tmem_alloc(s_tmem, C::kTmemCols);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -203,7 +212,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   const uint32_t tmem_a = tmem_base + C::kDColsPad;  // widened-weight stages follow the accumulators
   const bool ok_start = (*s_abort == 0);
 
-  if (warp == 8) {
+  if (warp == C::kProducerWarp) {
     // ------------------------------------------------------------------ copy producer
     if (lane == 0 && ok_start) {
       const uint8_t* wtiles = p.codes + (static_cast<int64_t>(blockIdx.x) * p.kblocks + kb0) * kTileBytes;
@@ -228,7 +237,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
         }
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == C::kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && ok_start) {
       const uint32_t idesc = umma_idesc_e4m3(BM);
@@ -288,11 +297,12 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     const uint32_t lane_base = static_cast<uint32_t>(q4 * 32) << 16;
     bool failed = !ok_start;
 
-    if (warp < 8 && !failed) {
+    if (warp < C::kWidenWarps && !failed) {
       // A lane widens whole rows: 64 packed bytes -> 128 E4M3 bytes = 32 TMEM columns of its own lane.
       const int grp = warp >> 2;
-      for (int i = grp; i < nkb; i += kWidenGroups) {
+      for (int i = grp; i < nkb; i += C::NG) {
         const int s = i % C::NS;
+        // stage s is always this group's (NS % NG == 0), so the parity below is unambiguous;
         // tma_full(i) implies empty(i - NS): the producer refilled the stage only after that MMA was done,
         // so the TMEM stage is free as well
         if (!mbar_wait_warp(&tma_full[s], (i / C::NS) & 1, s_abort)) {
@@ -334,15 +344,15 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     }
 
     // ---- accumulators -> registers -> y
-    const bool epi_role = NONE ? (warp >= 10) : true;
+    const bool epi_role = NONE ? (warp >= C::kPromoteWarp0) : true;
     if (epi_role) {
-      const int half = NONE ? 0 : (warp >> 2);
-      constexpr int kMyCols = NONE ? BM : (BM >= 32 ? BM / 2 : 16);
+      const int part = NONE ? 0 : (warp >> 2);  // which share of the columns this widen group finishes
+      constexpr int kMyCols = NONE ? BM : (BM / C::NG >= 16 ? BM / C::NG : 16);
       // Mode none keeps its running sums in a register array, which needs the column loop unrolled; the
       // other modes keep the loop rolled so that its body stays resident in the instruction cache.
       constexpr int kEpiUnroll = NONE ? kMyCols / 16 : 1;
-      const int col0 = NONE ? 0 : (BM >= 32 ? half * (BM / 2) : 0);
-      const bool has_cols = NONE ? true : (BM >= 32 || half == 0);
+      const int col0 = NONE ? 0 : part * kMyCols;
+      const bool has_cols = NONE ? true : (col0 < BM);
       const uint32_t t_lane = tmem_base + lane_base;
       const int tile_id = blockIdx.y * gridDim.x + blockIdx.x;
       float* my_partial = p.partials + (static_cast<size_t>(tile_id) * p.splits + blockIdx.z) * (BM * kTileN);
@@ -438,7 +448,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
         }
         __threadfence();
         named_bar_sync(1, C::kEpiThreads);
-        const bool leader = NONE ? (threadIdx.x == 320) : (threadIdx.x == 0);
+        const bool leader = NONE ? (threadIdx.x == 32 * C::kPromoteWarp0) : (threadIdx.x == 0);
         if (leader) {
           const int ticket = (*s_abort) ? -1 : atomicAdd(p.counters + tile_id, 1);
           *s_last = (ticket == p.splits - 1) ? 1 : 0;
@@ -467,7 +477,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
 
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == C::kMmaWarp) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, C::kTmemCols);
   }
