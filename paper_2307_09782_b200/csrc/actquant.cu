@@ -178,11 +178,135 @@ act_quant_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, uint8_t* _
   }
 }
 
+// ---- many tokens: eight rows per CTA -------------------------------------------------------------
+// With one row per CTA every row re-reads all of V (r x K fp16) from L2, eight times the bytes of the
+// row itself at rank 8.  Here a thread converts its slice of V to FP32 once and applies it to eight
+// rows, so V costs no more than x.  Pass 1 streams the rows once from HBM for absmax and t; pass 2
+// reads them again (they are still in L2: 8 rows per CTA) for the cast.
+constexpr int kRows = 8;
+constexpr int kRowsThreads = 256;
+
+template <bool HAS_V>
+__global__ void __launch_bounds__(kRowsThreads)
+act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec, uint8_t* __restrict__ q,
+                      float* __restrict__ sx, const uint4* __restrict__ V, float* __restrict__ t) {
+  __shared__ float s_amax[kRowsThreads / 32][kRows];
+  __shared__ float s_acc[kRowsThreads / 32][kRows * 8];
+  __shared__ float s_inv[kRows];
+  const int m0 = blockIdx.x * kRows;
+  const int nrows = min(kRows, M - m0);
+  const int nvec = K / 8;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint4* xr = x + static_cast<int64_t>(m0) * ldx_vec;
+
+  float amax[kRows];
+  float acc[kRows][8];
+#pragma unroll
+  for (int r = 0; r < kRows; ++r) {
+    amax[r] = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[r][j] = 0.0f;
+  }
+  for (int u = tid; u < nvec; u += kRowsThreads) {
+    uint4 xv[kRows];
+#pragma unroll
+    for (int r = 0; r < kRows; ++r)
+      xv[r] = (r < nrows) ? __ldg(xr + r * ldx_vec + u) : make_uint4(0, 0, 0, 0);
+    float vf[8][8];
+    if (HAS_V) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint4 vv = __ldg(V + static_cast<int64_t>(j) * nvec + u);
+        const uint32_t vw[4] = {vv.x, vv.y, vv.z, vv.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __half2 h;
+          *reinterpret_cast<uint32_t*>(&h) = vw[e];
+          const float2 f = __half22float2(h);
+          vf[j][2 * e] = f.x;
+          vf[j][2 * e + 1] = f.y;
+        }
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < kRows; ++r) {
+      const uint32_t w[4] = {xv[r].x, xv[r].y, xv[r].z, xv[r].w};
+      float xf[8];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        xf[2 * e] = bf16_lo(w[e]);
+        xf[2 * e + 1] = bf16_hi(w[e]);
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) amax[r] = fmaxf(amax[r], fabsf(xf[e]));
+      if (HAS_V) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[r][j] = fmaf(xf[e], vf[j][e], acc[r][j]);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < kRows; ++r) {
+    const float a = warp_max(amax[r]);
+    if (lane == 0) s_amax[warp][r] = a;
+    if (HAS_V) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float v = warp_sum(acc[r][j]);
+        if (lane == 0) s_acc[warp][r * 8 + j] = v;
+      }
+    }
+  }
+  __syncthreads();
+  if (tid < kRows) {
+    float a = s_amax[0][tid];
+    for (int w = 1; w < kRowsThreads / 32; ++w) a = fmaxf(a, s_amax[w][tid]);
+    float s = 1.0f, inv = 1.0f;
+    if (a != 0.0f) {
+      s = __fdiv_rn(a, 448.0f);
+      inv = __fdiv_rn(448.0f, a);
+    }
+    s_inv[tid] = inv;
+    if (tid < nrows) sx[m0 + tid] = s;
+  }
+  if (HAS_V && tid < kRows * 8 && (tid >> 3) < nrows) {
+    float v = 0.0f;
+    for (int w = 0; w < kRowsThreads / 32; ++w) v += s_acc[w][tid];
+    t[static_cast<int64_t>(m0) * 8 + tid] = v;
+  }
+  __syncthreads();
+  const int nunits = K / kUnit;
+  for (int r = 0; r < nrows; ++r) {
+    const float inv = s_inv[r];
+    const uint4* row = xr + r * ldx_vec;
+    uint4* qrow = reinterpret_cast<uint4*>(q + static_cast<int64_t>(m0 + r) * K);
+    for (int u = tid; u < nunits; u += kRowsThreads) {
+      const uint2 lo = cast8(__ldg(row + 2 * u), inv), hi = cast8(__ldg(row + 2 * u + 1), inv);
+      qrow[u] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+    }
+  }
+}
+
 }  // namespace
 
 int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
                      const void* V, int r, float* t, cudaStream_t st) {
   if (M == 0) return ZQ_OK;
+  // enough rows to fill the GPU with eight-row CTAs, and the rank the row kernel is written for
+  if (M >= 8 * 148 && (V == nullptr || r == 8)) {
+    dim3 grid(static_cast<unsigned>((M + kRows - 1) / kRows));
+    if (V)
+      act_quant_rows_kernel<true><<<grid, kRowsThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(M),
+                                                                static_cast<int>(K), ldx / 8, q, sx,
+                                                                static_cast<const uint4*>(V), t);
+    else
+      act_quant_rows_kernel<false><<<grid, kRowsThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(M),
+                                                                 static_cast<int>(K), ldx / 8, q, sx, nullptr, t);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+  }
   const int nunits = static_cast<int>(K / kUnit);
   int threads = ((nunits + 31) / 32) * 32;
   if (threads > kMaxThreads) threads = kMaxThreads;

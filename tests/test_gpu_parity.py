@@ -26,6 +26,20 @@ def test_act_quant_bit_exact(M, K):
     assert np.abs(host(t) - t_o).max() <= 1e-4 * np.abs(t_o).max()
 
 
+@pytest.mark.parametrize("M,K,lorc", [(1187, 768, True), (1184, 2048, False), (2500, 256, True)])
+def test_act_quant_many_rows_kernel(M, K, lorc):
+    """Token counts large enough for the eight-rows-per-CTA kernel, with a ragged last CTA."""
+    x_bits = synth.make_x(300 + M, M, K, max(1, K // 100), 20.0)
+    x_bits[5] = 0                                 # an all-zero token
+    V = synth.make_lorc(300 + M, 8, K, 8)[1] if lorc else None
+    q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
+    q, sx, t = binding.quantize_act_fp8(to_bf16(x_bits), up(V))
+    assert np.array_equal(host(q), q_o)
+    assert np.array_equal(host(sx).view(np.uint32), sx_o.view(np.uint32))
+    if lorc:
+        assert np.abs(host(t) - t_o).max() <= 1e-4 * np.abs(t_o).max()
+
+
 def test_act_quant_edge_rows_and_strided_input():
     K = 256
     x = np.zeros((6, K), dtype=np.float32)
