@@ -217,17 +217,24 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     if (lane == 0 && ok_start) {
       const uint8_t* wtiles = p.codes + (static_cast<int64_t>(blockIdx.x) * p.kblocks + kb0) * kTileBytes;
       int issued = 0;
-      for (int i = 0; i < nkb; ++i) {
-        const int s = i % C::NS;
-        const uint32_t ph = (i / C::NS) & 1;
-        if (!mbar_wait(&empty[s], ph ^ 1, s_abort)) {
-          raise_error(p, s_abort, kErrProducer);
-          break;
+      bool stop = false;
+      for (int i0 = 0; i0 < nkb && !stop; i0 += C::NS) {  // one ring round per outer iteration
+        const uint32_t ph = (i0 / C::NS) & 1;
+#pragma unroll
+        for (int s = 0; s < C::NS; ++s) {
+          const int i = i0 + s;
+          if (i >= nkb) break;
+          if (!mbar_wait(&empty[s], ph ^ 1, s_abort)) {
+            raise_error(p, s_abort, kErrProducer);
+            stop = true;
+            break;
+          }
+          mbar_arrive_expect_tx(&tma_full[s], kTileBytes + C::kTokBytes);
+          bulk_load(s_packed + s * kTileBytes, wtiles + static_cast<int64_t>(i) * kTileBytes, kTileBytes,
+                    &tma_full[s]);
+          tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, (kb0 + i) * kBlockK, m0, &tma_full[s]);
+          issued = i + 1;
         }
-        mbar_arrive_expect_tx(&tma_full[s], kTileBytes + C::kTokBytes);
-        bulk_load(s_packed + s * kTileBytes, wtiles + static_cast<int64_t>(i) * kTileBytes, kTileBytes, &tma_full[s]);
-        tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, (kb0 + i) * kBlockK, m0, &tma_full[s]);
-        issued = i + 1;
       }
       // never leave with copies still in flight: wait (bounded) for the last phase issued per stage
       for (int i = max(0, issued - C::NS); i < issued; ++i) {
@@ -244,39 +251,45 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       const int mpg = p.group / 32;  // MMAs per weight group (mode none)
       int mma_count = 0;
       bool failed = false;
-      for (int i = 0; i < nkb && !failed; ++i) {
-        const int s = i % C::NS;
-        // the widen warps saw the stage's copies land before they arrived here, so this one wait also
-        // orders the token tile (same barrier as the packed tile) before the MMAs that read it
-        if (!mbar_wait(&a_full[s], (i / C::NS) & 1, s_abort)) {
-          failed = true;
-          break;
-        }
-        tc_fence_after_sync();
-        const uint32_t a_addr = tmem_a + s * kAStageCols;
-        const uint64_t bdesc = umma_desc_k128(smem_u32(s_tok + s * C::kTokBytes));
+      const uint64_t bdesc0 = umma_desc_k128(smem_u32(s_tok));
+      for (int i0 = 0; i0 < nkb && !failed; i0 += C::NS) {  // one ring round per outer iteration
+        const uint32_t ph = (i0 / C::NS) & 1;
 #pragma unroll
-        for (int k = 0; k < kBlockK / 32; ++k) {
-          uint32_t d_tmem = tmem_base;
-          uint32_t accumulate = (i > 0 || k > 0) ? 1u : 0u;
-          if (NONE) {
-            const int grp = mma_count / mpg, within = mma_count % mpg, b = grp & 1;
-            if (within == 0) {
-              if (!mbar_wait(&acc_empty[b], ((grp >> 1) & 1) ^ 1, s_abort)) {
-                failed = true;
-                break;
-              }
-              tc_fence_after_sync();
-            }
-            d_tmem = tmem_base + b * BM;
-            accumulate = within > 0 ? 1u : 0u;
+        for (int s = 0; s < C::NS; ++s) {
+          const int i = i0 + s;
+          if (i >= nkb || failed) break;
+          // the widen warps saw the stage's copies land before they arrived here, so this one wait also
+          // orders the token tile (same barrier as the packed tile) before the MMAs that read it
+          if (!mbar_wait(&a_full[s], ph, s_abort)) {
+            failed = true;
+            break;
           }
-          umma_f8_tmem_a(d_tmem, a_addr + 8 * k, bdesc + 2 * k, idesc, accumulate);
-          ++mma_count;
-          if (NONE && (mma_count % mpg) == 0) umma_commit(&acc_full[((mma_count / mpg) - 1) & 1]);
+          tc_fence_after_sync();
+          const uint32_t a_addr = tmem_a + s * kAStageCols;
+          const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((s * C::kTokBytes) >> 4);
+#pragma unroll
+          for (int k = 0; k < kBlockK / 32; ++k) {
+            uint32_t d_tmem = tmem_base;
+            uint32_t accumulate = (i > 0 || k > 0) ? 1u : 0u;
+            if (NONE) {
+              const int grp = mma_count / mpg, within = mma_count % mpg, b = grp & 1;
+              if (within == 0) {
+                if (!mbar_wait(&acc_empty[b], ((grp >> 1) & 1) ^ 1, s_abort)) {
+                  failed = true;
+                  break;
+                }
+                tc_fence_after_sync();
+              }
+              d_tmem = tmem_base + b * BM;
+              accumulate = within > 0 ? 1u : 0u;
+            }
+            umma_f8_tmem_a(d_tmem, a_addr + 8 * k, bdesc + 2 * k, idesc, accumulate);
+            ++mma_count;
+            if (NONE && (mma_count % mpg) == 0) umma_commit(&acc_full[((mma_count / mpg) - 1) & 1]);
+          }
+          if (failed) break;
+          umma_commit(&empty[s]);
         }
-        if (failed) break;
-        umma_commit(&empty[s]);
       }
       if (failed) {
         raise_error(p, s_abort, kErrMma);
@@ -300,12 +313,16 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     if (warp < C::kWidenWarps && !failed) {
       // A lane widens whole rows: 64 packed bytes -> 128 E4M3 bytes = 32 TMEM columns of its own lane.
       const int grp = warp >> 2;
-      for (int i = grp; i < nkb; i += C::NG) {
-        const int s = i % C::NS;
-        // stage s is always this group's (NS % NG == 0), so the parity below is unambiguous;
-        // tma_full(i) implies empty(i - NS): the producer refilled the stage only after that MMA was done,
-        // so the TMEM stage is free as well
-        if (!mbar_wait_warp(&tma_full[s], (i / C::NS) & 1, s_abort)) {
+      for (int i0 = 0; i0 < nkb && !failed; i0 += C::NS)  // one ring round per outer iteration
+#pragma unroll
+      for (int ss = 0; ss < C::NS / C::NG; ++ss) {
+        // stage s is always this group's (NS % NG == 0), so the group sees every round of the stage's
+        // barrier and the parity below is unambiguous; tma_full(i) implies empty(i - NS): the producer
+        // refilled the stage only after that MMA was done, so the TMEM stage is free as well
+        const int s = grp + ss * C::NG;
+        const int i = i0 + s;
+        if (i >= nkb || failed) break;
+        if (!mbar_wait_warp(&tma_full[s], (i0 / C::NS) & 1, s_abort)) {
           raise_error(p, s_abort, kErrWiden);
           failed = true;
           break;

@@ -73,8 +73,9 @@ int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st);
 
 #ifdef __CUDACC__
 // ---- device: bounded waits -----------------------------------------------------------------------
-// Every spin in this library gives up after kSpinLimit polls; the kernel then records an error in the
-// workspace status word and unwinds instead of hanging.
+// Every wait in this library is bounded (a poll count and, for the parked waits, two seconds of
+// wall time); when one runs out the kernel records an error in the workspace status word and
+// unwinds instead of hanging.
 constexpr uint32_t kSpinLimit = 1u << 24;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -105,14 +106,34 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Returns false when the wait ran out or another thread of the CTA already raised `abort_flag`.
+// The same test, but the hardware may park the thread for up to `hint_ns` while the phase is pending
+// (it resumes as soon as the phase completes), so a waiting warp costs almost no issue slots.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when kWaitLimitNs passed or another thread of the CTA already raised
+// `abort_flag`; the caller then records the error and unwinds.
+constexpr uint64_t kWaitLimitNs = 2000000000ull;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer_ns();
   for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (spin > 64) {
-      if (*abort_flag) return false;
-      if (spin > 4096) __nanosleep(64);
-    }
+    if (mbar_try_wait_parked(bar, parity, 50000u)) return true;
+    if (*abort_flag) return false;
+    if ((spin & 7u) == 7u && global_timer_ns() - t0 > kWaitLimitNs) return false;
   }
   return false;
 }
