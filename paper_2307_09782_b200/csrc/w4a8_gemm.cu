@@ -15,14 +15,23 @@
 // mapping for widening (a thread writes its own TMEM lane) and turns every per-channel quantity
 // (scale, shift, U row, group scale) into a per-thread scalar in the epilogue.
 //
-// Warp roles (NG = 2 widen groups, 4 for the 256-token tile):
+// Three rings, each as deep as its own resource allows, because the copy -> widen -> MMA -> release
+// chain is several K blocks long and each resource is held for a different part of it:
+//   P  packed weight tiles in shared memory   producer -> widen warps     (released by the widen warps)
+//   T  token tiles in shared memory           producer -> MMA             (released by tcgen05.commit)
+//   A  widened weight tiles in tensor memory  widen warps -> MMA          (released by tcgen05.commit)
+//
+// Warp roles (NG widen groups):
 //   0 .. 4NG-1   widen groups of four warps (one warp per TMEM lane quarter); group g widens the K
 //                blocks i with i % NG == g, so NG K blocks are in flight and the hand-off latencies
 //                overlap.  M1/M2: the same warps run the epilogue (group g takes 1/NG of the columns).
-//   4NG          TMA / bulk-copy producer (one lane)
-//   4NG+1        TMEM allocation, MMA issue (one lane)
-//   4NG+2 .. +5  mode none only: per-group promotion (TMEM -> registers, times the FP32 group scale)
+//   4NG          packed-weight producer (bulk copies, one lane)
+//   4NG+1        token producer (TMA, one lane)
+//   4NG+2        TMEM allocation, MMA issue (one lane)
+//   4NG+3 .. +6  mode none only: per-group promotion (TMEM -> registers, times the FP32 group scale)
 //                and the epilogue
+// Ring depths NP and NA are multiples of NG, so a P or A stage is always handled by the same widen
+// group; that group then sees every round of the stage's barriers, which a parity wait needs.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -61,41 +70,40 @@ struct Params {
   float* partials;
 };
 
+constexpr int cmin(int a, int b) { return a < b ? a : b; }
+
 template <int BM, bool NONE>
 struct Cfg {
-  // widen groups of four warps each; group g takes the K blocks i with i % NG == g
-  static constexpr int NG = (!NONE && BM > 128) ? 4 : 2;
+  static constexpr int NG = 2;  // widen groups
   static constexpr int kWidenWarps = 4 * NG;
-  static constexpr int kProducerWarp = kWidenWarps;
-  static constexpr int kMmaWarp = kWidenWarps + 1;
-  static constexpr int kPromoteWarp0 = kWidenWarps + 2;  // mode none: four promotion / epilogue warps
-  static constexpr int kThreads = 32 * (kWidenWarps + 2 + (NONE ? 4 : 0));
+  static constexpr int kWeightWarp = kWidenWarps;
+  static constexpr int kTokenWarp = kWidenWarps + 1;
+  static constexpr int kMmaWarp = kWidenWarps + 2;
+  static constexpr int kPromoteWarp0 = kWidenWarps + 3;  // mode none: four promotion / epilogue warps
+  static constexpr int kThreads = 32 * (kWidenWarps + 3 + (NONE ? 4 : 0));
   static constexpr int kTokBytes = BM * kBlockK;
   static constexpr int kDCols = NONE ? 2 * BM : BM;                 // accumulator columns (two buffers in mode none)
   static constexpr int kDColsPad = kDCols < 32 ? 32 : kDCols;
   static constexpr int kMinBlocks = (NONE || BM > 128) ? 1 : 2;    // CTAs per SM this configuration is sized for
   static constexpr int kTmemCols = kMinBlocks == 2 ? 256 : 512;
-  static constexpr int kMaxA = (kTmemCols - kDColsPad) / kAStageCols;   // widened stages that fit in TMEM
-  // copy stages (packed weights + tokens): as many as fit in half (or all) of the SM's shared memory
-  static constexpr int kStageBytes = kTileBytes + kTokBytes;
-  static constexpr int kBudget = kMinBlocks == 2 ? 104 * 1024 : 208 * 1024;
-  static constexpr int kMaxS = kBudget / kStageBytes;
-  // one ring: stage s = packed tile + token tile in shared memory and the widened tile in TMEM
-  // The depth is a multiple of NG, so that a stage is always widened by the same group: that group
-  // then sees every round of the stage's barrier in order, which a parity wait needs.
-  static constexpr int kMaxStages = (kMaxS < kMaxA ? kMaxS : kMaxA) > 8 ? 8 : (kMaxS < kMaxA ? kMaxS : kMaxA);
-  static constexpr int NS = kMaxStages / NG * NG;
+  static constexpr int NA = cmin(8, (kTmemCols - kDColsPad) / kAStageCols) / NG * NG;  // widened stages in TMEM
+  // shared memory: token stages first (as many as the chain needs, at most 10), the rest to packed stages
+  static constexpr int kBudget = (kMinBlocks == 2 ? 104 : 220) * 1024 - BM * 36 - 512;
+  static constexpr int kBoth = cmin(10, kBudget / (kTileBytes + kTokBytes));
+  static constexpr int NT = kBoth;
+  static constexpr int NP = cmin(12, (kBudget - NT * kTokBytes) / kTileBytes) / NG * NG;
   static constexpr int kEpiThreads = NONE ? 128 : 128 * NG;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int offTok = 0;
-  static constexpr int offPacked = offTok + NS * kTokBytes;
-  static constexpr int offSx = offPacked + NS * kTileBytes;   // [BM] token scales
+  static constexpr int offPacked = offTok + NT * kTokBytes;
+  static constexpr int offSx = offPacked + NP * kTileBytes;   // [BM] token scales
   static constexpr int offT = offSx + BM * 4;                 // [BM][8] LoRC down-projection (rank 8)
   static constexpr int offBars = offT + BM * 32;
-  static constexpr int kNumBars = 3 * NS + 6;
+  static constexpr int kNumBars = 2 * NP + 2 * NT + 2 * NA + 6;
   static constexpr int offMisc = offBars + kNumBars * 8;
   static constexpr int kSmemBytes = offMisc + 32;
-  static_assert(NS >= 4 && NS % NG == 0, "pipeline too shallow or not a multiple of the widen groups");
+  static_assert(NA >= NG && NP >= NG && NT >= 3 && NA % NG == 0 && NP % NG == 0, "ring depths");
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory");
 };
 
 // Expand 8 packed E2M1 codes (one 32-bit word of the tile format: magnitude of element i in bits
@@ -163,10 +171,13 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   uint8_t* s_tok = smem + C::offTok;
   uint8_t* s_packed = smem + C::offPacked;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offBars);
-  uint64_t* tma_full = bars;                   // [NS] copies landed (waited by the widen warps)
-  uint64_t* a_full = bars + C::NS;             // [NS] widened tile complete in TMEM (4 warp arrivals; waited by the MMA)
-  uint64_t* empty = bars + 2 * C::NS;          // [NS] MMA of the stage's K block done: smem and TMEM stage reusable
-  uint64_t* acc_full = bars + 3 * C::NS;       // [2]
+  uint64_t* p_full = bars;                     // [NP] packed tile landed            (widen warps wait)
+  uint64_t* p_empty = p_full + C::NP;          // [NP] packed tile read (4 warps)    (weight producer waits)
+  uint64_t* t_full = p_empty + C::NP;          // [NT] token tile landed             (MMA waits)
+  uint64_t* t_empty = t_full + C::NT;          // [NT] MMAs that read it done        (token producer waits)
+  uint64_t* a_full = t_empty + C::NT;          // [NA] widened tile in TMEM (4 warps) (MMA waits)
+  uint64_t* a_empty = a_full + C::NA;          // [NA] MMAs that read it done        (widen warps wait)
+  uint64_t* acc_full = a_empty + C::NA;        // [2]
   uint64_t* acc_empty = acc_full + 2;          // [2]
   uint64_t* drain_bar = acc_full + 4;          // [1]
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::offMisc);
@@ -181,10 +192,17 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   const int nkb = min(p.kb_per_split, p.kblocks - kb0);
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < C::NS; ++i) {
-      mbar_init(&tma_full[i], 1);
+    for (int i = 0; i < C::NP; ++i) {
+      mbar_init(&p_full[i], 1);
+      mbar_init(&p_empty[i], 4);
+    }
+    for (int i = 0; i < C::NT; ++i) {
+      mbar_init(&t_full[i], 1);
+      mbar_init(&t_empty[i], 1);
+    }
+    for (int i = 0; i < C::NA; ++i) {
       mbar_init(&a_full[i], 4);
-      mbar_init(&empty[i], 1);
+      mbar_init(&a_empty[i], 1);
     }
     mbar_init(&acc_full[0], 1);
     mbar_init(&acc_full[1], 1);
@@ -196,7 +214,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     fence_mbar_init();
     if ((smem_u32(smem) & 1023u) != 0) raise_error(p, s_abort, kErrAlign);
   }
-  if (warp == C::kProducerWarp && lane == 0) prefetch_tensormap(&tm_q);
+  if (warp == C::kTokenWarp && lane == 0) prefetch_tensormap(&tm_q);
   if (warp < C::kWidenWarps) {
     // token scales and (rank 8) LoRC rows of this tile's tokens, for the epilogue
     for (int c = threadIdx.x; c < BM; c += 32 * C::kWidenWarps) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
@@ -212,35 +230,53 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   const uint32_t tmem_a = tmem_base + C::kDColsPad;  // widened-weight stages follow the accumulators
   const bool ok_start = (*s_abort == 0);
 
-  if (warp == C::kProducerWarp) {
-    // ------------------------------------------------------------------ copy producer
+  if (warp == C::kWeightWarp) {
+    // ------------------------------------------------------------------ packed-weight producer
     if (lane == 0 && ok_start) {
       const uint8_t* wtiles = p.codes + (static_cast<int64_t>(blockIdx.x) * p.kblocks + kb0) * kTileBytes;
-      int issued = 0;
-      bool stop = false;
-      for (int i0 = 0; i0 < nkb && !stop; i0 += C::NS) {  // one ring round per outer iteration
-        const uint32_t ph = (i0 / C::NS) & 1;
-#pragma unroll
-        for (int s = 0; s < C::NS; ++s) {
-          const int i = i0 + s;
-          if (i >= nkb) break;
-          if (!mbar_wait(&empty[s], ph ^ 1, s_abort)) {
-            raise_error(p, s_abort, kErrProducer);
-            stop = true;
-            break;
-          }
-          mbar_arrive_expect_tx(&tma_full[s], kTileBytes + C::kTokBytes);
-          bulk_load(s_packed + s * kTileBytes, wtiles + static_cast<int64_t>(i) * kTileBytes, kTileBytes,
-                    &tma_full[s]);
-          tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, (kb0 + i) * kBlockK, m0, &tma_full[s]);
-          issued = i + 1;
+      int s = 0, issued = 0;
+      uint32_t ph = 0;
+      for (int i = 0; i < nkb; ++i) {
+        if (!mbar_wait(&p_empty[s], ph ^ 1, s_abort)) {
+          raise_error(p, s_abort, kErrProducer);
+          break;
+        }
+        mbar_arrive_expect_tx(&p_full[s], kTileBytes);
+        bulk_load(s_packed + s * kTileBytes, wtiles + static_cast<int64_t>(i) * kTileBytes, kTileBytes, &p_full[s]);
+        issued = i + 1;
+        if (++s == C::NP) {
+          s = 0;
+          ph ^= 1;
         }
       }
       // never leave with copies still in flight: wait (bounded) for the last phase issued per stage
-      for (int i = max(0, issued - C::NS); i < issued; ++i) {
-        const int s = i % C::NS;
+      for (int i = max(0, issued - C::NP); i < issued; ++i) {
         uint32_t spin = 0;
-        while (!mbar_try_wait(&tma_full[s], (i / C::NS) & 1) && ++spin < kSpinLimit) {
+        while (!mbar_try_wait(&p_full[i % C::NP], (i / C::NP) & 1) && ++spin < kSpinLimit) {
+        }
+      }
+    }
+  } else if (warp == C::kTokenWarp) {
+    // ------------------------------------------------------------------ token producer
+    if (lane == 0 && ok_start) {
+      int s = 0, issued = 0;
+      uint32_t ph = 0;
+      for (int i = 0; i < nkb; ++i) {
+        if (!mbar_wait(&t_empty[s], ph ^ 1, s_abort)) {
+          raise_error(p, s_abort, kErrProducer);
+          break;
+        }
+        mbar_arrive_expect_tx(&t_full[s], C::kTokBytes);
+        tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, (kb0 + i) * kBlockK, m0, &t_full[s]);
+        issued = i + 1;
+        if (++s == C::NT) {
+          s = 0;
+          ph ^= 1;
+        }
+      }
+      for (int i = max(0, issued - C::NT); i < issued; ++i) {
+        uint32_t spin = 0;
+        while (!mbar_try_wait(&t_full[i % C::NT], (i / C::NT) & 1) && ++spin < kSpinLimit) {
         }
       }
     }
@@ -248,47 +284,50 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && ok_start) {
       const uint32_t idesc = umma_idesc_e4m3(BM);
+      const uint64_t bdesc0 = umma_desc_k128(smem_u32(s_tok));
       const int mpg = p.group / 32;  // MMAs per weight group (mode none)
       int mma_count = 0;
+      int st = 0, sa = 0;
+      uint32_t pht = 0, pha = 0;
       bool failed = false;
-      const uint64_t bdesc0 = umma_desc_k128(smem_u32(s_tok));
-      for (int i0 = 0; i0 < nkb && !failed; i0 += C::NS) {  // one ring round per outer iteration
-        const uint32_t ph = (i0 / C::NS) & 1;
+      for (int i = 0; i < nkb && !failed; ++i) {
+        if (!mbar_wait(&a_full[sa], pha, s_abort) || !mbar_wait(&t_full[st], pht, s_abort)) {
+          failed = true;
+          break;
+        }
+        tc_fence_after_sync();
+        const uint32_t a_addr = tmem_a + sa * kAStageCols;
+        const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((st * C::kTokBytes) >> 4);
 #pragma unroll
-        for (int s = 0; s < C::NS; ++s) {
-          const int i = i0 + s;
-          if (i >= nkb || failed) break;
-          // the widen warps saw the stage's copies land before they arrived here, so this one wait also
-          // orders the token tile (same barrier as the packed tile) before the MMAs that read it
-          if (!mbar_wait(&a_full[s], ph, s_abort)) {
-            failed = true;
-            break;
-          }
-          tc_fence_after_sync();
-          const uint32_t a_addr = tmem_a + s * kAStageCols;
-          const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((s * C::kTokBytes) >> 4);
-#pragma unroll
-          for (int k = 0; k < kBlockK / 32; ++k) {
-            uint32_t d_tmem = tmem_base;
-            uint32_t accumulate = (i > 0 || k > 0) ? 1u : 0u;
-            if (NONE) {
-              const int grp = mma_count / mpg, within = mma_count % mpg, b = grp & 1;
-              if (within == 0) {
-                if (!mbar_wait(&acc_empty[b], ((grp >> 1) & 1) ^ 1, s_abort)) {
-                  failed = true;
-                  break;
-                }
-                tc_fence_after_sync();
+        for (int k = 0; k < kBlockK / 32; ++k) {
+          uint32_t d_tmem = tmem_base;
+          uint32_t accumulate = (i > 0 || k > 0) ? 1u : 0u;
+          if (NONE) {
+            const int grp = mma_count / mpg, within = mma_count % mpg, b = grp & 1;
+            if (within == 0) {
+              if (!mbar_wait(&acc_empty[b], ((grp >> 1) & 1) ^ 1, s_abort)) {
+                failed = true;
+                break;
               }
-              d_tmem = tmem_base + b * BM;
-              accumulate = within > 0 ? 1u : 0u;
+              tc_fence_after_sync();
             }
-            umma_f8_tmem_a(d_tmem, a_addr + 8 * k, bdesc + 2 * k, idesc, accumulate);
-            ++mma_count;
-            if (NONE && (mma_count % mpg) == 0) umma_commit(&acc_full[((mma_count / mpg) - 1) & 1]);
+            d_tmem = tmem_base + b * BM;
+            accumulate = within > 0 ? 1u : 0u;
           }
-          if (failed) break;
-          umma_commit(&empty[s]);
+          umma_f8_tmem_a(d_tmem, a_addr + 8 * k, bdesc + 2 * k, idesc, accumulate);
+          ++mma_count;
+          if (NONE && (mma_count % mpg) == 0) umma_commit(&acc_full[((mma_count / mpg) - 1) & 1]);
+        }
+        if (failed) break;
+        umma_commit(&t_empty[st]);
+        umma_commit(&a_empty[sa]);
+        if (++st == C::NT) {
+          st = 0;
+          pht ^= 1;
+        }
+        if (++sa == C::NA) {
+          sa = 0;
+          pha ^= 1;
         }
       }
       if (failed) {
@@ -313,22 +352,16 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     if (warp < C::kWidenWarps && !failed) {
       // A lane widens whole rows: 64 packed bytes -> 128 E4M3 bytes = 32 TMEM columns of its own lane.
       const int grp = warp >> 2;
-      for (int i0 = 0; i0 < nkb && !failed; i0 += C::NS)  // one ring round per outer iteration
-#pragma unroll
-      for (int ss = 0; ss < C::NS / C::NG; ++ss) {
-        // stage s is always this group's (NS % NG == 0), so the group sees every round of the stage's
-        // barrier and the parity below is unambiguous; tma_full(i) implies empty(i - NS): the producer
-        // refilled the stage only after that MMA was done, so the TMEM stage is free as well
-        const int s = grp + ss * C::NG;
-        const int i = i0 + s;
-        if (i >= nkb || failed) break;
-        if (!mbar_wait_warp(&tma_full[s], (i0 / C::NS) & 1, s_abort)) {
+      int sp = grp, sa = grp;  // this group's stages: grp, grp + NG, ... (NP and NA are multiples of NG)
+      uint32_t php = 0, pha = 0;
+      for (int i = grp; i < nkb; i += C::NG) {
+        if (!mbar_wait_warp(&p_full[sp], php, s_abort) || !mbar_wait_warp(&a_empty[sa], pha ^ 1, s_abort)) {
           raise_error(p, s_abort, kErrWiden);
           failed = true;
           break;
         }
         tc_fence_after_sync();
-        const uint8_t* tile = s_packed + s * kTileBytes;
+        const uint8_t* tile = s_packed + sp * kTileBytes;
         uint4 pk[4];
 #pragma unroll
         for (int c = 0; c < 4; ++c) pk[c] = *reinterpret_cast<const uint4*>(tile + (c * kTileRows + row) * 16);
@@ -350,13 +383,26 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
             widen8(v.w, lut_lo, lut_hi, o[6], o[7]);
           }
         }
-        const uint32_t dst = tmem_a + s * kAStageCols + lane_base;
+        // every lane's loads of the packed tile have been consumed: hand the stage back
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_empty[sp]);
+        const uint32_t dst = tmem_a + sa * kAStageCols + lane_base;
         tmem_st16(dst, w);
         tmem_st16(dst + 16, w + 16);
         tmem_st_wait();
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&a_full[s]);
+        if (lane == 0) mbar_arrive(&a_full[sa]);
+        sp += C::NG;
+        if (sp >= C::NP) {
+          sp -= C::NP;
+          php ^= 1;
+        }
+        sa += C::NG;
+        if (sa >= C::NA) {
+          sa -= C::NA;
+          pha ^= 1;
+        }
       }
     }
 
