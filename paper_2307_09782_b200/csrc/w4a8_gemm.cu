@@ -282,7 +282,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     }
   } else if (warp == C::kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0 && ok_start) {
+    // The whole warp runs the loop (uniform control flow and addresses); one elected lane issues.
+    if (ok_start) {
+      const bool issuer = elect_one();
       const uint32_t idesc = umma_idesc_e4m3(BM);
       const uint64_t bdesc0 = umma_desc_k128(smem_u32(s_tok));
       const int mpg = p.group / 32;  // MMAs per weight group (mode none)
@@ -290,12 +292,20 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       int st = 0, sa = 0;
       uint32_t pht = 0, pha = 0;
       bool failed = false;
+      // A barrier test takes a few hundred cycles to answer even when the phase is long complete, so the
+      // test for the next K block is issued before this block's MMAs and only read afterwards.
+      bool ready = mbar_try_wait(&a_full[0], 0) && mbar_try_wait(&t_full[0], 0);
       for (int i = 0; i < nkb && !failed; ++i) {
-        if (!mbar_wait(&a_full[sa], pha, s_abort) || !mbar_wait(&t_full[st], pht, s_abort)) {
+        if (!ready && (!mbar_wait(&a_full[sa], pha, s_abort) || !mbar_wait(&t_full[st], pht, s_abort))) {
           failed = true;
           break;
         }
         tc_fence_after_sync();
+        {
+          const int sa_n = (sa + 1 == C::NA) ? 0 : sa + 1, st_n = (st + 1 == C::NT) ? 0 : st + 1;
+          const uint32_t pha_n = (sa + 1 == C::NA) ? pha ^ 1 : pha, pht_n = (st + 1 == C::NT) ? pht ^ 1 : pht;
+          ready = (i + 1 < nkb) && mbar_try_wait(&a_full[sa_n], pha_n) && mbar_try_wait(&t_full[st_n], pht_n);
+        }
         const uint32_t a_addr = tmem_a + sa * kAStageCols;
         const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((st * C::kTokBytes) >> 4);
 #pragma unroll
@@ -314,13 +324,16 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
             d_tmem = tmem_base + b * BM;
             accumulate = within > 0 ? 1u : 0u;
           }
-          umma_f8_tmem_a(d_tmem, a_addr + 8 * k, bdesc + 2 * k, idesc, accumulate);
+          if (issuer) umma_f8_tmem_a(d_tmem, a_addr + 8 * k, bdesc + 2 * k, idesc, accumulate);
           ++mma_count;
-          if (NONE && (mma_count % mpg) == 0) umma_commit(&acc_full[((mma_count / mpg) - 1) & 1]);
+          if (NONE && (mma_count % mpg) == 0 && issuer) umma_commit(&acc_full[((mma_count / mpg) - 1) & 1]);
         }
         if (failed) break;
-        umma_commit(&t_empty[st]);
-        umma_commit(&a_empty[sa]);
+        if (issuer) {
+          umma_commit(&t_empty[st]);
+          umma_commit(&a_empty[sa]);
+        }
+        __syncwarp();
         if (++st == C::NT) {
           st = 0;
           pht ^= 1;
@@ -331,14 +344,17 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
         }
       }
       if (failed) {
-        raise_error(p, s_abort, kErrMma);
-        umma_commit(drain_bar);  // let the MMAs already issued finish before TMEM is released
+        if (issuer) {
+          raise_error(p, s_abort, kErrMma);
+          umma_commit(drain_bar);  // let the MMAs already issued finish before TMEM is released
+        }
         uint32_t spin = 0;
         while (!mbar_try_wait(drain_bar, 0) && ++spin < kSpinLimit) {
         }
       } else if (!NONE) {
-        umma_commit(&acc_full[0]);
+        if (issuer) umma_commit(&acc_full[0]);
       }
+      __syncwarp();
     }
   } else {
     // ------------------------------------------------------------------ widen / promote / epilogue
