@@ -232,17 +232,21 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
 
   if (warp == C::kWeightWarp) {
     // ------------------------------------------------------------------ packed-weight producer
-    if (lane == 0 && ok_start) {
+    if (ok_start) {  // warp-uniform loop, one elected lane issues the copies
+      const bool issuer = elect_one();
       const uint8_t* wtiles = p.codes + (static_cast<int64_t>(blockIdx.x) * p.kblocks + kb0) * kTileBytes;
       int s = 0, issued = 0;
       uint32_t ph = 0;
       for (int i = 0; i < nkb; ++i) {
         if (!mbar_wait(&p_empty[s], ph ^ 1, s_abort)) {
-          raise_error(p, s_abort, kErrProducer);
+          if (issuer) raise_error(p, s_abort, kErrProducer);
           break;
         }
-        mbar_arrive_expect_tx(&p_full[s], kTileBytes);
-        bulk_load(s_packed + s * kTileBytes, wtiles + static_cast<int64_t>(i) * kTileBytes, kTileBytes, &p_full[s]);
+        if (issuer) {
+          mbar_arrive_expect_tx(&p_full[s], kTileBytes);
+          bulk_load(s_packed + s * kTileBytes, wtiles + static_cast<int64_t>(i) * kTileBytes, kTileBytes, &p_full[s]);
+        }
+        __syncwarp();
         issued = i + 1;
         if (++s == C::NP) {
           s = 0;
@@ -258,16 +262,20 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     }
   } else if (warp == C::kTokenWarp) {
     // ------------------------------------------------------------------ token producer
-    if (lane == 0 && ok_start) {
+    if (ok_start) {  // warp-uniform loop, one elected lane issues the copies
+      const bool issuer = elect_one();
       int s = 0, issued = 0;
       uint32_t ph = 0;
       for (int i = 0; i < nkb; ++i) {
         if (!mbar_wait(&t_empty[s], ph ^ 1, s_abort)) {
-          raise_error(p, s_abort, kErrProducer);
+          if (issuer) raise_error(p, s_abort, kErrProducer);
           break;
         }
-        mbar_arrive_expect_tx(&t_full[s], C::kTokBytes);
-        tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, (kb0 + i) * kBlockK, m0, &t_full[s]);
+        if (issuer) {
+          mbar_arrive_expect_tx(&t_full[s], C::kTokBytes);
+          tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, (kb0 + i) * kBlockK, m0, &t_full[s]);
+        }
+        __syncwarp();
         issued = i + 1;
         if (++s == C::NT) {
           s = 0;
