@@ -167,7 +167,7 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
   const size_t need = x_bf16 ? w.total : w.off_q;
   if (workspace_bytes < need) return ZQ_ERR_WORKSPACE;
   const GemmPlan pl = plan_gemm(M, N, K, mode);
-  if (pl.m_tiles > 65535 || pl.splits > 65535) return ZQ_ERR_SHAPE;
+  if (pl.ctas <= 0) return ZQ_ERR_SHAPE;
   if (int e = check_device_sm100()) return e;
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);

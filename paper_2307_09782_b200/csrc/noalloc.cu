@@ -69,7 +69,7 @@ int zq_w4a8_linear_noalloc(const uint8_t* q, const float* sx, int64_t M, int64_t
     return ZQ_ERR_ALIGN;
   // the fixed scratch bounds the split-K partial sums this problem may need
   const GemmPlan pl = plan_gemm(M, N, K, mode);
-  if (pl.partial_floats > kScratchPartialFloats || pl.m_tiles > 65535) return ZQ_ERR_WORKSPACE;
+  if (pl.partial_floats > kScratchPartialFloats || pl.ctas <= 0) return ZQ_ERR_WORKSPACE;
 
   void* scratch = nullptr;
   if (int e = scratch_address(&scratch)) return e;

@@ -53,9 +53,15 @@ struct Params {
   int M, N, K;
   int G;             // groups per row
   int group;
-  int kb_per_split;  // K blocks handled by one CTA
-  int kblocks;       // total K blocks
-  int splits;
+  int kblocks;       // K blocks per output tile
+  int n_tiles, tiles;  // output tiles along N, and in total (tile index = m_tile * n_tiles + n_tile)
+  // Work is counted in units of one K block of one output tile, unit u = tile * kblocks + kb.  A CTA
+  // owns the contiguous units [u0, u1) and walks them as segments (one per output tile it touches):
+  //   stream == 0: CTA c = z * tiles + tile owns K blocks [z * kb_per_split, ...) of that tile
+  //   stream == 1: the units of all tiles are dealt out evenly, base (+1 for the first rem CTAs) each
+  int stream;
+  int splits, kb_per_split;
+  int base, rem;
   const uint8_t* codes;  // tiled weight
   const float* scale;
   const float* sx;
@@ -128,6 +134,29 @@ __device__ __forceinline__ void raise_error(const Params& p, volatile int* abort
   if (atomicCAS(p.status, 0, ZQ_ERR_DEVICE_TIMEOUT) == 0) p.status[1] = detail;
 }
 
+__device__ __forceinline__ int range_start(const Params& p, int c) { return c * p.base + min(c, p.rem); }
+__device__ __forceinline__ int cta_of_unit(const Params& p, int u) {
+  const int big = p.rem * (p.base + 1);
+  return u < big ? u / (p.base + 1) : p.rem + (u - big) / p.base;
+}
+// The CTAs that contribute partial sums to `tile`: first CTA and their number.
+__device__ __forceinline__ void contributors(const Params& p, int tile, int* first, int* count) {
+  if (p.stream) {
+    *first = cta_of_unit(p, tile * p.kblocks);
+    *count = cta_of_unit(p, tile * p.kblocks + p.kblocks - 1) - *first + 1;
+  } else {
+    *first = 0;
+    *count = p.splits;
+  }
+}
+// Workspace slot of the partial sum that contributor j (CTA first + j) leaves for `tile`.  A streaming
+// CTA can leave two (for the tile its range starts in and for the one it ends in).
+__device__ __forceinline__ size_t partial_slot(const Params& p, int tile, int first, int j) {
+  if (!p.stream) return static_cast<size_t>(tile) * p.splits + j;
+  const int c = first + j;
+  return 2 * static_cast<size_t>(c) + (range_start(p, c) / p.kblocks == tile ? 0 : 1);
+}
+
 // Final arithmetic of 16 consecutive tokens (tile columns c0 .. c0+15) of one output channel, and the store.
 //   y[m, n] = sx[m] * cs * acc + sum_j t[m, j] * U[n, j]
 // s_sx / s_t are the tile's token scales and rank-8 LoRC rows in shared memory; u8 holds the channel's
@@ -187,9 +216,19 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   float* s_t = reinterpret_cast<float*>(smem + C::offT);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * BM;
-  const int kb0 = blockIdx.z * p.kb_per_split;
-  const int nkb = min(p.kb_per_split, p.kblocks - kb0);
+  // this CTA's units [u0, u1)
+  int u0, u1;
+  if (p.stream) {
+    u0 = range_start(p, blockIdx.x);
+    u1 = range_start(p, blockIdx.x + 1);
+  } else {
+    const int z = blockIdx.x / p.tiles, tile = blockIdx.x % p.tiles;
+    u0 = tile * p.kblocks + z * p.kb_per_split;
+    u1 = min(u0 + p.kb_per_split, (tile + 1) * p.kblocks);
+  }
+  const int nunits = u1 - u0;
+  // all of a CTA's tiles share one token tile (streaming is only used with a single row of tiles)
+  const int m0 = ((u0 / p.kblocks) / p.n_tiles) * BM;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < C::NP; ++i) {
@@ -206,7 +245,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     }
     mbar_init(&acc_full[0], 1);
     mbar_init(&acc_full[1], 1);
-    mbar_init(&acc_empty[0], 128);
+    // mode none: two buffers, released by the 128 promotion threads; otherwise one accumulator,
+    // handed back once per segment by the widen warps (one arrival per warp)
+    mbar_init(&acc_empty[0], NONE ? 128 : C::kWidenWarps);
     mbar_init(&acc_empty[1], 128);
     mbar_init(drain_bar, 1);
     *s_abort = 0;
@@ -216,7 +257,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
   }
   if (warp == C::kTokenWarp && lane == 0) prefetch_tensormap(&tm_q);
   if (warp < C::kWidenWarps) {
-    // token scales and (rank 8) LoRC rows of this tile's tokens, for the epilogue
+    // token scales and (rank 8) LoRC rows of this CTA's tokens, for the epilogue
     for (int c = threadIdx.x; c < BM; c += 32 * C::kWidenWarps) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
     if (p.r == 8)
       for (int c = threadIdx.x; c < BM * 8; c += 32 * C::kWidenWarps)
@@ -234,20 +275,26 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     // ------------------------------------------------------------------ packed-weight producer
     if (ok_start) {  // warp-uniform loop, one elected lane issues the copies
       const bool issuer = elect_one();
-      const uint8_t* wtiles = p.codes + (static_cast<int64_t>(blockIdx.x) * p.kblocks + kb0) * kTileBytes;
       int s = 0, issued = 0;
       uint32_t ph = 0;
-      for (int i = 0; i < nkb; ++i) {
+      int tile = u0 / p.kblocks, kb = u0 % p.kblocks;
+      for (int i = 0; i < nunits; ++i) {
         if (!mbar_wait(&p_empty[s], ph ^ 1, s_abort)) {
           if (issuer) raise_error(p, s_abort, kErrProducer);
           break;
         }
         if (issuer) {
+          const uint8_t* src =
+              p.codes + (static_cast<int64_t>(tile % p.n_tiles) * p.kblocks + kb) * kTileBytes;
           mbar_arrive_expect_tx(&p_full[s], kTileBytes);
-          bulk_load(s_packed + s * kTileBytes, wtiles + static_cast<int64_t>(i) * kTileBytes, kTileBytes, &p_full[s]);
+          bulk_load(s_packed + s * kTileBytes, src, kTileBytes, &p_full[s]);
         }
         __syncwarp();
         issued = i + 1;
+        if (++kb == p.kblocks) {
+          kb = 0;
+          ++tile;
+        }
         if (++s == C::NP) {
           s = 0;
           ph ^= 1;
@@ -266,17 +313,19 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       const bool issuer = elect_one();
       int s = 0, issued = 0;
       uint32_t ph = 0;
-      for (int i = 0; i < nkb; ++i) {
+      int kb = u0 % p.kblocks;
+      for (int i = 0; i < nunits; ++i) {
         if (!mbar_wait(&t_empty[s], ph ^ 1, s_abort)) {
           if (issuer) raise_error(p, s_abort, kErrProducer);
           break;
         }
         if (issuer) {
           mbar_arrive_expect_tx(&t_full[s], C::kTokBytes);
-          tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, (kb0 + i) * kBlockK, m0, &t_full[s]);
+          tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, kb * kBlockK, m0, &t_full[s]);
         }
         __syncwarp();
         issued = i + 1;
+        if (++kb == p.kblocks) kb = 0;
         if (++s == C::NT) {
           s = 0;
           ph ^= 1;
@@ -299,27 +348,28 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       int mma_count = 0;
       int st = 0, sa = 0;
       uint32_t pht = 0, pha = 0;
+      int kb = u0 % p.kblocks, seg = 0;
+      bool seg_first = true;  // the next K block starts a segment (a new accumulation)
       bool failed = false;
-      // A barrier test takes a few hundred cycles to answer even when the phase is long complete, so the
-      // test for the next K block is issued before this block's MMAs and only read afterwards.
-      bool ready = mbar_try_wait(&a_full[0], 0) && mbar_try_wait(&t_full[0], 0);
-      for (int i = 0; i < nkb && !failed; ++i) {
-        if (!ready && (!mbar_wait(&a_full[sa], pha, s_abort) || !mbar_wait(&t_full[st], pht, s_abort))) {
+      for (int i = 0; i < nunits && !failed; ++i) {
+        if (!mbar_wait(&a_full[sa], pha, s_abort) || !mbar_wait(&t_full[st], pht, s_abort)) {
           failed = true;
           break;
         }
-        tc_fence_after_sync();
-        {
-          const int sa_n = (sa + 1 == C::NA) ? 0 : sa + 1, st_n = (st + 1 == C::NT) ? 0 : st + 1;
-          const uint32_t pha_n = (sa + 1 == C::NA) ? pha ^ 1 : pha, pht_n = (st + 1 == C::NT) ? pht ^ 1 : pht;
-          ready = (i + 1 < nkb) && mbar_try_wait(&a_full[sa_n], pha_n) && mbar_try_wait(&t_full[st_n], pht_n);
+        if (!NONE && seg_first && seg > 0) {
+          // the epilogue of the previous segment must have read the accumulator
+          if (!mbar_wait(&acc_empty[0], (seg - 1) & 1, s_abort)) {
+            failed = true;
+            break;
+          }
         }
+        tc_fence_after_sync();
         const uint32_t a_addr = tmem_a + sa * kAStageCols;
         const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((st * C::kTokBytes) >> 4);
 #pragma unroll
         for (int k = 0; k < kBlockK / 32; ++k) {
           uint32_t d_tmem = tmem_base;
-          uint32_t accumulate = (i > 0 || k > 0) ? 1u : 0u;
+          uint32_t accumulate = (!seg_first || k > 0) ? 1u : 0u;
           if (NONE) {
             const int grp = mma_count / mpg, within = mma_count % mpg, b = grp & 1;
             if (within == 0) {
@@ -337,11 +387,16 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
           if (NONE && (mma_count % mpg) == 0 && issuer) umma_commit(&acc_full[((mma_count / mpg) - 1) & 1]);
         }
         if (failed) break;
+        const bool seg_last = (kb + 1 == p.kblocks) || (i + 1 == nunits);
         if (issuer) {
           umma_commit(&t_empty[st]);
           umma_commit(&a_empty[sa]);
+          if (!NONE && seg_last) umma_commit(&acc_full[seg & 1]);
         }
         __syncwarp();
+        seg_first = seg_last;
+        if (seg_last) ++seg;
+        if (++kb == p.kblocks) kb = 0;
         if (++st == C::NT) {
           st = 0;
           pht ^= 1;
@@ -359,8 +414,6 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
         uint32_t spin = 0;
         while (!mbar_try_wait(drain_bar, 0) && ++spin < kSpinLimit) {
         }
-      } else if (!NONE) {
-        if (issuer) umma_commit(&acc_full[0]);
       }
       __syncwarp();
     }
@@ -368,197 +421,221 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     // ------------------------------------------------------------------ widen / promote / epilogue
     const int q4 = warp & 3;         // TMEM lane quarter of this warp
     const int row = q4 * 32 + lane;  // output channel within the tile = TMEM lane
-    const int n = n0 + row;
-    const bool n_ok = n < p.N;
     const uint32_t lane_base = static_cast<uint32_t>(q4 * 32) << 16;
+    const bool widen_role = warp < C::kWidenWarps;
+    const bool epi_role = NONE ? (warp >= C::kPromoteWarp0) : true;
+    const int grp = warp >> 2;  // widen group (widen warps only)
     bool failed = !ok_start;
 
-    if (warp < C::kWidenWarps && !failed) {
-      // A lane widens whole rows: 64 packed bytes -> 128 E4M3 bytes = 32 TMEM columns of its own lane.
-      const int grp = warp >> 2;
-      int sp = grp, sa = grp;  // this group's stages: grp, grp + NG, ... (NP and NA are multiples of NG)
-      uint32_t php = 0, pha = 0;
-      for (int i = grp; i < nkb; i += C::NG) {
-        if (!mbar_wait_warp(&p_full[sp], php, s_abort) || !mbar_wait_warp(&a_empty[sa], pha ^ 1, s_abort)) {
-          raise_error(p, s_abort, kErrWiden);
-          failed = true;
-          break;
-        }
-        tc_fence_after_sync();
-        const uint8_t* tile = s_packed + sp * kTileBytes;
-        uint4 pk[4];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) pk[c] = *reinterpret_cast<const uint4*>(tile + (c * kTileRows + row) * 16);
-        // the tile carries its shift bytes (zero in mode none): one per row and 64-element half
-        const uint32_t d2 = NONE ? 0u : *reinterpret_cast<const uint16_t*>(tile + kTileCodeBytes + 2 * row);
-        uint32_t w[32];
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          const uint32_t d = (d2 >> (8 * h)) & 0xFFu;
-          const uint32_t lut_lo = 0x3C383000u - d * 0x08080800u;
-          const uint32_t lut_hi = 0x4C484440u - d * 0x08080808u;
-#pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            const uint4 v = pk[2 * h + c];
-            uint32_t* o = w + (2 * h + c) * 8;
-            widen8(v.x, lut_lo, lut_hi, o[0], o[1]);
-            widen8(v.y, lut_lo, lut_hi, o[2], o[3]);
-            widen8(v.z, lut_lo, lut_hi, o[4], o[5]);
-            widen8(v.w, lut_lo, lut_hi, o[6], o[7]);
-          }
-        }
-        // every lane's loads of the packed tile have been consumed: hand the stage back
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&p_empty[sp]);
-        const uint32_t dst = tmem_a + sa * kAStageCols + lane_base;
-        tmem_st16(dst, w);
-        tmem_st16(dst + 16, w + 16);
-        tmem_st_wait();
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&a_full[sa]);
-        sp += C::NG;
-        if (sp >= C::NP) {
-          sp -= C::NP;
-          php ^= 1;
-        }
-        sa += C::NG;
-        if (sa >= C::NA) {
-          sa -= C::NA;
-          pha ^= 1;
-        }
-      }
-    }
+    // ring positions of this widen group: stages grp, grp + NG, ... (NP and NA are multiples of NG)
+    int wi = grp, sp = grp, sa = grp;
+    uint32_t php = 0, pha = 0;
 
-    // ---- accumulators -> registers -> y
-    const bool epi_role = NONE ? (warp >= C::kPromoteWarp0) : true;
-    if (epi_role) {
-      const int part = NONE ? 0 : (warp >> 2);  // which share of the columns this widen group finishes
-      constexpr int kMyCols = NONE ? BM : (BM / C::NG >= 16 ? BM / C::NG : 16);
-      // Mode none keeps its running sums in a register array, which needs the column loop unrolled; the
-      // other modes keep the loop rolled so that its body stays resident in the instruction cache.
-      constexpr int kEpiUnroll = NONE ? kMyCols / 16 : 1;
-      const int col0 = NONE ? 0 : part * kMyCols;
-      const bool has_cols = NONE ? true : (col0 < BM);
-      const uint32_t t_lane = tmem_base + lane_base;
-      const int tile_id = blockIdx.y * gridDim.x + blockIdx.x;
-      float* my_partial = p.partials + (static_cast<size_t>(tile_id) * p.splits + blockIdx.z) * (BM * kTileN);
+    const int part = NONE ? 0 : grp;  // which share of the columns this widen group finishes
+    constexpr int kMyCols = NONE ? BM : (BM / C::NG >= 16 ? BM / C::NG : 16);
+    // Mode none keeps its running sums in a register array, which needs the column loop unrolled; the
+    // other modes keep the loop rolled so that its body stays resident in the instruction cache.
+    constexpr int kEpiUnroll = NONE ? kMyCols / 16 : 1;
+    const int col0 = NONE ? 0 : part * kMyCols;
+    const bool has_cols = NONE ? true : (col0 < BM);
+    const uint32_t t_lane = tmem_base + lane_base;
 
-      float cs = 1.0f;
-      float u[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) u[e] = 0.0f;
-      if (!NONE && n_ok) cs = __ldg(p.scale + n);
-      if (p.r == 8 && n_ok) {
-        const uint4 h = __ldg(reinterpret_cast<const uint4*>(p.U + static_cast<int64_t>(n) * 8));
-        const uint32_t hw[4] = {h.x, h.y, h.z, h.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          __half2 h2;
-          *reinterpret_cast<uint32_t*>(&h2) = hw[e];
-          const float2 f = __half22float2(h2);
-          u[2 * e] = f.x;
-          u[2 * e + 1] = f.y;
-        }
-      }
+    // Every thread walks every segment and executes the same named-barrier sequence whether or not it
+    // has failed, so a bounded wait that ran out can never leave others stuck at a hardware barrier.
+    int seg = 0;
+    for (int us = u0; us < u1; ++seg) {
+      const int tile = us / p.kblocks;
+      const int ue = min(u1, (tile + 1) * p.kblocks);
+      const int n0 = (tile % p.n_tiles) * kTileN;
+      const int n = n0 + row;
+      const bool n_ok = n < p.N;
 
-      float run[NONE ? BM : 1];
-      if (NONE) {
-        // per-group promotion: run += S[n, g] * (this group's FP32 partial sum)
-#pragma unroll
-        for (int c = 0; c < BM; ++c) run[c] = 0.0f;
-        const int groups = (nkb * kBlockK) / p.group;
-        const int g0 = (kb0 * kBlockK) / p.group;
-        const float* srow = n_ok ? p.scale + static_cast<int64_t>(n) * p.G : nullptr;
-        float S_next = (srow && groups > 0) ? __ldg(srow + g0) : 0.0f;
-        for (int g = 0; g < groups && !failed; ++g) {
-          const int b = g & 1;
-          const float S = S_next;
-          if (srow && g + 1 < groups) S_next = __ldg(srow + g0 + g + 1);
-          if (!mbar_wait_warp(&acc_full[b], (g >> 1) & 1, s_abort)) {
-            raise_error(p, s_abort, kErrPromote);
+      if (widen_role) {
+        // A lane widens whole rows: 64 packed bytes -> 128 E4M3 bytes = 32 TMEM columns of its own lane.
+        for (; wi < ue - u0 && !failed; wi += C::NG) {
+          if (!mbar_wait_warp(&p_full[sp], php, s_abort) || !mbar_wait_warp(&a_empty[sa], pha ^ 1, s_abort)) {
+            raise_error(p, s_abort, kErrWiden);
             failed = true;
             break;
           }
           tc_fence_after_sync();
+          const uint8_t* tile_s = s_packed + sp * kTileBytes;
+          uint4 pk[4];
 #pragma unroll
-          for (int c = 0; c < BM; c += 16) {
-            float v[16];
-            tmem_ld16(t_lane + b * BM + c, v);
-            tmem_ld_wait();
+          for (int c = 0; c < 4; ++c) pk[c] = *reinterpret_cast<const uint4*>(tile_s + (c * kTileRows + row) * 16);
+          // the tile carries its shift bytes (zero in mode none): one per row and 64-element half
+          const uint32_t d2 = NONE ? 0u : *reinterpret_cast<const uint16_t*>(tile_s + kTileCodeBytes + 2 * row);
+          uint32_t w[32];
 #pragma unroll
-            for (int e = 0; e < 16; ++e) run[c + e] = fmaf(S, v[e], run[c + e]);
+          for (int h = 0; h < 2; ++h) {
+            const uint32_t d = (d2 >> (8 * h)) & 0xFFu;
+            const uint32_t lut_lo = 0x3C383000u - d * 0x08080800u;
+            const uint32_t lut_hi = 0x4C484440u - d * 0x08080808u;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              const uint4 v = pk[2 * h + c];
+              uint32_t* o = w + (2 * h + c) * 8;
+              widen8(v.x, lut_lo, lut_hi, o[0], o[1]);
+              widen8(v.y, lut_lo, lut_hi, o[2], o[3]);
+              widen8(v.z, lut_lo, lut_hi, o[4], o[5]);
+              widen8(v.w, lut_lo, lut_hi, o[6], o[7]);
+            }
           }
+          // every lane's loads of the packed tile have been consumed: hand the stage back
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&p_empty[sp]);
+          const uint32_t dst = tmem_a + sa * kAStageCols + lane_base;
+          tmem_st16(dst, w);
+          tmem_st16(dst + 16, w + 16);
+          tmem_st_wait();
           tc_fence_before_sync();
-          mbar_arrive(&acc_empty[b]);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&a_full[sa]);
+          sp += C::NG;
+          if (sp >= C::NP) {
+            sp -= C::NP;
+            php ^= 1;
+          }
+          sa += C::NG;
+          if (sa >= C::NA) {
+            sa -= C::NA;
+            pha ^= 1;
+          }
         }
-      } else if (!failed) {
-        if (!mbar_wait_warp(&acc_full[0], 0, s_abort)) {
-          raise_error(p, s_abort, kErrEpilogue);
-          failed = true;
-        }
-        tc_fence_after_sync();
       }
 
-      if (p.splits == 1) {
-        if (!failed && has_cols) {
-#pragma unroll(kEpiUnroll)
-          for (int c = 0; c < kMyCols; c += 16) {
-            float v[16];
-            if (NONE) {
+      // ---- accumulators -> registers -> y (or -> workspace, when other CTAs share the tile)
+      if (epi_role) {
+        float cs = 1.0f;
+        float u[8];
 #pragma unroll
-              for (int e = 0; e < 16; ++e) v[e] = run[c + e];
-            } else {
-              tmem_ld16(t_lane + col0 + c, v);
-              tmem_ld_wait();
-            }
-            if (n_ok) finalize16(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+        for (int e = 0; e < 8; ++e) u[e] = 0.0f;
+        if (!NONE && n_ok) cs = __ldg(p.scale + n);
+        if (p.r == 8 && n_ok) {
+          const uint4 h = __ldg(reinterpret_cast<const uint4*>(p.U + static_cast<int64_t>(n) * 8));
+          const uint32_t hw[4] = {h.x, h.y, h.z, h.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            __half2 h2;
+            *reinterpret_cast<uint32_t*>(&h2) = hw[e];
+            const float2 f = __half22float2(h2);
+            u[2 * e] = f.x;
+            u[2 * e + 1] = f.y;
           }
         }
-      } else {
-        // split-K: leave the raw partial sums in the workspace; the CTA that arrives last for this
-        // output tile adds all of them in split order (deterministic) and finishes the tile.
-        if (!failed && has_cols) {
-#pragma unroll(kEpiUnroll)
-          for (int c = 0; c < kMyCols; c += 16) {
-            float v[16];
-            if (NONE) {
+
+        float run[NONE ? BM : 1];
+        if (NONE) {
+          // per-group promotion: run += S[n, g] * (this group's FP32 partial sum)
 #pragma unroll
-              for (int e = 0; e < 16; ++e) v[e] = run[c + e];
-            } else {
-              tmem_ld16(t_lane + col0 + c, v);
-              tmem_ld_wait();
+          for (int c = 0; c < BM; ++c) run[c] = 0.0f;
+          const int kb_first = us % p.kblocks;
+          const int groups = ((ue - us) * kBlockK) / p.group;
+          const int g0 = (kb_first * kBlockK) / p.group;
+          const float* srow = n_ok ? p.scale + static_cast<int64_t>(n) * p.G : nullptr;
+          float S_next = (srow && groups > 0) ? __ldg(srow + g0) : 0.0f;
+          for (int g = 0; g < groups && !failed; ++g) {
+            const int b = g & 1;
+            const float S = S_next;
+            if (srow && g + 1 < groups) S_next = __ldg(srow + g0 + g + 1);
+            if (!mbar_wait_warp(&acc_full[b], (g >> 1) & 1, s_abort)) {
+              raise_error(p, s_abort, kErrPromote);
+              failed = true;
+              break;
             }
+            tc_fence_after_sync();
 #pragma unroll
-            for (int e = 0; e < 16; ++e) my_partial[(col0 + c + e) * kTileN + row] = v[e];
+            for (int c = 0; c < BM; c += 16) {
+              float v[16];
+              tmem_ld16(t_lane + b * BM + c, v);
+              tmem_ld_wait();
+#pragma unroll
+              for (int e = 0; e < 16; ++e) run[c + e] = fmaf(S, v[e], run[c + e]);
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&acc_empty[b]);
           }
+        } else if (!failed) {
+          if (!mbar_wait_warp(&acc_full[seg & 1], (seg >> 1) & 1, s_abort)) {
+            raise_error(p, s_abort, kErrEpilogue);
+            failed = true;
+          }
+          tc_fence_after_sync();
         }
-        __threadfence();
-        named_bar_sync(1, C::kEpiThreads);
-        const bool leader = NONE ? (threadIdx.x == 32 * C::kPromoteWarp0) : (threadIdx.x == 0);
-        if (leader) {
-          const int ticket = (*s_abort) ? -1 : atomicAdd(p.counters + tile_id, 1);
-          *s_last = (ticket == p.splits - 1) ? 1 : 0;
-          if (ticket == p.splits - 1) p.counters[tile_id] = 0;  // ready for the next call
-        }
-        named_bar_sync(1, C::kEpiThreads);
-        if (*s_last && has_cols) {
+
+        const bool whole_tile = (ue - us) == p.kblocks;
+        if (whole_tile) {
+          if (!failed && has_cols) {
+#pragma unroll(kEpiUnroll)
+            for (int c = 0; c < kMyCols; c += 16) {
+              float v[16];
+              if (NONE) {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = run[c + e];
+              } else {
+                tmem_ld16(t_lane + col0 + c, v);
+                tmem_ld_wait();
+              }
+              if (n_ok) finalize16(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+            }
+          }
+        } else {
+          // Several CTAs share this tile: leave the raw partial sums in the workspace; the CTA that
+          // arrives last adds all of them in contributor order (deterministic) and finishes the tile.
+          int first, count;
+          contributors(p, tile, &first, &count);
+          const int my_j = p.stream ? static_cast<int>(blockIdx.x) - first : static_cast<int>(blockIdx.x) / p.tiles;
+          float* my_partial = p.partials + partial_slot(p, tile, first, my_j) * (BM * kTileN);
+          if (!failed && has_cols) {
+#pragma unroll(kEpiUnroll)
+            for (int c = 0; c < kMyCols; c += 16) {
+              float v[16];
+              if (NONE) {
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] = run[c + e];
+              } else {
+                tmem_ld16(t_lane + col0 + c, v);
+                tmem_ld_wait();
+              }
+#pragma unroll
+              for (int e = 0; e < 16; ++e) my_partial[(col0 + c + e) * kTileN + row] = v[e];
+            }
+          }
           __threadfence();
-          const float* tile_partials = p.partials + static_cast<size_t>(tile_id) * p.splits * (BM * kTileN);
-#pragma unroll 1
-          for (int c = 0; c < kMyCols; c += 16) {
-            float v[16];
-#pragma unroll
-            for (int e = 0; e < 16; ++e) v[e] = 0.0f;
-            for (int z = 0; z < p.splits; ++z) {
-              const float* src = tile_partials + static_cast<size_t>(z) * (BM * kTileN) + (col0 + c) * kTileN + row;
-#pragma unroll
-              for (int e = 0; e < 16; ++e) v[e] += __ldcg(src + e * kTileN);
-            }
-            if (n_ok) finalize16(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+          named_bar_sync(1, C::kEpiThreads);
+          const bool leader = NONE ? (threadIdx.x == 32 * C::kPromoteWarp0) : (threadIdx.x == 0);
+          if (leader) {
+            const int ticket = (*s_abort) ? -1 : atomicAdd(p.counters + tile, 1);
+            *s_last = (ticket == count - 1) ? 1 : 0;
+            if (ticket == count - 1) p.counters[tile] = 0;  // ready for the next call
           }
+          named_bar_sync(1, C::kEpiThreads);
+          if (*s_last && has_cols) {
+            __threadfence();
+#pragma unroll 1
+            for (int c = 0; c < kMyCols; c += 16) {
+              float v[16];
+#pragma unroll
+              for (int e = 0; e < 16; ++e) v[e] = 0.0f;
+              for (int j = 0; j < count; ++j) {
+                const float* src =
+                    p.partials + partial_slot(p, tile, first, j) * (BM * kTileN) + (col0 + c) * kTileN + row;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) v[e] += __ldcg(src + e * kTileN);
+              }
+              if (n_ok) finalize16(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+            }
+          }
+          named_bar_sync(1, C::kEpiThreads);  // s_last is reused by the next segment
+        }
+        if (!NONE) {
+          // the accumulator has been read: the MMA warp may start the next segment
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&acc_empty[0]);
         }
       }
+      us = ue;
     }
   }
 
@@ -616,13 +693,27 @@ int launch_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStr
                                     C::kSmemBytes);
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
-  dim3 grid(plan.n_tiles, plan.m_tiles, plan.splits);
+  dim3 grid(static_cast<unsigned>(plan.ctas));
   w4a8_gemm_kernel<BM, NONE><<<grid, C::kThreads, C::kSmemBytes, st>>>(tm_q, p);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
 }
 
 }  // namespace
+
+// SMs of the current device (148 when no device can be asked, e.g. for a host-only size query).
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+      n = v;
+    else
+      return 148;
+  }
+  return n;
+}
 
 GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
   GemmPlan pl{};
@@ -634,10 +725,28 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
   pl.n_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
   const int64_t tiles = static_cast<int64_t>(pl.m_tiles) * pl.n_tiles;
   const int kblocks = static_cast<int>(K / kBlockK);
-  // split K until about two CTAs per SM are in flight, keeping at least 4 K blocks per CTA and (for
+  const int ctas_per_sm = (mode == ZQ_SCALE_NONE || bm > 128) ? 1 : 2;
+  const int64_t resident = static_cast<int64_t>(ctas_per_sm) * sm_count();
+  const int64_t units = tiles * kblocks;
+  if (mode != ZQ_SCALE_NONE && pl.m_tiles == 1 && tiles <= kWsMaxTiles && units >= 8 && units < (int64_t(1) << 30)) {
+    // One row of output tiles (decode): the weight streams exactly once, so deal the (tile, K block)
+    // units out evenly to one resident wave of CTAs, at least 4 units each.
+    int64_t g = resident < units / 4 ? resident : units / 4;
+    if (g < 1) g = 1;
+    pl.stream = 1;
+    pl.ctas = static_cast<int>(g);
+    pl.base = static_cast<int>(units / g);
+    pl.rem = static_cast<int>(units % g);
+    pl.splits = 1;
+    pl.kb_per_split = kblocks;
+    // a CTA leaves at most two partial sums (the tile its range starts in and the one it ends in)
+    pl.partial_floats = (g == tiles && pl.rem == 0 && pl.base == kblocks) ? 0 : 2 * static_cast<size_t>(g) * bm * kTileN;
+    return pl;
+  }
+  // split K until about one resident wave of CTAs exists, keeping at least 4 K blocks per CTA and (for
   // 256-wide groups) whole groups per CTA
   int splits = 1;
-  const int64_t target = 2 * 148;
+  const int64_t target = 2 * sm_count();
   if (tiles < target && tiles <= kWsMaxTiles) {
     splits = static_cast<int>((target + tiles - 1) / tiles);
     const int max_splits = kblocks / 4 > 0 ? kblocks / 4 : 1;
@@ -647,8 +756,10 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
   if (kbps % 2) ++kbps;  // whole 256-element groups per split
   if (kbps > kblocks) kbps = kblocks;
   splits = (kblocks + kbps - 1) / kbps;
+  pl.stream = 0;
   pl.splits = splits;
   pl.kb_per_split = kbps;
+  pl.ctas = static_cast<int>(tiles * splits);
   pl.partial_floats = splits > 1 ? static_cast<size_t>(tiles) * splits * bm * kTileN : 0;
   return pl;
 }
@@ -663,8 +774,13 @@ int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st) {
   p.group = a.group;
   p.G = static_cast<int>(a.K / a.group);
   p.kblocks = static_cast<int>(a.K / kBlockK);
+  p.n_tiles = plan.n_tiles;
+  p.tiles = plan.n_tiles * plan.m_tiles;
+  p.stream = plan.stream;
   p.splits = plan.splits;
   p.kb_per_split = plan.kb_per_split;
+  p.base = plan.base;
+  p.rem = plan.rem;
   p.codes = a.codes;
   p.scale = a.scale;
   p.sx = a.sx;

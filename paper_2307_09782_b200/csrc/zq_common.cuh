@@ -63,9 +63,12 @@ struct GemmArgs {
 // Tile shape chosen for a problem (shared by the workspace-size query and the launcher).
 struct GemmPlan {
   int bm;      // tokens per tile (the MMA's N extent)
-  int splits;  // split-K factor
-  int kb_per_split;  // 128-element K blocks per split
   int m_tiles, n_tiles;
+  int stream;  // 1: the (tile, K block) units are dealt out evenly to `ctas` CTAs; 0: tiles x splits CTAs
+  int ctas;
+  int splits;        // stream == 0: split-K factor
+  int kb_per_split;  // stream == 0: 128-element K blocks per split
+  int base, rem;     // stream == 1: units per CTA (the first `rem` CTAs take one more)
   size_t partial_floats;
 };
 GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode);
