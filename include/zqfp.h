@@ -128,8 +128,10 @@ int zq_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  * U : fp16 [N, r] dense or NULL (r = 0);  V : fp16 [r, K], only read when x_bf16 is given and r > 0
  * y : out, [M, ldy] FP32 or bf16 (ydt), ldy >= N in elements
  * K % 128 == 0; group in {64, 128, 256}; r in {0, 8, 16, ..., 64}; q, codes 16-byte aligned.
- * M == 0 or N == 0 is a no-op.  Summation order over K depends on the launch shape (split-K), so
- * FP32 results are reproducible for a fixed (M, N, K) but not bit-identical across token counts.
+ * M == 0 or N == 0 is a no-op.  Summation order over K depends on the launch shape, so FP32 results are
+ * not bit-identical across token counts.  When all tokens fit one tile (M <= 256, constrained modes,
+ * FP32 y) the K range of a tile is shared by CTAs that add into y with FP32 atomics (y is zeroed by the
+ * call first): the last bit can then differ from run to run; other shapes are reproducible.
  */
 int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M,
                    int64_t N, int64_t K, int group, zq_scale_mode mode, const uint8_t* codes,

@@ -60,6 +60,7 @@ struct Params {
   //   stream == 0: CTA c = z * tiles + tile owns K blocks [z * kb_per_split, ...) of that tile
   //   stream == 1: the units of all tiles are dealt out evenly, base (+1 for the first rem CTAs) each
   int stream;
+  int atomic_y;  // streaming launch with FP32 y: CTAs that share a tile add their share into a zeroed y
   int splits, kb_per_split;
   int base, rem;
   const uint8_t* codes;  // tiled weight
@@ -157,18 +158,23 @@ __device__ __forceinline__ size_t partial_slot(const Params& p, int tile, int fi
   return 2 * static_cast<size_t>(c) + (range_start(p, c) / p.kblocks == tile ? 0 : 1);
 }
 
-// Final arithmetic of 16 consecutive tokens (tile columns c0 .. c0+15) of one output channel, and the store.
+// Final arithmetic of NC consecutive tokens (tile columns c0 .. c0+NC-1) of one output channel, and the store.
 //   y[m, n] = sx[m] * cs * acc + sum_j t[m, j] * U[n, j]
 // s_sx / s_t are the tile's token scales and rank-8 LoRC rows in shared memory; u8 holds the channel's
 // U row when r == 8 (the common rank); other ranks read t and U through the cache.
-__device__ __forceinline__ void finalize16(const Params& p, const float* v, int m0, int c0, int n, float cs,
-                                           const float* u8, const float* s_sx, const float* s_t) {
+// `add`: y was zeroed by the launcher and this CTA holds only part of the K range, so it adds (FP32 atomics,
+// order-dependent in the last bit); `lorc`: this CTA is the one that contributes the LoRC term.
+template <int NC>
+__device__ __forceinline__ void finalize(const Params& p, const float* v, int m0, int c0, int n, float cs,
+                                         const float* u8, const float* s_sx, const float* s_t,
+                                         bool add = false, bool lorc = true) {
 #pragma unroll
-  for (int c = 0; c < 16; ++c) {
+  for (int c = 0; c < NC; ++c) {
     const int m = m0 + c0 + c;
     if (m < p.M) {
       float out = s_sx[c0 + c] * cs * v[c];
-      if (p.r == 8) {
+      if (!lorc) {
+      } else if (p.r == 8) {
         const float4 t0 = *reinterpret_cast<const float4*>(s_t + (c0 + c) * 8);
         const float4 t1 = *reinterpret_cast<const float4*>(s_t + (c0 + c) * 8 + 4);
         out = fmaf(t0.x, u8[0], out);
@@ -184,12 +190,21 @@ __device__ __forceinline__ void finalize16(const Params& p, const float* v, int 
         const __half* ur = p.U + static_cast<int64_t>(n) * p.r;
         for (int j = 0; j < p.r; ++j) out = fmaf(__ldg(tr + j), __half2float(__ldg(ur + j)), out);
       }
-      if (p.ydt == ZQ_OUT_F32)
+      if (add)
+        atomicAdd(static_cast<float*>(p.y) + static_cast<int64_t>(m) * p.ldy + n, out);
+      else if (p.ydt == ZQ_OUT_F32)
         static_cast<float*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = out;
       else
         static_cast<__nv_bfloat16*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = __float2bfloat16_rn(out);
     }
   }
+}
+
+template <int NC>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float* v) {
+  if (NC == 16) tmem_ld16(taddr, v);
+  else tmem_ld4(taddr, v);
+  tmem_ld_wait();
 }
 
 template <int BM, bool NONE>
@@ -436,6 +451,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     // Mode none keeps its running sums in a register array, which needs the column loop unrolled; the
     // other modes keep the loop rolled so that its body stays resident in the instruction cache.
     constexpr int kEpiUnroll = NONE ? kMyCols / 16 : 1;
+    // Columns per epilogue step.  A decode CTA runs its epilogue once or twice, on code that is cold in the
+    // instruction cache, so there the body is kept to four columns; larger tiles reuse the body many times.
+    constexpr int EC = (!NONE && BM <= 32) ? 4 : 16;
     const int col0 = NONE ? 0 : part * kMyCols;
     const bool has_cols = NONE ? true : (col0 < BM);
     const uint32_t t_lane = tmem_base + lane_base;
@@ -567,16 +585,29 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
         if (whole_tile) {
           if (!failed && has_cols) {
 #pragma unroll(kEpiUnroll)
-            for (int c = 0; c < kMyCols; c += 16) {
-              float v[16];
+            for (int c = 0; c < kMyCols; c += EC) {
+              float v[EC];
               if (NONE) {
 #pragma unroll
-                for (int e = 0; e < 16; ++e) v[e] = run[c + e];
+                for (int e = 0; e < EC; ++e) v[e] = run[c + e];
               } else {
-                tmem_ld16(t_lane + col0 + c, v);
-                tmem_ld_wait();
+                tmem_ld_cols<EC>(t_lane + col0 + c, v);
               }
-              if (n_ok) finalize16(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+              if (n_ok) finalize<EC>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+            }
+          }
+        } else if (!NONE && p.atomic_y) {
+          // Several CTAs share this tile and y was zeroed before the launch: every CTA scales its share
+          // and adds it; the first contributor also adds the LoRC term.  No fence, ticket or second pass.
+          int first, count;
+          contributors(p, tile, &first, &count);
+          const bool lorc = static_cast<int>(blockIdx.x) == first;
+          if (!failed && has_cols) {
+#pragma unroll 1
+            for (int c = 0; c < kMyCols; c += EC) {
+              float v[EC];
+              tmem_ld_cols<EC>(t_lane + col0 + c, v);
+              if (n_ok) finalize<EC>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t, true, lorc);
             }
           }
         } else {
@@ -588,17 +619,16 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
           float* my_partial = p.partials + partial_slot(p, tile, first, my_j) * (BM * kTileN);
           if (!failed && has_cols) {
 #pragma unroll(kEpiUnroll)
-            for (int c = 0; c < kMyCols; c += 16) {
-              float v[16];
+            for (int c = 0; c < kMyCols; c += EC) {
+              float v[EC];
               if (NONE) {
 #pragma unroll
-                for (int e = 0; e < 16; ++e) v[e] = run[c + e];
+                for (int e = 0; e < EC; ++e) v[e] = run[c + e];
               } else {
-                tmem_ld16(t_lane + col0 + c, v);
-                tmem_ld_wait();
+                tmem_ld_cols<EC>(t_lane + col0 + c, v);
               }
 #pragma unroll
-              for (int e = 0; e < 16; ++e) my_partial[(col0 + c + e) * kTileN + row] = v[e];
+              for (int e = 0; e < EC; ++e) my_partial[(col0 + c + e) * kTileN + row] = v[e];
             }
           }
           __threadfence();
@@ -613,17 +643,17 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
           if (*s_last && has_cols) {
             __threadfence();
 #pragma unroll 1
-            for (int c = 0; c < kMyCols; c += 16) {
-              float v[16];
+            for (int c = 0; c < kMyCols; c += EC) {
+              float v[EC];
 #pragma unroll
-              for (int e = 0; e < 16; ++e) v[e] = 0.0f;
+              for (int e = 0; e < EC; ++e) v[e] = 0.0f;
               for (int j = 0; j < count; ++j) {
                 const float* src =
                     p.partials + partial_slot(p, tile, first, j) * (BM * kTileN) + (col0 + c) * kTileN + row;
 #pragma unroll
-                for (int e = 0; e < 16; ++e) v[e] += __ldcg(src + e * kTileN);
+                for (int e = 0; e < EC; ++e) v[e] += __ldcg(src + e * kTileN);
               }
-              if (n_ok) finalize16(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+              if (n_ok) finalize<EC>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
             }
           }
           named_bar_sync(1, C::kEpiThreads);  // s_last is reused by the next segment
@@ -693,6 +723,10 @@ int launch_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStr
                                     C::kSmemBytes);
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
+  if (p.atomic_y &&
+      cudaMemset2DAsync(a.y, static_cast<size_t>(a.ldy) * 4, 0, static_cast<size_t>(a.N) * 4, static_cast<size_t>(a.M),
+                        st) != cudaSuccess)
+    return ZQ_ERR_CUDA;
   dim3 grid(static_cast<unsigned>(plan.ctas));
   w4a8_gemm_kernel<BM, NONE><<<grid, C::kThreads, C::kSmemBytes, st>>>(tm_q, p);
   count_launch();
@@ -777,6 +811,7 @@ int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st) {
   p.n_tiles = plan.n_tiles;
   p.tiles = plan.n_tiles * plan.m_tiles;
   p.stream = plan.stream;
+  p.atomic_y = (plan.stream && a.ydt == ZQ_OUT_F32 && plan.partial_floats > 0) ? 1 : 0;
   p.splits = plan.splits;
   p.kb_per_split = plan.kb_per_split;
   p.base = plan.base;
