@@ -93,12 +93,17 @@ struct Cfg {
   static constexpr int kDColsPad = kDCols < 32 ? 32 : kDCols;
   static constexpr int kMinBlocks = (NONE || BM > 128) ? 1 : 2;    // CTAs per SM this configuration is sized for
   static constexpr int kTmemCols = kMinBlocks == 2 ? 256 : 512;
+  // Small token tiles (decode) tie the three rings into one: a stage holds the packed tile, the
+  // 2-8 KB token tile and the TMEM stage, is filled by one producer and released by one tcgen05.commit,
+  // so the MMA warp waits once and commits once per K block (its loop is what bounds a decode CTA).
+  static constexpr bool kTied = !NONE && BM <= 64;
   static constexpr int NA = cmin(8, (kTmemCols - kDColsPad) / kAStageCols) / NG * NG;  // widened stages in TMEM
   // shared memory: token stages first (as many as the chain needs, at most 10), the rest to packed stages
   static constexpr int kBudget = (kMinBlocks == 2 ? 104 : 220) * 1024 - BM * 36 - 512;
   static constexpr int kBoth = cmin(10, kBudget / (kTileBytes + kTokBytes));
-  static constexpr int NT = kBoth;
-  static constexpr int NP = cmin(12, (kBudget - NT * kTokBytes) / kTileBytes) / NG * NG;
+  static constexpr int NT = kTied ? cmin(NA, kBoth / NG * NG) : kBoth;
+  static constexpr int NP = kTied ? NT : cmin(12, (kBudget - NT * kTokBytes) / kTileBytes) / NG * NG;
+  static_assert(!kTied || (NT == NA && NP == NA), "tied rings share one depth");
   static constexpr int kEpiThreads = NONE ? 128 : 128 * NG;
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int offTok = 0;
@@ -294,15 +299,18 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       uint32_t ph = 0;
       int tile = u0 / p.kblocks, kb = u0 % p.kblocks;
       for (int i = 0; i < nunits; ++i) {
-        if (!mbar_wait(&p_empty[s], ph ^ 1, s_abort)) {
+        // tied rings: the stage (packed tile, token tile, TMEM stage) is free once the MMAs of the K block
+        // that used it last have completed
+        if (!mbar_wait(C::kTied ? &a_empty[s] : &p_empty[s], ph ^ 1, s_abort)) {
           if (issuer) raise_error(p, s_abort, kErrProducer);
           break;
         }
         if (issuer) {
           const uint8_t* src =
               p.codes + (static_cast<int64_t>(tile % p.n_tiles) * p.kblocks + kb) * kTileBytes;
-          mbar_arrive_expect_tx(&p_full[s], kTileBytes);
+          mbar_arrive_expect_tx(&p_full[s], C::kTied ? kTileBytes + C::kTokBytes : kTileBytes);
           bulk_load(s_packed + s * kTileBytes, src, kTileBytes, &p_full[s]);
+          if (C::kTied) tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, kb * kBlockK, m0, &p_full[s]);
         }
         __syncwarp();
         issued = i + 1;
@@ -324,7 +332,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     }
   } else if (warp == C::kTokenWarp) {
     // ------------------------------------------------------------------ token producer
-    if (ok_start) {  // warp-uniform loop, one elected lane issues the copies
+    if (ok_start && !C::kTied) {  // warp-uniform loop, one elected lane issues the copies
       const bool issuer = elect_one();
       int s = 0, issued = 0;
       uint32_t ph = 0;
@@ -367,7 +375,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       bool seg_first = true;  // the next K block starts a segment (a new accumulation)
       bool failed = false;
       for (int i = 0; i < nunits && !failed; ++i) {
-        if (!mbar_wait(&a_full[sa], pha, s_abort) || !mbar_wait(&t_full[st], pht, s_abort)) {
+        // tied rings: the widen warps saw the stage's barrier (which counts both copies) complete before
+        // they arrived on a_full, so this one wait also orders the token tile before the MMAs
+        if (!mbar_wait(&a_full[sa], pha, s_abort) || (!C::kTied && !mbar_wait(&t_full[st], pht, s_abort))) {
           failed = true;
           break;
         }
@@ -404,7 +414,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
         if (failed) break;
         const bool seg_last = (kb + 1 == p.kblocks) || (i + 1 == nunits);
         if (issuer) {
-          umma_commit(&t_empty[st]);
+          if (!C::kTied) umma_commit(&t_empty[st]);
           umma_commit(&a_empty[sa]);
           if (!NONE && seg_last) umma_commit(&acc_full[seg & 1]);
         }
@@ -471,7 +481,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       if (widen_role) {
         // A lane widens whole rows: 64 packed bytes -> 128 E4M3 bytes = 32 TMEM columns of its own lane.
         for (; wi < ue - u0 && !failed; wi += C::NG) {
-          if (!mbar_wait_warp(&p_full[sp], php, s_abort) || !mbar_wait_warp(&a_empty[sa], pha ^ 1, s_abort)) {
+          // tied rings: the producer refilled the stage only after the MMAs that read its TMEM half were done
+          if (!mbar_wait_warp(&p_full[sp], php, s_abort) ||
+              (!C::kTied && !mbar_wait_warp(&a_empty[sa], pha ^ 1, s_abort))) {
             raise_error(p, s_abort, kErrWiden);
             failed = true;
             break;
@@ -501,7 +513,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
           }
           // every lane's loads of the packed tile have been consumed: hand the stage back
           __syncwarp();
-          if (lane == 0) mbar_arrive(&p_empty[sp]);
+          if (!C::kTied && lane == 0) mbar_arrive(&p_empty[sp]);
           const uint32_t dst = tmem_a + sa * kAStageCols + lane_base;
           tmem_st16(dst, w);
           tmem_st16(dst + 16, w + 16);
@@ -762,9 +774,11 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
   const int ctas_per_sm = (mode == ZQ_SCALE_NONE || bm > 128) ? 1 : 2;
   const int64_t resident = static_cast<int64_t>(ctas_per_sm) * sm_count();
   const int64_t units = tiles * kblocks;
-  if (mode != ZQ_SCALE_NONE && pl.m_tiles == 1 && tiles <= kWsMaxTiles && units >= 8 && units < (int64_t(1) << 30)) {
-    // One row of output tiles (decode): the weight streams exactly once, so deal the (tile, K block)
-    // units out evenly to one resident wave of CTAs, at least 4 units each.
+  if (mode != ZQ_SCALE_NONE && bm == 16 && pl.m_tiles == 1 && tiles <= kWsMaxTiles && units >= 8 &&
+      units < (int64_t(1) << 30)) {
+    // At most 16 tokens (decode): the weight streams exactly once and the per-tile epilogue is tiny, so deal
+    // the (tile, K block) units out evenly to one resident wave of CTAs, at least 4 units each.  (Wider
+    // token tiles measured slower this way: their shared tiles cost more atomics than the wave balance saves.)
     int64_t g = resident < units / 4 ? resident : units / 4;
     if (g < 1) g = 1;
     pl.stream = 1;
