@@ -171,43 +171,61 @@ __device__ __forceinline__ size_t partial_slot(const Params& p, int tile, int fi
 // order-dependent in the last bit); `lorc`: this CTA is the one that contributes the LoRC term.
 template <int NC>
 __device__ __forceinline__ void finalize(const Params& p, const float* v, int m0, int c0, int n, float cs,
-                                         const float* u8, const float* s_sx, const float* s_t,
-                                         bool add = false, bool lorc = true) {
+                                         const float* u8, const float* __restrict__ s_sx,
+                                         const float* __restrict__ s_t, bool add = false, bool lorc = true) {
+  // All NC results are computed before the first store, so that the columns' loads and FMA chains
+  // interleave instead of running one column at a time behind each store.
+  float out[NC];
 #pragma unroll
-  for (int c = 0; c < NC; ++c) {
-    const int m = m0 + c0 + c;
-    if (m < p.M) {
-      float out = s_sx[c0 + c] * cs * v[c];
-      if (!lorc) {
-      } else if (p.r == 8) {
-        const float4 t0 = *reinterpret_cast<const float4*>(s_t + (c0 + c) * 8);
-        const float4 t1 = *reinterpret_cast<const float4*>(s_t + (c0 + c) * 8 + 4);
-        out = fmaf(t0.x, u8[0], out);
-        out = fmaf(t0.y, u8[1], out);
-        out = fmaf(t0.z, u8[2], out);
-        out = fmaf(t0.w, u8[3], out);
-        out = fmaf(t1.x, u8[4], out);
-        out = fmaf(t1.y, u8[5], out);
-        out = fmaf(t1.z, u8[6], out);
-        out = fmaf(t1.w, u8[7], out);
-      } else if (p.r > 0) {
+  for (int c = 0; c < NC; ++c) out[c] = s_sx[c0 + c] * cs * v[c];
+  if (lorc && p.r == 8) {
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      const float4 t0 = *reinterpret_cast<const float4*>(s_t + (c0 + c) * 8);
+      const float4 t1 = *reinterpret_cast<const float4*>(s_t + (c0 + c) * 8 + 4);
+      float lo = t0.x * u8[0], hi = t1.x * u8[4];
+      lo = fmaf(t0.y, u8[1], lo);
+      hi = fmaf(t1.y, u8[5], hi);
+      lo = fmaf(t0.z, u8[2], lo);
+      hi = fmaf(t1.z, u8[6], hi);
+      lo = fmaf(t0.w, u8[3], lo);
+      hi = fmaf(t1.w, u8[7], hi);
+      out[c] += lo + hi;
+    }
+  } else if (lorc && p.r > 0) {
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      const int m = m0 + c0 + c;
+      if (m < p.M) {
         const float* tr = p.t + static_cast<int64_t>(m) * p.r;
         const __half* ur = p.U + static_cast<int64_t>(n) * p.r;
-        for (int j = 0; j < p.r; ++j) out = fmaf(__ldg(tr + j), __half2float(__ldg(ur + j)), out);
+        for (int j = 0; j < p.r; ++j) out[c] = fmaf(__ldg(tr + j), __half2float(__ldg(ur + j)), out[c]);
       }
-      if (add)
-        atomicAdd(static_cast<float*>(p.y) + static_cast<int64_t>(m) * p.ldy + n, out);
-      else if (p.ydt == ZQ_OUT_F32)
-        static_cast<float*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = out;
-      else
-        static_cast<__nv_bfloat16*>(p.y)[static_cast<int64_t>(m) * p.ldy + n] = __float2bfloat16_rn(out);
     }
+  }
+  const int64_t base = static_cast<int64_t>(m0 + c0) * p.ldy + n;
+  if (add) {
+    float* y = static_cast<float*>(p.y) + base;
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+      if (m0 + c0 + c < p.M) atomicAdd(y + c * p.ldy, out[c]);
+  } else if (p.ydt == ZQ_OUT_F32) {
+    float* y = static_cast<float*>(p.y) + base;
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+      if (m0 + c0 + c < p.M) y[c * p.ldy] = out[c];
+  } else {
+    __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.y) + base;
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+      if (m0 + c0 + c < p.M) y[c * p.ldy] = __float2bfloat16_rn(out[c]);
   }
 }
 
 template <int NC>
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float* v) {
   if (NC == 16) tmem_ld16(taddr, v);
+  else if (NC == 8) tmem_ld8(taddr, v);
   else tmem_ld4(taddr, v);
   tmem_ld_wait();
 }
@@ -462,8 +480,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     // other modes keep the loop rolled so that its body stays resident in the instruction cache.
     constexpr int kEpiUnroll = NONE ? kMyCols / 16 : 1;
     // Columns per epilogue step.  A decode CTA runs its epilogue once or twice, on code that is cold in the
-    // instruction cache, so there the body is kept to four columns; larger tiles reuse the body many times.
-    constexpr int EC = (!NONE && BM <= 32) ? 4 : 16;
+    // instruction cache, so there the body is kept to four columns; larger tiles reuse the body many times
+    // (eight columns where two CTAs share an SM and registers are scarcer).
+    constexpr int EC = NONE ? 16 : (BM <= 32 ? 4 : (BM <= 128 ? 8 : 16));
     const int col0 = NONE ? 0 : part * kMyCols;
     const bool has_cols = NONE ? true : (col0 < BM);
     const uint32_t t_lane = tmem_base + lane_base;
