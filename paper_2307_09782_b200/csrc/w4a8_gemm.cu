@@ -81,7 +81,10 @@ constexpr int cmin(int a, int b) { return a < b ? a : b; }
 
 template <int BM, bool NONE>
 struct Cfg {
-  static constexpr int NG = 2;  // widen groups
+  // CTAs per SM this configuration is sized for.  Decode tiles run three small CTAs per SM, so that one
+  // CTA's start-up and per-tile epilogue overlap the others' main loops.
+  static constexpr int kMinBlocks = (NONE || BM > 128) ? 1 : (BM <= 16 ? 3 : 2);
+  static constexpr int NG = kMinBlocks == 3 ? 1 : 2;  // widen groups
   static constexpr int kWidenWarps = 4 * NG;
   static constexpr int kWeightWarp = kWidenWarps;
   static constexpr int kTokenWarp = kWidenWarps + 1;
@@ -91,15 +94,14 @@ struct Cfg {
   static constexpr int kTokBytes = BM * kBlockK;
   static constexpr int kDCols = NONE ? 2 * BM : BM;                 // accumulator columns (two buffers in mode none)
   static constexpr int kDColsPad = kDCols < 32 ? 32 : kDCols;
-  static constexpr int kMinBlocks = (NONE || BM > 128) ? 1 : 2;    // CTAs per SM this configuration is sized for
-  static constexpr int kTmemCols = kMinBlocks == 2 ? 256 : 512;
+  static constexpr int kTmemCols = kMinBlocks == 1 ? 512 : (kMinBlocks == 2 ? 256 : 128);
   // Small token tiles (decode) tie the three rings into one: a stage holds the packed tile, the
   // 2-8 KB token tile and the TMEM stage, is filled by one producer and released by one tcgen05.commit,
   // so the MMA warp waits once and commits once per K block (its loop is what bounds a decode CTA).
-  static constexpr bool kTied = !NONE && BM <= 64;
+  static constexpr bool kTied = !NONE && BM >= 32 && BM <= 64;
   static constexpr int NA = cmin(8, (kTmemCols - kDColsPad) / kAStageCols) / NG * NG;  // widened stages in TMEM
   // shared memory: token stages first (as many as the chain needs, at most 10), the rest to packed stages
-  static constexpr int kBudget = (kMinBlocks == 2 ? 104 : 220) * 1024 - BM * 36 - 512;
+  static constexpr int kBudget = (kMinBlocks == 1 ? 220 : (kMinBlocks == 2 ? 104 : 70)) * 1024 - BM * 36 - 512;
   static constexpr int kBoth = cmin(10, kBudget / (kTileBytes + kTokBytes));
   static constexpr int NT = kTied ? cmin(NA, kBoth / NG * NG) : kBoth;
   static constexpr int NP = kTied ? NT : cmin(12, (kBudget - NT * kTokBytes) / kTileBytes) / NG * NG;
@@ -790,7 +792,7 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
   pl.n_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
   const int64_t tiles = static_cast<int64_t>(pl.m_tiles) * pl.n_tiles;
   const int kblocks = static_cast<int>(K / kBlockK);
-  const int ctas_per_sm = (mode == ZQ_SCALE_NONE || bm > 128) ? 1 : 2;
+  const int ctas_per_sm = (mode == ZQ_SCALE_NONE || bm > 128) ? 1 : (bm <= 16 ? 3 : 2);
   const int64_t resident = static_cast<int64_t>(ctas_per_sm) * sm_count();
   const int64_t units = tiles * kblocks;
   if (mode != ZQ_SCALE_NONE && bm == 16 && pl.m_tiles == 1 && tiles <= kWsMaxTiles && units >= 8 &&
@@ -813,7 +815,7 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
   // split K until about one resident wave of CTAs exists, keeping at least 4 K blocks per CTA and (for
   // 256-wide groups) whole groups per CTA
   int splits = 1;
-  const int64_t target = 2 * sm_count();
+  const int64_t target = static_cast<int64_t>(ctas_per_sm < 2 ? 2 : ctas_per_sm) * sm_count();
   if (tiles < target && tiles <= kWsMaxTiles) {
     splits = static_cast<int>((target + tiles - 1) / tiles);
     const int max_splits = kblocks / 4 > 0 ? kblocks / 4 : 1;
