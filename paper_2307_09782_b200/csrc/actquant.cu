@@ -4,6 +4,7 @@
 // One CTA per token.  The row is read once from HBM with 16-byte loads and kept in registers
 // between the absmax reduction and the cast (rows longer than the register budget are re-read).
 // A thread's unit is 16 consecutive elements: two 16-byte loads in, one 16-byte store out.
+#include <cooperative_groups.h>
 #include <cuda_fp16.h>
 
 #include "zq_common.cuh"
@@ -289,6 +290,117 @@ act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec
   }
 }
 
+// ---- few tokens: a cluster of eight CTAs per row -------------------------------------------------
+// With one CTA per token a decode-size call (1-64 tokens) leaves most SMs idle and its latency is one
+// CTA walking a whole row and all of V.  Here eight CTAs of a thread-block cluster share a row: each
+// takes an eighth of K, the partial absmax and LoRC sums meet through distributed shared memory, and
+// every CTA casts its own part.
+constexpr int kClusterSize = 8;
+constexpr int kClusterThreads = 256;
+constexpr int kClusterVpt = 2;  // 16-element units a thread keeps in registers
+
+__global__ void __cluster_dims__(kClusterSize, 1, 1) __launch_bounds__(kClusterThreads)
+act_quant_cluster_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, uint8_t* __restrict__ q,
+                         float* __restrict__ sx, const uint4* __restrict__ V, int r, float* __restrict__ t) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = static_cast<int>(cluster.block_rank());
+  const int64_t m = blockIdx.y;
+  const int nunits = K / kUnit;
+  const int per = (nunits + kClusterSize - 1) / kClusterSize;
+  const int u_begin = rank * per, u_end = min(nunits, u_begin + per);
+  const uint4* row = x + m * ldx_vec;
+  uint4* qrow = reinterpret_cast<uint4*>(q + m * static_cast<int64_t>(K));
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  __shared__ float s_warp[kClusterThreads / 32];
+  __shared__ float s_warp_t[kClusterThreads / 32][kRChunk];
+  __shared__ float s_amax;        // this CTA's partial absmax (read by the whole cluster)
+  __shared__ float s_tpart[64];   // this CTA's partial LoRC sums (read by rank 0)
+
+  uint4 c0[kClusterVpt], c1[kClusterVpt];
+  float a = 0.0f;
+#pragma unroll
+  for (int i = 0; i < kClusterVpt; ++i) {
+    const int u = u_begin + tid + i * kClusterThreads;
+    if (u < u_end) {
+      c0[i] = __ldg(row + 2 * u);
+      c1[i] = __ldg(row + 2 * u + 1);
+    } else {
+      c0[i] = make_uint4(0, 0, 0, 0);
+      c1[i] = make_uint4(0, 0, 0, 0);
+    }
+    a = absmax8(c1[i], absmax8(c0[i], a));
+  }
+  a = warp_max(a);
+  if (lane == 0) s_warp[warp] = a;
+
+  if (V != nullptr) {
+    const int kvec = K / 8;
+    for (int j0 = 0; j0 < r; j0 += kRChunk) {
+      float acc[kRChunk];
+#pragma unroll
+      for (int j = 0; j < kRChunk; ++j) acc[j] = 0.0f;
+#pragma unroll
+      for (int i = 0; i < kClusterVpt; ++i) {
+        const int u = u_begin + tid + i * kClusterThreads;
+        if (u < u_end) {
+#pragma unroll
+          for (int j = 0; j < kRChunk; ++j)
+            if (j0 + j < r) {
+              const uint4* vr = V + static_cast<int64_t>(j0 + j) * kvec;
+              acc[j] = dot8(c1[i], __ldg(vr + 2 * u + 1), dot8(c0[i], __ldg(vr + 2 * u), acc[j]));
+            }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < kRChunk; ++j) {
+        const float v = warp_sum(acc[j]);
+        if (lane == 0) s_warp_t[warp][j] = v;
+      }
+      __syncthreads();
+      if (tid < kRChunk && j0 + tid < r) {
+        float v = 0.0f;
+        for (int w = 0; w < kClusterThreads / 32; ++w) v += s_warp_t[w][tid];
+        s_tpart[j0 + tid] = v;
+      }
+      __syncthreads();
+    }
+  } else {
+    __syncthreads();
+  }
+  if (tid == 0) {
+    float v = s_warp[0];
+    for (int w = 1; w < kClusterThreads / 32; ++w) v = fmaxf(v, s_warp[w]);
+    s_amax = v;
+  }
+  cluster.sync();  // every CTA's s_amax and s_tpart are written and visible cluster-wide
+
+  float amax = 0.0f;
+  for (int k = 0; k < kClusterSize; ++k) amax = fmaxf(amax, *cluster.map_shared_rank(&s_amax, k));
+  float s = 1.0f, inv = 1.0f;
+  if (amax != 0.0f) {
+    s = __fdiv_rn(amax, 448.0f);
+    inv = __fdiv_rn(448.0f, amax);
+  }
+  if (rank == 0) {
+    if (tid == 0) sx[m] = s;
+    if (V != nullptr && tid < r) {
+      float v = 0.0f;
+      for (int k = 0; k < kClusterSize; ++k) v += cluster.map_shared_rank(s_tpart, k)[tid];
+      t[m * r + tid] = v;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kClusterVpt; ++i) {
+    const int u = u_begin + tid + i * kClusterThreads;
+    if (u < u_end) {
+      const uint2 lo = cast8(c0[i], inv), hi = cast8(c1[i], inv);
+      qrow[u] = make_uint4(lo.x, lo.y, hi.x, hi.y);
+    }
+  }
+  cluster.sync();  // no CTA may exit while a peer can still read its shared memory
+}
+
 }  // namespace
 
 int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
@@ -304,6 +416,14 @@ int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* 
     else
       act_quant_rows_kernel<false><<<grid, kRowsThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(M),
                                                                  static_cast<int>(K), ldx / 8, q, sx, nullptr, t);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+  }
+  // few tokens and rows long enough to be worth sharing: a cluster of eight CTAs per row
+  if (M <= 64 && K >= 2048 && K / kUnit <= kClusterSize * kClusterThreads * kClusterVpt) {
+    dim3 grid(kClusterSize, static_cast<unsigned>(M));
+    act_quant_cluster_kernel<<<grid, kClusterThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(K),
+                                                              ldx / 8, q, sx, static_cast<const uint4*>(V), r, t);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
   }
