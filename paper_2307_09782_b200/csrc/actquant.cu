@@ -419,8 +419,9 @@ int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* 
     count_launch();
     return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
   }
-  // few tokens and rows long enough to be worth sharing: a cluster of eight CTAs per row
-  if (M <= 64 && K >= 2048 && K / kUnit <= kClusterSize * kClusterThreads * kClusterVpt) {
+  // fewer tokens than the eight-row kernel needs, rows long enough to be worth sharing: a cluster of eight CTAs per row
+  if (M < 8 * 148 && (M <= 256 || K >= 16384) && K >= 2048 &&
+      K / kUnit <= kClusterSize * kClusterThreads * kClusterVpt) {
     dim3 grid(kClusterSize, static_cast<unsigned>(M));
     act_quant_cluster_kernel<<<grid, kClusterThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(K),
                                                               ldx / 8, q, sx, static_cast<const uint4*>(V), r, t);
