@@ -167,34 +167,42 @@ __device__ __forceinline__ size_t partial_slot(const Params& p, int tile, int fi
 
 // Final arithmetic of NC consecutive tokens (tile columns c0 .. c0+NC-1) of one output channel, and the store.
 //   y[m, n] = sx[m] * cs * acc + sum_j t[m, j] * U[n, j]
-// s_sx / s_t are the tile's token scales and rank-8 LoRC rows in shared memory; u8 holds the channel's
-// U row when r == 8 (the common rank); other ranks read t and U through the cache.
+// s_sx holds the tile's token scales and s_tT its rank-8 LoRC rows, transposed ([j][BM]) so that two
+// neighbouring tokens' t values sit side by side: tokens are finished in pairs with packed FP32
+// instructions.  u2 holds the channel's U row, each value in both halves, when r == 8 (the common rank);
+// other ranks read t and U through the cache.
 // `add`: y was zeroed by the launcher and this CTA holds only part of the K range, so it adds (FP32 atomics,
 // order-dependent in the last bit); `lorc`: this CTA is the one that contributes the LoRC term.
-template <int NC>
+template <int NC, int BM>
 __device__ __forceinline__ void finalize(const Params& p, const float* v, int m0, int c0, int n, float cs,
-                                         const float* u8, const float* __restrict__ s_sx,
-                                         const float* __restrict__ s_t, bool add = false, bool lorc = true) {
+                                         const uint64_t* u2, const float* __restrict__ s_sx,
+                                         const float* __restrict__ s_tT, bool add = false, bool lorc = true) {
   // All NC results are computed before the first store, so that the columns' loads and FMA chains
   // interleave instead of running one column at a time behind each store.
-  float out[NC];
+  static_assert(NC % 4 == 0, "columns are taken four at a time");
+  uint64_t o2[NC / 2];
+  const uint64_t cs2 = pack2(cs, cs);
 #pragma unroll
-  for (int c = 0; c < NC; ++c) out[c] = s_sx[c0 + c] * cs * v[c];
+  for (int c = 0; c < NC; c += 4) {
+    const float4 s4 = *reinterpret_cast<const float4*>(s_sx + c0 + c);
+    o2[c / 2] = mul2(mul2(pack2(s4.x, s4.y), cs2), pack2(v[c], v[c + 1]));
+    o2[c / 2 + 1] = mul2(mul2(pack2(s4.z, s4.w), cs2), pack2(v[c + 2], v[c + 3]));
+  }
   if (lorc && p.r == 8) {
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      const float4 t0 = *reinterpret_cast<const float4*>(s_t + (c0 + c) * 8);
-      const float4 t1 = *reinterpret_cast<const float4*>(s_t + (c0 + c) * 8 + 4);
-      float lo = t0.x * u8[0], hi = t1.x * u8[4];
-      lo = fmaf(t0.y, u8[1], lo);
-      hi = fmaf(t1.y, u8[5], hi);
-      lo = fmaf(t0.z, u8[2], lo);
-      hi = fmaf(t1.z, u8[6], hi);
-      lo = fmaf(t0.w, u8[3], lo);
-      hi = fmaf(t1.w, u8[7], hi);
-      out[c] += lo + hi;
+    for (int j = 0; j < 8; ++j) {
+#pragma unroll
+      for (int c = 0; c < NC; c += 4) {
+        const float4 t4 = *reinterpret_cast<const float4*>(s_tT + j * BM + c0 + c);
+        o2[c / 2] = fma2(pack2(t4.x, t4.y), u2[j], o2[c / 2]);
+        o2[c / 2 + 1] = fma2(pack2(t4.z, t4.w), u2[j], o2[c / 2 + 1]);
+      }
     }
-  } else if (lorc && p.r > 0) {
+  }
+  float out[NC];
+#pragma unroll
+  for (int c = 0; c < NC; c += 2) unpack2(o2[c / 2], out[c], out[c + 1]);
+  if (lorc && p.r > 0 && p.r != 8) {
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
       const int m = m0 + c0 + c;
@@ -225,10 +233,14 @@ __device__ __forceinline__ void finalize(const Params& p, const float* v, int m0
 }
 
 template <int NC>
-__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float* v) {
+__device__ __forceinline__ void tmem_ld_issue(uint32_t taddr, float* v) {
   if (NC == 16) tmem_ld16(taddr, v);
   else if (NC == 8) tmem_ld8(taddr, v);
   else tmem_ld4(taddr, v);
+}
+template <int NC>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float* v) {
+  tmem_ld_issue<NC>(taddr, v);
   tmem_ld_wait();
 }
 
@@ -300,8 +312,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     // token scales and (rank 8) LoRC rows of this CTA's tokens, for the epilogue
     for (int c = threadIdx.x; c < BM; c += 32 * C::kWidenWarps) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
     if (p.r == 8)
-      for (int c = threadIdx.x; c < BM * 8; c += 32 * C::kWidenWarps)
-        s_t[c] = (m0 + (c >> 3) < p.M) ? __ldg(p.t + static_cast<int64_t>(m0) * 8 + c) : 0.0f;
+      for (int c = threadIdx.x; c < BM * 8; c += 32 * C::kWidenWarps)  // transposed: [j][BM]
+        s_t[(c & 7) * BM + (c >> 3)] = (m0 + (c >> 3) < p.M) ? __ldg(p.t + static_cast<int64_t>(m0) * 8 + c) : 0.0f;
   }
   if (warp == C::kMmaWarp) tmem_alloc(s_tmem, C::kTmemCols);
   tc_fence_before_sync();
@@ -558,9 +570,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
       // ---- accumulators -> registers -> y (or -> workspace, when other CTAs share the tile)
       if (epi_role) {
         float cs = 1.0f;
-        float u[8];
+        uint64_t u[8];  // the channel's U row, each value in both halves of a packed pair
 #pragma unroll
-        for (int e = 0; e < 8; ++e) u[e] = 0.0f;
+        for (int e = 0; e < 8; ++e) u[e] = 0ull;
         if (!NONE && n_ok) cs = __ldg(p.scale + n);
         if (p.r == 8 && n_ok) {
           const uint4 h = __ldg(reinterpret_cast<const uint4*>(p.U + static_cast<int64_t>(n) * 8));
@@ -570,8 +582,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
             __half2 h2;
             *reinterpret_cast<uint32_t*>(&h2) = hw[e];
             const float2 f = __half22float2(h2);
-            u[2 * e] = f.x;
-            u[2 * e + 1] = f.y;
+            u[2 * e] = pack2(f.x, f.x);
+            u[2 * e + 1] = pack2(f.y, f.y);
           }
         }
 
@@ -616,17 +628,24 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
 
         const bool whole_tile = (ue - us) == p.kblocks;
         if (whole_tile) {
-          if (!failed && has_cols) {
-#pragma unroll(kEpiUnroll)
+          if (NONE) {
+            if (!failed) {
+#pragma unroll
+              for (int c = 0; c < BM; c += EC)
+                if (n_ok) finalize<EC, BM>(p, run + c, m0, c, n, cs, u, s_sx, s_t);
+            }
+          } else if (!failed && has_cols) {
+            // the next step's accumulator columns are in flight while this step's are finished
+            float nxt[EC];
+            tmem_ld_issue<EC>(t_lane + col0, nxt);
+#pragma unroll 1
             for (int c = 0; c < kMyCols; c += EC) {
               float v[EC];
-              if (NONE) {
+              tmem_ld_wait_regs<EC>(nxt);
 #pragma unroll
-                for (int e = 0; e < EC; ++e) v[e] = run[c + e];
-              } else {
-                tmem_ld_cols<EC>(t_lane + col0 + c, v);
-              }
-              if (n_ok) finalize<EC>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+              for (int e = 0; e < EC; ++e) v[e] = nxt[e];
+              if (c + EC < kMyCols) tmem_ld_issue<EC>(t_lane + col0 + c + EC, nxt);
+              if (n_ok) finalize<EC, BM>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
             }
           }
         } else if (!NONE && p.atomic_y) {
@@ -640,7 +659,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
             for (int c = 0; c < kMyCols; c += EC) {
               float v[EC];
               tmem_ld_cols<EC>(t_lane + col0 + c, v);
-              if (n_ok) finalize<EC>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t, true, lorc);
+              if (n_ok) finalize<EC, BM>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t, true, lorc);
             }
           }
         } else {
@@ -686,7 +705,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
 #pragma unroll
                 for (int e = 0; e < EC; ++e) v[e] += __ldcg(src + e * kTileN);
               }
-              if (n_ok) finalize<EC>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+              if (n_ok) finalize<EC, BM>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
             }
           }
           named_bar_sync(1, C::kEpiThreads);  // s_last is reused by the next segment
