@@ -41,6 +41,14 @@ typedef enum {
 
 typedef enum { ZQ_OUT_F32 = 0, ZQ_OUT_BF16 = 1 } zq_out_dtype;
 
+/* How the packed weight is laid out, which decides who performs the cast FP4 -> FP8 of Section 3
+ * ("Casting the FP4 to FP8") during the GEMM.  Codes, shifts and scales are the same either way. */
+typedef enum {
+  ZQ_WEIGHTS_CAST = 0, /* the kernel casts each code to E4M3 itself, as an exponent-field subtraction */
+  ZQ_WEIGHTS_MX = 1    /* modes M1 / M2 only: the tensor core reads the E2M1 codes directly and applies the
+                          power-of-two shift of each group as an E8M0 block scale (exact, being a power of two) */
+} zq_weight_layout;
+
 const char* zq_status_string(int status);
 
 /*
@@ -63,11 +71,12 @@ int zq_quantize_act_fp8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, u
 
 /*
  * Sizes in bytes of the three buffers zq_pack_weight_fp4 writes:
- *   codes: ceil(N/128) * (K/128) * 8448 (tiled, see below) ; shift: N*G (M1, M2) or 0 (none) ;
+ *   codes: ceil(N/128) * (K/128) * 8448 (ZQ_WEIGHTS_CAST) or * 8704 (ZQ_WEIGHTS_MX), tiled, see below ;
+ *   shift: N*G (M1, M2) or 0 (none) ;
  *   scale: 4*N (M1, M2) or 4*N*G (none).
  */
-int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, size_t* codes_bytes,
-                           size_t* shift_bytes, size_t* scale_bytes);
+int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout,
+                           size_t* codes_bytes, size_t* shift_bytes, size_t* scale_bytes);
 
 /*
  * Fine-grained FP4 weight quantization (Section 3: FGQ; Appendix A: group size) with the scale
@@ -94,12 +103,18 @@ int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, 
  *             (b = 0..3);
  *           - byte 8192 + 2r + h = the shift of row r for elements 64h .. 64h+63 (0 in mode none).
  *         Rows of the last tile beyond N are zero.
+ *         With ZQ_WEIGHTS_MX (M1 / M2 only; ZQ_ERR_MODE otherwise) a tile is 8704 bytes, 32-byte aligned:
+ *           - [0, 8192): row r at r*64, element k of the K block in byte k/2, even k in the low nibble, a
+ *             nibble being the E2M1 code s e1 e0 m;
+ *           - byte 8192 + 16*(r % 32) + 4*(r / 32) + s = 127 - shift of row r for elements 32s .. 32s+31
+ *             (the E8M0 encoding of 2^-shift), the order in which the tensor core's scale copy reads them.
+ *         Rows beyond N have zero codes and scale bytes 127.
  * shift : out, u8 [N, G] (M1, M2), the same shifts in plain form; ignored (may be NULL) in mode none
  * scale : out, FP32 [N] (M1, M2) or [N, G] (none)
  * group in {64, 128, 256}; K % group == 0 and K % 128 == 0; N >= 0.
  */
 int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale_mode mode,
-                       uint8_t* codes, uint8_t* shift, float* scale, void* stream);
+                       zq_weight_layout layout, uint8_t* codes, uint8_t* shift, float* scale, void* stream);
 
 /*
  * Workspace for zq_w4a8_linear: a status word, split-K tile counters and partial sums, and (when the
@@ -116,26 +131,29 @@ int zq_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  *            + sum_{j<r} U[n,j] * t[m,j]
  * For M1 / M2 the weight is cast to E4M3 inside the kernel by subtracting shift[n, k/group] from the
  * exponent field (Section 3, "Casting the FP4 to FP8"), the FP8 x FP8 products are accumulated in
- * FP32 over all of K, and sx[m] * scale[n] multiplies the sum once.  In mode none the FP32
- * group scale multiplies each group's partial sum.
+ * FP32 over all of K, and sx[m] * scale[n] multiplies the sum once.  With ZQ_WEIGHTS_MX the tensor core
+ * performs that cast: it multiplies the E2M1 codes by the E4M3 activations and by 2^-shift as a block
+ * scale; the products and their sum are the same numbers.  In mode none the FP32 group scale multiplies
+ * each group's partial sum.
  *
  * Activations come either pre-quantized (q, sx, and t when r > 0; x_bf16 = NULL) or raw
  * (x_bf16 [M, ldx] given, q = sx = t = NULL): then the call first runs zq_quantize_act_fp8 into the
  * workspace (with V when r > 0).
  *
- * codes / scale : as written by zq_pack_weight_fp4 for the same (N, K, group, mode); shift is not read
+ * codes / scale : as written by zq_pack_weight_fp4 for the same (N, K, group, mode, layout); shift is not read
  *                 (the tiles carry the shifts) and may be NULL
  * U : fp16 [N, r] dense or NULL (r = 0);  V : fp16 [r, K], only read when x_bf16 is given and r > 0
  * y : out, [M, ldy] FP32 or bf16 (ydt), ldy >= N in elements
- * K % 128 == 0; group in {64, 128, 256}; r in {0, 8, 16, ..., 64}; q, codes 16-byte aligned.
+ * K % 128 == 0; group in {64, 128, 256}; r in {0, 8, 16, ..., 64}; q, codes 16-byte aligned (codes 32-byte
+ * aligned with ZQ_WEIGHTS_MX).
  * M == 0 or N == 0 is a no-op.  Summation order over K depends on the launch shape, so FP32 results are
  * not bit-identical across token counts.  When all tokens fit one tile (M <= 256, constrained modes,
  * FP32 y) the K range of a tile is shared by CTAs that add into y with FP32 atomics (y is zeroed by the
  * call first): the last bit can then differ from run to run; other shapes are reproducible.
  */
 int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M,
-                   int64_t N, int64_t K, int group, zq_scale_mode mode, const uint8_t* codes,
-                   const uint8_t* shift, const float* scale, const void* U_f16, const void* V_f16,
+                   int64_t N, int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout,
+                   const uint8_t* codes, const uint8_t* shift, const float* scale, const void* U_f16, const void* V_f16,
                    const float* t, int r, void* y, zq_out_dtype ydt, int64_t ldy, void* workspace,
                    size_t workspace_bytes, void* stream);
 
@@ -148,8 +166,8 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
  */
 size_t zq_w4a8_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int r);
 int zq_w4a8_linear_host(const void* x_bf16_host, int64_t M, int64_t N, int64_t K, int group,
-                        zq_scale_mode mode, const uint8_t* codes, const uint8_t* shift,
-                        const float* scale, const void* U_f16, const void* V_f16, int r,
+                        zq_scale_mode mode, zq_weight_layout layout, const uint8_t* codes,
+                        const uint8_t* shift, const float* scale, const void* U_f16, const void* V_f16, int r,
                         float* y_host, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
@@ -169,7 +187,8 @@ int zq_device_status(void* workspace, int* detail, void* stream);
  * (zq_w4a8_linear_noalloc_max_scratch_bytes), resident on every GPU that loads the library until the
  * process exits.  The call allocates and frees nothing.
  *
- * Same operation, arguments and limits as zq_w4a8_linear with pre-quantized activations (q, sx, and
+ * Same operation, arguments and limits as zq_w4a8_linear with weights in the ZQ_WEIGHTS_CAST layout and
+ * pre-quantized activations (q, sx, and
  * t when r > 0; there is no raw-x path, since that would need scratch for q).  The fixed array bounds
  * the split-K partial sums (4 bytes x splits x padded M x padded N).  A problem that needs more
  * returns ZQ_ERR_WORKSPACE and launches nothing.  Problems with about 300 or more 128 x 256 output

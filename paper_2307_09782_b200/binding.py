@@ -19,6 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libzqfp.so")
 SCALE_NONE, SCALE_M1, SCALE_M2 = 0, 1, 2
 MODES = {"none": SCALE_NONE, "M1": SCALE_M1, "M2": SCALE_M2}
 OUT_F32, OUT_BF16 = 0, 1
+WEIGHTS_CAST, WEIGHTS_MX = 0, 1
+LAYOUTS = {"cast": WEIGHTS_CAST, "mx": WEIGHTS_MX}
 
 EXPORTS = [
     "zq_status_string", "zq_quantize_act_fp8", "zq_packed_weight_sizes", "zq_pack_weight_fp4",
@@ -50,9 +52,9 @@ def lib() -> C.CDLL:
         L.zq_quantize_act_fp8.restype = ci
         L.zq_quantize_act_fp8.argtypes = [vp, i64, i64, i64, vp, vp, vp, ci, vp, vp]
         L.zq_packed_weight_sizes.restype = ci
-        L.zq_packed_weight_sizes.argtypes = [i64, i64, ci, ci, C.POINTER(sz), C.POINTER(sz), C.POINTER(sz)]
+        L.zq_packed_weight_sizes.argtypes = [i64, i64, ci, ci, ci, C.POINTER(sz), C.POINTER(sz), C.POINTER(sz)]
         L.zq_pack_weight_fp4.restype = ci
-        L.zq_pack_weight_fp4.argtypes = [vp, i64, i64, ci, ci, vp, vp, vp, vp]
+        L.zq_pack_weight_fp4.argtypes = [vp, i64, i64, ci, ci, ci, vp, vp, vp, vp]
         L.zq_w4a8_linear_workspace_bytes.restype = sz
         L.zq_w4a8_linear_workspace_bytes.argtypes = [i64, i64, i64, ci]
         L.zq_w4a8_linear_host_workspace_bytes.restype = sz
@@ -60,10 +62,10 @@ def lib() -> C.CDLL:
         L.zq_workspace_init.restype = ci
         L.zq_workspace_init.argtypes = [vp, sz, vp]
         L.zq_w4a8_linear.restype = ci
-        L.zq_w4a8_linear.argtypes = [vp, vp, vp, i64, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, vp, ci, vp, ci,
+        L.zq_w4a8_linear.argtypes = [vp, vp, vp, i64, i64, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, vp, ci, vp, ci,
                                      i64, vp, sz, vp]
         L.zq_w4a8_linear_host.restype = ci
-        L.zq_w4a8_linear_host.argtypes = [vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, ci, vp, vp, sz, vp]
+        L.zq_w4a8_linear_host.argtypes = [vp, i64, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, ci, vp, vp, sz, vp]
         L.zq_device_status.restype = ci
         L.zq_device_status.argtypes = [vp, C.POINTER(ci), vp]
         L.zq_launch_count.restype = i64
@@ -88,6 +90,10 @@ def _mode(mode) -> int:
     return MODES[mode] if isinstance(mode, str) else int(mode)
 
 
+def _layout(layout) -> int:
+    return LAYOUTS[layout] if isinstance(layout, str) else int(layout)
+
+
 def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else C.c_void_p(t.data_ptr())
 
@@ -101,9 +107,10 @@ def _check(status: int, where: str):
         raise ZqError(status, where)
 
 
-def packed_weight_sizes(N: int, K: int, group: int, mode):
+def packed_weight_sizes(N: int, K: int, group: int, mode, layout=WEIGHTS_CAST):
     a, b, c = C.c_size_t(), C.c_size_t(), C.c_size_t()
-    _check(lib().zq_packed_weight_sizes(N, K, group, _mode(mode), C.byref(a), C.byref(b), C.byref(c)),
+    _check(lib().zq_packed_weight_sizes(N, K, group, _mode(mode), _layout(layout), C.byref(a), C.byref(b),
+                                        C.byref(c)),
            "zq_packed_weight_sizes")
     return a.value, b.value, c.value
 
@@ -135,26 +142,28 @@ class PackedWeight:
     K: int
     group: int
     mode: int
+    layout: int = WEIGHTS_CAST
 
     def clone(self) -> "PackedWeight":
         return PackedWeight(self.codes.clone(), None if self.shift is None else self.shift.clone(),
-                            self.scale.clone(), self.N, self.K, self.group, self.mode)
+                            self.scale.clone(), self.N, self.K, self.group, self.mode, self.layout)
 
 
-def pack_weight_fp4(W: torch.Tensor, group: int, mode) -> PackedWeight:
-    """W: float32 [N, K] contiguous."""
+def pack_weight_fp4(W: torch.Tensor, group: int, mode, layout=WEIGHTS_CAST) -> PackedWeight:
+    """W: float32 [N, K] contiguous.  ``layout``: "cast" (the kernel casts FP4 to FP8) or "mx" (the tensor core does)."""
     assert W.dtype == torch.float32 and W.is_contiguous() and W.dim() == 2
     N, K = W.shape
     mode = _mode(mode)
-    cb, sb, fb = packed_weight_sizes(N, K, group, mode)
+    layout = _layout(layout)
+    cb, sb, fb = packed_weight_sizes(N, K, group, mode, layout)
     G = K // group
     codes = torch.empty((cb,), dtype=torch.uint8, device=W.device)
     shift = None if mode == SCALE_NONE else torch.empty((N, G), dtype=torch.uint8, device=W.device)
     scale = torch.empty((N, G) if mode == SCALE_NONE else (N,), dtype=torch.float32, device=W.device)
     assert scale.numel() * 4 == fb and (shift is None or shift.numel() == sb)
-    _check(lib().zq_pack_weight_fp4(_ptr(W), N, K, group, mode, _ptr(codes), _ptr(shift), _ptr(scale), _stream()),
-           "zq_pack_weight_fp4")
-    return PackedWeight(codes, shift, scale, N, K, group, mode)
+    _check(lib().zq_pack_weight_fp4(_ptr(W), N, K, group, mode, layout, _ptr(codes), _ptr(shift), _ptr(scale),
+                                    _stream()), "zq_pack_weight_fp4")
+    return PackedWeight(codes, shift, scale, N, K, group, mode, layout)
 
 
 def linear_workspace_bytes(M: int, N: int, K: int, r: int) -> int:
@@ -187,9 +196,9 @@ def w4a8_linear(w: PackedWeight, *, q=None, sx=None, t=None, x=None, U=None, V=N
         y = torch.empty((M, N), dtype=out_dtype, device=codes.device)
     ydt = OUT_F32 if y.dtype == torch.float32 else OUT_BF16
     ldy = y.stride(0) if M > 1 else N
-    _check(lib().zq_w4a8_linear(_ptr(q), _ptr(sx), _ptr(x), ldx, M, N, K, group, _mode(mode), _ptr(codes), _ptr(shift),
-                                _ptr(scale), _ptr(U), _ptr(V), _ptr(t), r, _ptr(y), ydt, ldy, _ptr(workspace),
-                                workspace.numel(), _stream()), "zq_w4a8_linear")
+    _check(lib().zq_w4a8_linear(_ptr(q), _ptr(sx), _ptr(x), ldx, M, N, K, group, _mode(mode), w.layout, _ptr(codes),
+                                _ptr(shift), _ptr(scale), _ptr(U), _ptr(V), _ptr(t), r, _ptr(y), ydt, ldy,
+                                _ptr(workspace), workspace.numel(), _stream()), "zq_w4a8_linear")
     return y
 
 
@@ -197,6 +206,7 @@ def w4a8_linear_noalloc(w: PackedWeight, *, q, sx, t=None, U=None, y=None, out_d
     """``zq_w4a8_linear_noalloc``: same result as :func:`w4a8_linear` on pre-quantized activations, for
     callers that cannot allocate a workspace; the scratch is a fixed array inside the library."""
     codes, shift, scale, group, mode, N, K = w.codes, w.shift, w.scale, w.group, w.mode, w.N, w.K
+    assert w.layout == WEIGHTS_CAST, "zq_w4a8_linear_noalloc takes weights in the cast layout"
     M = q.shape[0]
     r = 0 if U is None else U.shape[1]
     if y is None:
@@ -217,7 +227,7 @@ def w4a8_linear_host(x_host: torch.Tensor, y_host: torch.Tensor, w: PackedWeight
     M, K = x_host.shape
     assert K == w.K
     r = 0 if U is None else U.shape[1]
-    _check(lib().zq_w4a8_linear_host(_ptr(x_host), M, N, K, group, _mode(mode), _ptr(codes), _ptr(shift),
+    _check(lib().zq_w4a8_linear_host(_ptr(x_host), M, N, K, group, _mode(mode), w.layout, _ptr(codes), _ptr(shift),
                                      _ptr(scale), _ptr(U), _ptr(V), r, _ptr(y_host), _ptr(workspace),
                                      workspace.numel(), _stream()), "zq_w4a8_linear_host")
     return y_host

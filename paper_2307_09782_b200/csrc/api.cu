@@ -23,16 +23,22 @@ int check_device_sm100() {
 
 bool valid_mode(int mode) { return mode == ZQ_SCALE_NONE || mode == ZQ_SCALE_M1 || mode == ZQ_SCALE_M2; }
 bool valid_group(int g) { return g == 64 || g == 128 || g == 256; }
+// the tensor core's block scales are powers of two: only the constrained modes can use that layout
+bool valid_layout(int layout, int mode) {
+  return layout == ZQ_WEIGHTS_CAST || (layout == ZQ_WEIGHTS_MX && mode != ZQ_SCALE_NONE);
+}
+inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 
 // Largest split-K scratch any token count up to M can need at this (N, K), over both kernel families.
 size_t max_partial_floats(int64_t M, int64_t N, int64_t K) {
   size_t best = 0;
   const int64_t cand[6] = {16, 32, 64, 128, 256, M};
-  for (int mode = 0; mode < 2; ++mode)
+  for (int variant = 0; variant < 3; ++variant)
     for (int i = 0; i < 6; ++i) {
       const int64_t m = cand[i] < M ? cand[i] : M;
       if (m <= 0) continue;
-      const GemmPlan pl = plan_gemm(m, N, K, mode == 0 ? ZQ_SCALE_NONE : ZQ_SCALE_M1);
+      const GemmPlan pl = plan_gemm(m, N, K, variant == 0 ? ZQ_SCALE_NONE : ZQ_SCALE_M1,
+                                    variant == 2 ? ZQ_WEIGHTS_MX : ZQ_WEIGHTS_CAST);
       if (pl.partial_floats > best) best = pl.partial_floats;
     }
   return best;
@@ -99,21 +105,21 @@ int zq_quantize_act_fp8(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_
   return launch_act_quant(x, M, K, ldx, q, sx, V, V ? r : 0, t, static_cast<cudaStream_t>(stream));
 }
 
-int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, size_t* codes_bytes,
-                           size_t* shift_bytes, size_t* scale_bytes) {
-  if (!valid_mode(mode)) return ZQ_ERR_MODE;
+int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout,
+                           size_t* codes_bytes, size_t* shift_bytes, size_t* scale_bytes) {
+  if (!valid_mode(mode) || !valid_layout(layout, mode)) return ZQ_ERR_MODE;
   if (N < 0 || K <= 0 || !valid_group(group) || K % group || K % kTileK) return ZQ_ERR_SHAPE;
   const size_t G = static_cast<size_t>(K / group);
   if (codes_bytes)
-    *codes_bytes = static_cast<size_t>((N + kTileRows - 1) / kTileRows) * static_cast<size_t>(K / kTileK) * kTileBytes;
+    *codes_bytes = static_cast<size_t>((N + kTileRows - 1) / kTileRows) * static_cast<size_t>(K / kTileK) * tile_bytes(layout);
   if (shift_bytes) *shift_bytes = mode == ZQ_SCALE_NONE ? 0 : static_cast<size_t>(N) * G;
   if (scale_bytes) *scale_bytes = mode == ZQ_SCALE_NONE ? static_cast<size_t>(N) * G * 4 : static_cast<size_t>(N) * 4;
   return ZQ_OK;
 }
 
-int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale_mode mode, uint8_t* codes,
-                       uint8_t* shift, float* scale, void* stream) {
-  if (!valid_mode(mode)) return ZQ_ERR_MODE;
+int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale_mode mode,
+                       zq_weight_layout layout, uint8_t* codes, uint8_t* shift, float* scale, void* stream) {
+  if (!valid_mode(mode) || !valid_layout(layout, mode)) return ZQ_ERR_MODE;
   if (N < 0 || K <= 0 || !valid_group(group) || K % group || K % kTileK || N > 0x7FFFFFFF - kTileRows ||
       K > (int64_t(1) << 30))
     return ZQ_ERR_SHAPE;
@@ -121,7 +127,7 @@ int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale
   if (!W || !codes || !scale || (mode != ZQ_SCALE_NONE && !shift)) return ZQ_ERR_NULL;
   if (!aligned16(W) || !aligned16(codes)) return ZQ_ERR_ALIGN;
   if (int e = check_device_sm100()) return e;
-  return launch_pack_weight(W, N, K, group, mode, codes, shift, scale, static_cast<cudaStream_t>(stream));
+  return launch_pack_weight(W, N, K, group, mode, layout, codes, shift, scale, static_cast<cudaStream_t>(stream));
 }
 
 size_t zq_w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int r) {
@@ -143,10 +149,11 @@ int zq_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
 }
 
 int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M, int64_t N,
-                   int64_t K, int group, zq_scale_mode mode, const uint8_t* codes, const uint8_t* shift,
-                   const float* scale, const void* U, const void* V, const float* t, int r, void* y,
-                   zq_out_dtype ydt, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
-  if (!valid_mode(mode) || (ydt != ZQ_OUT_F32 && ydt != ZQ_OUT_BF16)) return ZQ_ERR_MODE;
+                   int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout, const uint8_t* codes,
+                   const uint8_t* shift, const float* scale, const void* U, const void* V, const float* t, int r,
+                   void* y, zq_out_dtype ydt, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!valid_mode(mode) || !valid_layout(layout, mode) || (ydt != ZQ_OUT_F32 && ydt != ZQ_OUT_BF16))
+    return ZQ_ERR_MODE;
   if (M < 0 || N < 0 || K <= 0 || K % 128 || !valid_group(group) || K % group || r < 0 || r > 64 || r % 8 ||
       ldy < N || M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > (int64_t(1) << 30))
     return ZQ_ERR_SHAPE;
@@ -159,14 +166,15 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
     return ZQ_ERR_NULL;
   }
   if (!aligned16(codes) || (q && !aligned16(q)) || (U && !aligned16(U)) || (t && !aligned16(t)) ||
-      (x_bf16 && (!aligned16(x_bf16) || ldx % 8 || (V && !aligned16(V)))))
+      (x_bf16 && (!aligned16(x_bf16) || ldx % 8 || (V && !aligned16(V)))) ||
+      (layout == ZQ_WEIGHTS_MX && !aligned32(codes)))
     return ZQ_ERR_ALIGN;
   if (!workspace) return ZQ_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) & 255u) return ZQ_ERR_ALIGN;
   const WsLayout w = ws_layout(M, N, K, r, false);
   const size_t need = x_bf16 ? w.total : w.off_q;
   if (workspace_bytes < need) return ZQ_ERR_WORKSPACE;
-  const GemmPlan pl = plan_gemm(M, N, K, mode);
+  const GemmPlan pl = plan_gemm(M, N, K, mode, layout);
   if (pl.ctas <= 0) return ZQ_ERR_SHAPE;
   if (int e = check_device_sm100()) return e;
 
@@ -190,6 +198,7 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
   a.K = K;
   a.group = group;
   a.mode = mode;
+  a.layout = layout;
   a.codes = codes;
   a.shift = shift;
   a.scale = scale;
@@ -203,11 +212,11 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
   a.counters = reinterpret_cast<int*>(ws + kWsStatusBytes);
   a.partials = reinterpret_cast<float*>(ws + w.off_partials);
   a.partial_floats = w.partial_floats;
-  return launch_w4a8_gemm(a, st);
+  return layout == ZQ_WEIGHTS_MX ? launch_w4a8_mx_gemm(a, st) : launch_w4a8_gemm(a, st);
 }
 
 int zq_w4a8_linear_host(const void* x_host, int64_t M, int64_t N, int64_t K, int group, zq_scale_mode mode,
-                        const uint8_t* codes, const uint8_t* shift, const float* scale, const void* U,
+                        zq_weight_layout layout, const uint8_t* codes, const uint8_t* shift, const float* scale, const void* U,
                         const void* V, int r, float* y_host, void* workspace, size_t workspace_bytes,
                         void* stream) {
   if (M < 0 || N < 0 || K <= 0 || r < 0) return ZQ_ERR_SHAPE;
@@ -222,7 +231,7 @@ int zq_w4a8_linear_host(const void* x_host, int64_t M, int64_t N, int64_t K, int
   float* y_dev = reinterpret_cast<float*>(ws + w.off_y);
   if (cudaMemcpyAsync(x_dev, x_host, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return ZQ_ERR_CUDA;
-  const int e = zq_w4a8_linear(nullptr, nullptr, x_dev, K, M, N, K, group, mode, codes, shift, scale, U, V, nullptr,
+  const int e = zq_w4a8_linear(nullptr, nullptr, x_dev, K, M, N, K, group, mode, layout, codes, shift, scale, U, V, nullptr,
                                r, y_dev, ZQ_OUT_F32, N, workspace, w.off_x, stream);
   if (e) return e;
   if (cudaMemcpyAsync(y_host, y_dev, static_cast<size_t>(M) * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)

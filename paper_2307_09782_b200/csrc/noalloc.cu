@@ -68,7 +68,7 @@ int zq_w4a8_linear_noalloc(const uint8_t* q, const float* sx, int64_t M, int64_t
        reinterpret_cast<uintptr_t>(t)) & 15u)
     return ZQ_ERR_ALIGN;
   // the fixed scratch bounds the split-K partial sums this problem may need
-  const GemmPlan pl = plan_gemm(M, N, K, mode);
+  const GemmPlan pl = plan_gemm(M, N, K, mode, ZQ_WEIGHTS_CAST);
   if (pl.partial_floats > kScratchPartialFloats || pl.ctas <= 0) return ZQ_ERR_WORKSPACE;
 
   void* scratch = nullptr;

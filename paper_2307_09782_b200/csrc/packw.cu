@@ -6,7 +6,8 @@
 // every group (segmented warp shuffle) and leaves the group scales in shared memory; then the
 // row-wide quantity of the constrained modes (largest exponent for M1, largest scale for M2) is
 // reduced; pass 2 re-reads the row (still in L2), divides, rounds to E2M1 and writes the codes in
-// the tiled layout the GEMM streams.  All scale decisions use the bits of the FP32 scale, never a
+// one of the two tiled layouts the GEMM kernels stream (MX = true: plain nibbles plus E8M0 block scales for
+// the tensor core's own FP4 operand).  All scale decisions use the bits of the FP32 scale, never a
 // logarithm.
 #include <limits.h>
 
@@ -38,7 +39,7 @@ __device__ __forceinline__ uint32_t e2m1_magnitude(float v) {
   return (a > 0.25f) + (a >= 0.75f) + (a > 1.25f) + (a >= 1.75f) + (a > 2.5f) + (a >= 3.5f) + (a > 5.0f);
 }
 
-template <int GROUP>
+template <int GROUP, bool MX>
 __global__ void __launch_bounds__(kThreads)
 pack_weight_kernel(const float* __restrict__ W, int N, int K, int mode, uint8_t* __restrict__ tiles,
                    uint8_t* __restrict__ shift, float* __restrict__ scale) {
@@ -50,15 +51,21 @@ pack_weight_kernel(const float* __restrict__ W, int N, int K, int mode, uint8_t*
   const int G = K / GROUP;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int kblocks = K / kTileK;
-  uint8_t* tile_row = tiles + static_cast<int64_t>(n / kTileRows) * kblocks * kTileBytes;
+  constexpr int kTB = MX ? kMxTileBytes : kTileBytes;
+  uint8_t* tile_row = tiles + static_cast<int64_t>(n / kTileRows) * kblocks * kTB;
   const int r = n % kTileRows;
 
   if (n >= N) {  // padding row of the last tile: zero codes and shifts
     for (int k = threadIdx.x * 8; k < K; k += kThreads * 8) {
-      uint8_t* blk = tile_row + static_cast<int64_t>(k / kTileK) * kTileBytes;
+      uint8_t* blk = tile_row + static_cast<int64_t>(k / kTileK) * kTB;
       const int within = k % kTileK;
-      *reinterpret_cast<uint32_t*>(blk + ((within / 32) * kTileRows + r) * 16 + ((within % 32) / 8) * 4) = 0u;
-      if (within % 64 == 0) blk[kTileCodeBytes + 2 * r + within / 64] = 0;
+      if (MX) {
+        *reinterpret_cast<uint32_t*>(blk + r * 64 + within / 2) = 0u;
+        if (within % 32 == 0) blk[kTileCodeBytes + 16 * (r % 32) + 4 * (r / 32) + within / 32] = 127;
+      } else {
+        *reinterpret_cast<uint32_t*>(blk + ((within / 32) * kTileRows + r) * 16 + ((within % 32) / 8) * 4) = 0u;
+        if (within % 64 == 0) blk[kTileCodeBytes + 2 * r + within / 64] = 0;
+      }
     }
     return;
   }
@@ -148,30 +155,43 @@ pack_weight_kernel(const float* __restrict__ W, int N, int K, int mode, uint8_t*
     for (int i = 0; i < 8; ++i) {
       w |= e2m1_magnitude(q[i]) << (4 * i);
       const uint32_t sgn = __float_as_uint(q[i]) >> 31;
-      w |= sgn << (i < 4 ? 8 * i + 7 : 8 * (i - 4) + 3);
+      w |= sgn << (MX ? 4 * i + 3 : (i < 4 ? 8 * i + 7 : 8 * (i - 4) + 3));
     }
-    uint8_t* blk = tile_row + static_cast<int64_t>(k / kTileK) * kTileBytes;
+    uint8_t* blk = tile_row + static_cast<int64_t>(k / kTileK) * kTB;
     const int within = k % kTileK;
-    *reinterpret_cast<uint32_t*>(blk + ((within / 32) * kTileRows + r) * 16 + ((within % 32) / 8) * 4) = w;
-    if (within % 64 == 0) blk[kTileCodeBytes + 2 * r + within / 64] = static_cast<uint8_t>(d);
+    if (MX) {
+      *reinterpret_cast<uint32_t*>(blk + r * 64 + within / 2) = w;
+      if (within % 32 == 0)
+        blk[kTileCodeBytes + 16 * (r % 32) + 4 * (r / 32) + within / 32] = static_cast<uint8_t>(127 - d);
+    } else {
+      *reinterpret_cast<uint32_t*>(blk + ((within / 32) * kTileRows + r) * 16 + ((within % 32) / 8) * 4) = w;
+      if (within % 64 == 0) blk[kTileCodeBytes + 2 * r + within / 64] = static_cast<uint8_t>(d);
+    }
   }
 }
 
 }  // namespace
 
-int launch_pack_weight(const float* W, int64_t N, int64_t K, int group, int mode, uint8_t* codes,
+int launch_pack_weight(const float* W, int64_t N, int64_t K, int group, int mode, int layout, uint8_t* codes,
                        uint8_t* shift, float* scale, cudaStream_t st) {
   if (N == 0) return ZQ_OK;
   const int G = static_cast<int>(K / group);
   const size_t smem = static_cast<size_t>(G) * sizeof(float);
   const int rows = static_cast<int>((N + kTileRows - 1) / kTileRows) * kTileRows;
   dim3 grid(static_cast<unsigned>(rows));
+  const bool mx = layout == ZQ_WEIGHTS_MX;
+#define ZQ_PACK(GROUP)                                                                                             \
+  if (mx)                                                                                                          \
+    pack_weight_kernel<GROUP, true><<<grid, kThreads, smem, st>>>(W, int(N), int(K), mode, codes, shift, scale);   \
+  else                                                                                                             \
+    pack_weight_kernel<GROUP, false><<<grid, kThreads, smem, st>>>(W, int(N), int(K), mode, codes, shift, scale)
   switch (group) {
-    case 64: pack_weight_kernel<64><<<grid, kThreads, smem, st>>>(W, int(N), int(K), mode, codes, shift, scale); break;
-    case 128: pack_weight_kernel<128><<<grid, kThreads, smem, st>>>(W, int(N), int(K), mode, codes, shift, scale); break;
-    case 256: pack_weight_kernel<256><<<grid, kThreads, smem, st>>>(W, int(N), int(K), mode, codes, shift, scale); break;
+    case 64: ZQ_PACK(64); break;
+    case 128: ZQ_PACK(128); break;
+    case 256: ZQ_PACK(256); break;
     default: return ZQ_ERR_SHAPE;
   }
+#undef ZQ_PACK
   count_launch();
   return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
 }

@@ -32,52 +32,12 @@
 //                and the epilogue
 // Ring depths NP and NA are multiples of NG, so a P or A stage is always handled by the same widen
 // group; that group then sees every round of the stage's barriers, which a parity wait needs.
-#include <cuda_bf16.h>
-#include <cuda_fp16.h>
-
-#include <mutex>
-
-#include "zq_common.cuh"
+#include "w4a8_gemm_shared.cuh"
 
 namespace zq {
 namespace {
 
-constexpr int kTileN = 128;   // output channels per CTA (MMA M extent)
-constexpr int kBlockK = 128;  // K elements per pipeline step
-constexpr int kAStageCols = kBlockK / 4;  // TMEM columns of one widened 128 x 128 tile (4 bytes per column)
-
-// error detail codes written to status[1]
-enum { kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6 };
-
-struct Params {
-  int M, N, K;
-  int G;             // groups per row
-  int group;
-  int kblocks;       // K blocks per output tile
-  int n_tiles, tiles;  // output tiles along N, and in total (tile index = m_tile * n_tiles + n_tile)
-  // Work is counted in units of one K block of one output tile, unit u = tile * kblocks + kb.  A CTA
-  // owns the contiguous units [u0, u1) and walks them as segments (one per output tile it touches):
-  //   stream == 0: CTA c = z * tiles + tile owns K blocks [z * kb_per_split, ...) of that tile
-  //   stream == 1: the units of all tiles are dealt out evenly, base (+1 for the first rem CTAs) each
-  int stream;
-  int atomic_y;  // streaming launch with FP32 y: CTAs that share a tile add their share into a zeroed y
-  int splits, kb_per_split;
-  int base, rem;
-  const uint8_t* codes;  // tiled weight
-  const float* scale;
-  const float* sx;
-  const __half* U;
-  const float* t;
-  int r;
-  void* y;
-  int ydt;
-  int64_t ldy;
-  int* status;
-  int* counters;
-  float* partials;
-};
-
-constexpr int cmin(int a, int b) { return a < b ? a : b; }
+using namespace gemm;
 
 template <int BM, bool NONE>
 struct Cfg {
@@ -131,117 +91,6 @@ __device__ __forceinline__ void widen8(uint32_t w, uint32_t lut_lo, uint32_t lut
   asm("prmt.b32 %0, %1, %2, %3;" : "=r"(m1) : "r"(lut_lo), "r"(lut_hi), "r"(wm >> 16));
   o0 = m0 | (w & 0x80808080u);
   o1 = m1 | ((w << 4) & 0x80808080u);
-}
-
-__device__ __forceinline__ void named_bar_sync(int id, int count) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
-}
-
-__device__ __forceinline__ void raise_error(const Params& p, volatile int* abort_flag, int detail) {
-  *abort_flag = 1;
-  if (atomicCAS(p.status, 0, ZQ_ERR_DEVICE_TIMEOUT) == 0) p.status[1] = detail;
-}
-
-__device__ __forceinline__ int range_start(const Params& p, int c) { return c * p.base + min(c, p.rem); }
-__device__ __forceinline__ int cta_of_unit(const Params& p, int u) {
-  const int big = p.rem * (p.base + 1);
-  return u < big ? u / (p.base + 1) : p.rem + (u - big) / p.base;
-}
-// The CTAs that contribute partial sums to `tile`: first CTA and their number.
-__device__ __forceinline__ void contributors(const Params& p, int tile, int* first, int* count) {
-  if (p.stream) {
-    *first = cta_of_unit(p, tile * p.kblocks);
-    *count = cta_of_unit(p, tile * p.kblocks + p.kblocks - 1) - *first + 1;
-  } else {
-    *first = 0;
-    *count = p.splits;
-  }
-}
-// Workspace slot of the partial sum that contributor j (CTA first + j) leaves for `tile`.  A streaming
-// CTA can leave two (for the tile its range starts in and for the one it ends in).
-__device__ __forceinline__ size_t partial_slot(const Params& p, int tile, int first, int j) {
-  if (!p.stream) return static_cast<size_t>(tile) * p.splits + j;
-  const int c = first + j;
-  return 2 * static_cast<size_t>(c) + (range_start(p, c) / p.kblocks == tile ? 0 : 1);
-}
-
-// Final arithmetic of NC consecutive tokens (tile columns c0 .. c0+NC-1) of one output channel, and the store.
-//   y[m, n] = sx[m] * cs * acc + sum_j t[m, j] * U[n, j]
-// s_sx holds the tile's token scales and s_tT its rank-8 LoRC rows, transposed ([j][BM]) so that two
-// neighbouring tokens' t values sit side by side: tokens are finished in pairs with packed FP32
-// instructions.  u2 holds the channel's U row, each value in both halves, when r == 8 (the common rank);
-// other ranks read t and U through the cache.
-// `add`: y was zeroed by the launcher and this CTA holds only part of the K range, so it adds (FP32 atomics,
-// order-dependent in the last bit); `lorc`: this CTA is the one that contributes the LoRC term.
-template <int NC, int BM>
-__device__ __forceinline__ void finalize(const Params& p, const float* v, int m0, int c0, int n, float cs,
-                                         const uint64_t* u2, const float* __restrict__ s_sx,
-                                         const float* __restrict__ s_tT, bool add = false, bool lorc = true) {
-  // All NC results are computed before the first store, so that the columns' loads and FMA chains
-  // interleave instead of running one column at a time behind each store.
-  static_assert(NC % 4 == 0, "columns are taken four at a time");
-  uint64_t o2[NC / 2];
-  const uint64_t cs2 = pack2(cs, cs);
-#pragma unroll
-  for (int c = 0; c < NC; c += 4) {
-    const float4 s4 = *reinterpret_cast<const float4*>(s_sx + c0 + c);
-    o2[c / 2] = mul2(mul2(pack2(s4.x, s4.y), cs2), pack2(v[c], v[c + 1]));
-    o2[c / 2 + 1] = mul2(mul2(pack2(s4.z, s4.w), cs2), pack2(v[c + 2], v[c + 3]));
-  }
-  if (lorc && p.r == 8) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-#pragma unroll
-      for (int c = 0; c < NC; c += 4) {
-        const float4 t4 = *reinterpret_cast<const float4*>(s_tT + j * BM + c0 + c);
-        o2[c / 2] = fma2(pack2(t4.x, t4.y), u2[j], o2[c / 2]);
-        o2[c / 2 + 1] = fma2(pack2(t4.z, t4.w), u2[j], o2[c / 2 + 1]);
-      }
-    }
-  }
-  float out[NC];
-#pragma unroll
-  for (int c = 0; c < NC; c += 2) unpack2(o2[c / 2], out[c], out[c + 1]);
-  if (lorc && p.r > 0 && p.r != 8) {
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      const int m = m0 + c0 + c;
-      if (m < p.M) {
-        const float* tr = p.t + static_cast<int64_t>(m) * p.r;
-        const __half* ur = p.U + static_cast<int64_t>(n) * p.r;
-        for (int j = 0; j < p.r; ++j) out[c] = fmaf(__ldg(tr + j), __half2float(__ldg(ur + j)), out[c]);
-      }
-    }
-  }
-  const int64_t base = static_cast<int64_t>(m0 + c0) * p.ldy + n;
-  if (add) {
-    float* y = static_cast<float*>(p.y) + base;
-#pragma unroll
-    for (int c = 0; c < NC; ++c)
-      if (m0 + c0 + c < p.M) atomicAdd(y + c * p.ldy, out[c]);
-  } else if (p.ydt == ZQ_OUT_F32) {
-    float* y = static_cast<float*>(p.y) + base;
-#pragma unroll
-    for (int c = 0; c < NC; ++c)
-      if (m0 + c0 + c < p.M) y[c * p.ldy] = out[c];
-  } else {
-    __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.y) + base;
-#pragma unroll
-    for (int c = 0; c < NC; ++c)
-      if (m0 + c0 + c < p.M) y[c * p.ldy] = __float2bfloat16_rn(out[c]);
-  }
-}
-
-template <int NC>
-__device__ __forceinline__ void tmem_ld_issue(uint32_t taddr, float* v) {
-  if (NC == 16) tmem_ld16(taddr, v);
-  else if (NC == 8) tmem_ld8(taddr, v);
-  else tmem_ld4(taddr, v);
-}
-template <int NC>
-__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float* v) {
-  tmem_ld_issue<NC>(taddr, v);
-  tmem_ld_wait();
 }
 
 template <int BM, bool NONE>
@@ -730,36 +579,6 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
 }
 
 // ---- host ------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* f = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(f);
-  });
-  return fn;
-}
-
-// 2-D u8 tensor [rows, row_bytes] -> tiles of box_rows x box_bytes, written to shared memory swizzled.
-bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t rows, uint32_t box_bytes,
-              uint32_t box_rows, CUtensorMapSwizzle sw) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {row_bytes, rows};
-  const cuuint64_t strides[1] = {row_bytes};
-  const cuuint32_t box[2] = {box_bytes, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 
 template <int BM, bool NONE>
 int launch_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStream_t st) {
@@ -801,8 +620,9 @@ int sm_count() {
   return n;
 }
 
-GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
+GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   GemmPlan pl{};
+  const bool mx = layout == ZQ_WEIGHTS_MX;
   const int bm_max = (mode == ZQ_SCALE_NONE) ? 64 : 256;
   int bm = 16;
   while (bm < bm_max && bm < M) bm *= 2;
@@ -811,7 +631,8 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
   pl.n_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
   const int64_t tiles = static_cast<int64_t>(pl.m_tiles) * pl.n_tiles;
   const int kblocks = static_cast<int>(K / kBlockK);
-  const int ctas_per_sm = (mode == ZQ_SCALE_NONE || bm > 128) ? 1 : (bm <= 16 ? 3 : 2);
+  // CTAs per SM the kernel family is sized for at this tile
+  const int ctas_per_sm = mx ? (bm <= 64 ? 2 : 1) : ((mode == ZQ_SCALE_NONE || bm > 128) ? 1 : (bm <= 16 ? 3 : 2));
   const int64_t resident = static_cast<int64_t>(ctas_per_sm) * sm_count();
   const int64_t units = tiles * kblocks;
   if (mode != ZQ_SCALE_NONE && bm == 16 && pl.m_tiles == 1 && tiles <= kWsMaxTiles && units >= 8 &&
@@ -853,35 +674,9 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode) {
 }
 
 int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st) {
-  const GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode);
+  const GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode, ZQ_WEIGHTS_CAST);
   if (plan.partial_floats > a.partial_floats) return ZQ_ERR_WORKSPACE;
-  Params p{};
-  p.M = static_cast<int>(a.M);
-  p.N = static_cast<int>(a.N);
-  p.K = static_cast<int>(a.K);
-  p.group = a.group;
-  p.G = static_cast<int>(a.K / a.group);
-  p.kblocks = static_cast<int>(a.K / kBlockK);
-  p.n_tiles = plan.n_tiles;
-  p.tiles = plan.n_tiles * plan.m_tiles;
-  p.stream = plan.stream;
-  p.atomic_y = (plan.stream && a.ydt == ZQ_OUT_F32 && plan.partial_floats > 0) ? 1 : 0;
-  p.splits = plan.splits;
-  p.kb_per_split = plan.kb_per_split;
-  p.base = plan.base;
-  p.rem = plan.rem;
-  p.codes = a.codes;
-  p.scale = a.scale;
-  p.sx = a.sx;
-  p.U = static_cast<const __half*>(a.U);
-  p.t = a.t;
-  p.r = a.U ? a.r : 0;
-  p.y = a.y;
-  p.ydt = a.ydt;
-  p.ldy = a.ldy;
-  p.status = a.status;
-  p.counters = a.counters;
-  p.partials = a.partials;
+  const Params p = make_params(a, plan);
   const bool none = a.mode == ZQ_SCALE_NONE;
   switch (plan.bm) {
     case 16: return none ? launch_cfg<16, true>(a, plan, p, st) : launch_cfg<16, false>(a, plan, p, st);

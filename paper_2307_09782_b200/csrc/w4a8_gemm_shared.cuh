@@ -1,0 +1,232 @@
+// Pieces shared by the two W4A8 GEMM kernel families (the one that casts FP4 to FP8 on the CUDA cores and
+// the one that hands FP4 tiles and power-of-two block scales to the tensor core): work partition, the
+// split-K hand-over, the epilogue arithmetic of Section 3 (token scale x channel scale x accumulator plus
+// the LoRC term) and the tensor-map helper.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <mutex>
+
+#include "zq_common.cuh"
+
+namespace zq {
+namespace gemm {
+
+constexpr int kTileN = 128;   // output channels per CTA (MMA M extent)
+constexpr int kBlockK = 128;  // K elements per pipeline step
+constexpr int kAStageCols = kBlockK / 4;  // TMEM columns of one widened 128 x 128 tile (4 bytes per column)
+
+// error detail codes written to status[1]
+enum { kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6 };
+
+struct Params {
+  int M, N, K;
+  int G;             // groups per row
+  int group;
+  int kblocks;       // K blocks per output tile
+  int n_tiles, tiles;  // output tiles along N, and in total (tile index = m_tile * n_tiles + n_tile)
+  // Work is counted in units of one K block of one output tile, unit u = tile * kblocks + kb.  A CTA
+  // owns the contiguous units [u0, u1) and walks them as segments (one per output tile it touches):
+  //   stream == 0: CTA c = z * tiles + tile owns K blocks [z * kb_per_split, ...) of that tile
+  //   stream == 1: the units of all tiles are dealt out evenly, base (+1 for the first rem CTAs) each
+  int stream;
+  int atomic_y;  // streaming launch with FP32 y: CTAs that share a tile add their share into a zeroed y
+  int splits, kb_per_split;
+  int base, rem;
+  const uint8_t* codes;  // tiled weight
+  const float* scale;
+  const float* sx;
+  const __half* U;
+  const float* t;
+  int r;
+  void* y;
+  int ydt;
+  int64_t ldy;
+  int* status;
+  int* counters;
+  float* partials;
+};
+
+constexpr int cmin(int a, int b) { return a < b ? a : b; }
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void raise_error(const Params& p, volatile int* abort_flag, int detail) {
+  *abort_flag = 1;
+  if (atomicCAS(p.status, 0, ZQ_ERR_DEVICE_TIMEOUT) == 0) p.status[1] = detail;
+}
+
+__device__ __forceinline__ int range_start(const Params& p, int c) { return c * p.base + min(c, p.rem); }
+__device__ __forceinline__ int cta_of_unit(const Params& p, int u) {
+  const int big = p.rem * (p.base + 1);
+  return u < big ? u / (p.base + 1) : p.rem + (u - big) / p.base;
+}
+// The CTAs that contribute partial sums to `tile`: first CTA and their number.
+__device__ __forceinline__ void contributors(const Params& p, int tile, int* first, int* count) {
+  if (p.stream) {
+    *first = cta_of_unit(p, tile * p.kblocks);
+    *count = cta_of_unit(p, tile * p.kblocks + p.kblocks - 1) - *first + 1;
+  } else {
+    *first = 0;
+    *count = p.splits;
+  }
+}
+// Workspace slot of the partial sum that contributor j (CTA first + j) leaves for `tile`.  A streaming
+// CTA can leave two (for the tile its range starts in and for the one it ends in).
+__device__ __forceinline__ size_t partial_slot(const Params& p, int tile, int first, int j) {
+  if (!p.stream) return static_cast<size_t>(tile) * p.splits + j;
+  const int c = first + j;
+  return 2 * static_cast<size_t>(c) + (range_start(p, c) / p.kblocks == tile ? 0 : 1);
+}
+
+// Final arithmetic of NC consecutive tokens (tile columns c0 .. c0+NC-1) of one output channel, and the store.
+//   y[m, n] = sx[m] * cs * acc + sum_j t[m, j] * U[n, j]
+// s_sx holds the tile's token scales and s_tT its rank-8 LoRC rows, transposed ([j][BM]) so that two
+// neighbouring tokens' t values sit side by side: tokens are finished in pairs with packed FP32
+// instructions.  u2 holds the channel's U row, each value in both halves, when r == 8 (the common rank);
+// other ranks read t and U through the cache.
+// `add`: y was zeroed by the launcher and this CTA holds only part of the K range, so it adds (FP32 atomics,
+// order-dependent in the last bit); `lorc`: this CTA is the one that contributes the LoRC term.
+template <int NC, int BM>
+__device__ __forceinline__ void finalize(const Params& p, const float* v, int m0, int c0, int n, float cs,
+                                         const uint64_t* u2, const float* __restrict__ s_sx,
+                                         const float* __restrict__ s_tT, bool add = false, bool lorc = true) {
+  // All NC results are computed before the first store, so that the columns' loads and FMA chains
+  // interleave instead of running one column at a time behind each store.
+  static_assert(NC % 4 == 0, "columns are taken four at a time");
+  uint64_t o2[NC / 2];
+  const uint64_t cs2 = pack2(cs, cs);
+#pragma unroll
+  for (int c = 0; c < NC; c += 4) {
+    const float4 s4 = *reinterpret_cast<const float4*>(s_sx + c0 + c);
+    o2[c / 2] = mul2(mul2(pack2(s4.x, s4.y), cs2), pack2(v[c], v[c + 1]));
+    o2[c / 2 + 1] = mul2(mul2(pack2(s4.z, s4.w), cs2), pack2(v[c + 2], v[c + 3]));
+  }
+  if (lorc && p.r == 8) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+#pragma unroll
+      for (int c = 0; c < NC; c += 4) {
+        const float4 t4 = *reinterpret_cast<const float4*>(s_tT + j * BM + c0 + c);
+        o2[c / 2] = fma2(pack2(t4.x, t4.y), u2[j], o2[c / 2]);
+        o2[c / 2 + 1] = fma2(pack2(t4.z, t4.w), u2[j], o2[c / 2 + 1]);
+      }
+    }
+  }
+  float out[NC];
+#pragma unroll
+  for (int c = 0; c < NC; c += 2) unpack2(o2[c / 2], out[c], out[c + 1]);
+  if (lorc && p.r > 0 && p.r != 8) {
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      const int m = m0 + c0 + c;
+      if (m < p.M) {
+        const float* tr = p.t + static_cast<int64_t>(m) * p.r;
+        const __half* ur = p.U + static_cast<int64_t>(n) * p.r;
+        for (int j = 0; j < p.r; ++j) out[c] = fmaf(__ldg(tr + j), __half2float(__ldg(ur + j)), out[c]);
+      }
+    }
+  }
+  const int64_t base = static_cast<int64_t>(m0 + c0) * p.ldy + n;
+  if (add) {
+    float* y = static_cast<float*>(p.y) + base;
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+      if (m0 + c0 + c < p.M) atomicAdd(y + c * p.ldy, out[c]);
+  } else if (p.ydt == ZQ_OUT_F32) {
+    float* y = static_cast<float*>(p.y) + base;
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+      if (m0 + c0 + c < p.M) y[c * p.ldy] = out[c];
+  } else {
+    __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.y) + base;
+#pragma unroll
+    for (int c = 0; c < NC; ++c)
+      if (m0 + c0 + c < p.M) y[c * p.ldy] = __float2bfloat16_rn(out[c]);
+  }
+}
+
+template <int NC>
+__device__ __forceinline__ void tmem_ld_issue(uint32_t taddr, float* v) {
+  if (NC == 16) tmem_ld16(taddr, v);
+  else if (NC == 8) tmem_ld8(taddr, v);
+  else tmem_ld4(taddr, v);
+}
+template <int NC>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, float* v) {
+  tmem_ld_issue<NC>(taddr, v);
+  tmem_ld_wait();
+}
+
+#endif  // __CUDACC__
+
+// ---- host ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(f);
+  });
+  return fn;
+}
+
+// 2-D u8 tensor [rows, row_bytes] -> tiles of box_rows x box_bytes, written to shared memory swizzled.
+inline bool make_map(CUtensorMap* m, const void* base, uint64_t row_bytes, uint64_t rows, uint32_t box_bytes,
+              uint32_t box_rows, CUtensorMapSwizzle sw) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {row_bytes, rows};
+  const cuuint64_t strides[1] = {row_bytes};
+  const cuuint32_t box[2] = {box_bytes, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline Params make_params(const GemmArgs& a, const GemmPlan& plan) {
+  Params p{};
+  p.M = static_cast<int>(a.M);
+  p.N = static_cast<int>(a.N);
+  p.K = static_cast<int>(a.K);
+  p.group = a.group;
+  p.G = static_cast<int>(a.K / a.group);
+  p.kblocks = static_cast<int>(a.K / kBlockK);
+  p.n_tiles = plan.n_tiles;
+  p.tiles = plan.n_tiles * plan.m_tiles;
+  p.stream = plan.stream;
+  p.atomic_y = (plan.stream && a.ydt == ZQ_OUT_F32 && plan.partial_floats > 0) ? 1 : 0;
+  p.splits = plan.splits;
+  p.kb_per_split = plan.kb_per_split;
+  p.base = plan.base;
+  p.rem = plan.rem;
+  p.codes = a.codes;
+  p.scale = a.scale;
+  p.sx = a.sx;
+  p.U = static_cast<const __half*>(a.U);
+  p.t = a.t;
+  p.r = a.U ? a.r : 0;
+  p.y = a.y;
+  p.ydt = a.ydt;
+  p.ldy = a.ldy;
+  p.status = a.status;
+  p.counters = a.counters;
+  p.partials = a.partials;
+  return p;
+}
+
+}  // namespace gemm
+}  // namespace zq

@@ -1,0 +1,439 @@
+// W4A8 GEMM with the cast FP4 -> FP8 left to the tensor core:
+//   y = sx * scale * (Q_fp8(x) . (E2M1 codes * 2^-shift)^T) + t U^T                      (Section 3)
+//
+// Section 3 ("Casting the FP4 to FP8") constrains the group scales to powers of two (M1) or to
+// power-of-two fractions of a per-channel scale (M2) so that FP4 weights reach the FP8 tensor core
+// with a bit shift instead of a multiplication.  This architecture's tensor core takes that step itself: its
+// block-scaled MMA (kind::mxf8f6f4) multiplies an E2M1 operand by an E4M3 operand and applies one
+// power-of-two (E8M0) scale per row and 32 elements of K, which is exactly the constrained group
+// scale 2^-shift.  The kernel therefore moves bytes and issues MMAs; no CUDA core touches a weight.
+//
+//   weights  one TMA load per K block brings a 128 x 128 tile of packed nibbles (8 KB, contiguous in
+//            HBM) into shared memory, expanded by the copy engine to the tensor core's 16-byte-aligned
+//            FP4 form (8 bytes of nibbles, 8 bytes of padding);
+//   scales   the tile's 512 E8M0 bytes follow it in HBM, arrive by a bulk copy and go to tensor memory
+//            with tcgen05.cp, issued by the MMA thread right before the tile's four MMAs;
+//   tokens   E4M3 tiles by TMA, the shared-memory B operand, with a block scale of one;
+//   D        FP32 in tensor memory, two buffers where they fit, so that the epilogue of one output tile
+//            overlaps the main loop of the next.
+//
+// Orientation, work partition (units of one K block of one output tile, dealt out as contiguous ranges
+// or as split-K), the split-K hand-over and the epilogue are those of the casting kernel.
+//
+// Warp roles: 0..3 epilogue (one TMEM lane quarter each), 4 producer (one lane issues all copies of a
+// stage onto one barrier), 5 TMEM allocation and MMA issue.
+#include "w4a8_gemm_shared.cuh"
+
+namespace zq {
+namespace {
+
+using namespace gemm;
+
+constexpr int kSfbCols = 16;  // token-side block scales (all one): room for 256 tokens, written once
+
+template <int BM>
+struct MxCfg {
+  static constexpr int kMinBlocks = BM <= 64 ? 2 : 1;  // CTAs per SM this configuration is sized for
+  static constexpr int kProducerWarp = 4;
+  static constexpr int kMmaWarp = 5;
+  static constexpr int kThreads = 192;
+  static constexpr int kEpiThreads = 128;
+  static constexpr int kABytes = kTileRows * kTileK;  // shared-memory footprint of a code tile (padded FP4)
+  static constexpr int kTokBytes = BM * kBlockK;
+  static constexpr int kStageTx = kTileCodeBytes + kMxTileScaleBytes + kTokBytes;  // bytes a stage's barrier counts
+  static constexpr int kBudget = (kMinBlocks == 1 ? 220 : 110) * 1024 - BM * 36 - 512;
+  static constexpr int NS = cmin(12, kBudget / (kABytes + kMxTileScaleBytes + kTokBytes));
+  static constexpr int NB = BM <= 128 ? 2 : 1;  // accumulator buffers
+  static constexpr int kDColsPad = BM < 32 ? 32 : BM;
+  static constexpr int kSfaCol0 = NB * kDColsPad;
+  static constexpr int kSfbCol0 = kSfaCol0 + 4 * NS;
+  static constexpr int kColsUsed = kSfbCol0 + kSfbCols;
+  static constexpr int kTmemCols = kColsUsed <= 128 ? 128 : (kColsUsed <= 256 ? 256 : 512);
+  // shared memory map (offsets from a 1024-byte aligned base)
+  static constexpr int offA = 0;
+  static constexpr int offTok = offA + NS * kABytes;
+  static constexpr int offSf = offTok + NS * kTokBytes;
+  static constexpr int offSx = offSf + NS * kMxTileScaleBytes;  // [BM] token scales
+  static constexpr int offT = offSx + BM * 4;                   // [8][BM] LoRC down-projection (rank 8)
+  static constexpr int offBars = offT + BM * 32;
+  static constexpr int kNumBars = 2 * NS + 2 * NB + 1;
+  static constexpr int offMisc = offBars + kNumBars * 8;
+  static constexpr int kSmemBytes = offMisc + 32;
+  static_assert(NS >= 3, "pipeline depth");
+  static_assert(kTmemCols * kMinBlocks <= 512, "tensor memory");
+  static_assert(kSmemBytes * kMinBlocks <= 226 * 1024, "shared memory");
+};
+
+template <int BM>
+__global__ void __launch_bounds__(MxCfg<BM>::kThreads, MxCfg<BM>::kMinBlocks)
+w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
+                    const Params p) {
+  using C = MxCfg<BM>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint8_t* s_a = smem + C::offA;
+  uint8_t* s_tok = smem + C::offTok;
+  uint8_t* s_sf = smem + C::offSf;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offBars);
+  uint64_t* full = bars;                  // [NS] all three copies of the stage landed   (MMA waits)
+  uint64_t* empty = full + C::NS;         // [NS] the MMAs that read the stage are done   (producer waits)
+  uint64_t* acc_full = empty + C::NS;     // [NB] a segment's accumulation is complete    (epilogue waits)
+  uint64_t* acc_empty = acc_full + C::NB; // [NB] the epilogue has read the buffer        (MMA waits)
+  uint64_t* drain_bar = acc_empty + C::NB;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::offMisc);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::offMisc + 4);
+  int* s_last = reinterpret_cast<int*>(smem + C::offMisc + 8);
+  float* s_sx = reinterpret_cast<float*>(smem + C::offSx);
+  float* s_t = reinterpret_cast<float*>(smem + C::offT);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // this CTA's units [u0, u1)
+  int u0, u1;
+  if (p.stream) {
+    u0 = range_start(p, blockIdx.x);
+    u1 = range_start(p, blockIdx.x + 1);
+  } else {
+    const int z = blockIdx.x / p.tiles, tile = blockIdx.x % p.tiles;
+    u0 = tile * p.kblocks + z * p.kb_per_split;
+    u1 = min(u0 + p.kb_per_split, (tile + 1) * p.kblocks);
+  }
+  const int nunits = u1 - u0;
+  // all of a CTA's tiles share one token tile (streaming is only used with a single row of tiles)
+  const int m0 = ((u0 / p.kblocks) / p.n_tiles) * BM;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < C::NS; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
+    }
+    for (int i = 0; i < C::NB; ++i) {
+      mbar_init(&acc_full[i], 1);
+      mbar_init(&acc_empty[i], 4);  // one arrival per epilogue warp
+    }
+    mbar_init(drain_bar, 1);
+    *s_abort = 0;
+    *s_last = 0;
+    fence_mbar_init();
+    if ((smem_u32(smem) & 1023u) != 0) raise_error(p, s_abort, kErrAlign);
+  }
+  if (warp == C::kProducerWarp && lane == 0) {
+    prefetch_tensormap(&tm_w);
+    prefetch_tensormap(&tm_q);
+  }
+  if (warp < 4) {
+    // token scales and (rank 8) LoRC rows of this CTA's tokens, for the epilogue
+    for (int c = threadIdx.x; c < BM; c += 128) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
+    if (p.r == 8)
+      for (int c = threadIdx.x; c < BM * 8; c += 128)  // transposed: [j][BM]
+        s_t[(c & 7) * BM + (c >> 3)] = (m0 + (c >> 3) < p.M) ? __ldg(p.t + static_cast<int64_t>(m0) * 8 + c) : 0.0f;
+  }
+  if (warp == C::kMmaWarp) tmem_alloc(s_tmem, C::kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *s_tmem;
+  const uint32_t tmem_sfa = tmem_base + C::kSfaCol0;
+  const uint32_t tmem_sfb = tmem_base + C::kSfbCol0;
+  const bool ok_start = (*s_abort == 0);
+  if (warp < 4) {
+    // the tokens' block scales are all 2^0: fill their columns once (every lane quarter holds a copy)
+    uint32_t ones[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) ones[i] = 0x7F7F7F7Fu;
+    tmem_st16(tmem_sfb + (static_cast<uint32_t>(warp * 32) << 16), ones);
+    tmem_st_wait();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+
+  if (warp == C::kProducerWarp) {
+    // ------------------------------------------------------------------ producer
+    if (ok_start) {  // warp-uniform loop, one elected lane issues the copies
+      const bool issuer = elect_one();
+      int s = 0, issued = 0;
+      uint32_t ph = 0;
+      int tile = u0 / p.kblocks, kb = u0 % p.kblocks;
+      for (int i = 0; i < nunits; ++i) {
+        if (!mbar_wait(&empty[s], ph ^ 1, s_abort)) {
+          if (issuer) raise_error(p, s_abort, kErrProducer);
+          break;
+        }
+        if (issuer) {
+          const int wt = (tile % p.n_tiles) * p.kblocks + kb;  // index of the weight tile
+          mbar_arrive_expect_tx(&full[s], C::kStageTx);
+          tma_load_3d(s_a + s * C::kABytes, &tm_w, 0, 0, wt, &full[s]);
+          bulk_load(s_sf + s * kMxTileScaleBytes, p.codes + static_cast<int64_t>(wt) * kMxTileBytes + kTileCodeBytes,
+                    kMxTileScaleBytes, &full[s]);
+          tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, kb * kBlockK, m0, &full[s]);
+        }
+        __syncwarp();
+        issued = i + 1;
+        if (++kb == p.kblocks) {
+          kb = 0;
+          ++tile;
+        }
+        if (++s == C::NS) {
+          s = 0;
+          ph ^= 1;
+        }
+      }
+      // never leave with copies still in flight: wait (bounded) for the last phase issued per stage
+      for (int i = max(0, issued - C::NS); i < issued; ++i) {
+        uint32_t spin = 0;
+        while (!mbar_try_wait(&full[i % C::NS], (i / C::NS) & 1) && ++spin < kSpinLimit) {
+        }
+      }
+    }
+  } else if (warp == C::kMmaWarp) {
+    // ------------------------------------------------------------------ MMA issuer
+    // The whole warp runs the loop (uniform control flow and addresses); one elected lane issues.
+    if (ok_start) {
+      const bool issuer = elect_one();
+      const uint64_t adesc0 = umma_desc_k128(smem_u32(s_a));
+      const uint64_t bdesc0 = umma_desc_k128(smem_u32(s_tok));
+      const uint64_t sfdesc0 = umma_desc_rows16(smem_u32(s_sf), 128);
+      int s = 0;
+      uint32_t ph = 0;
+      int kb = u0 % p.kblocks, seg = 0;
+      bool seg_first = true;  // the next K block starts a segment (a new accumulation)
+      bool failed = false;
+      for (int i = 0; i < nunits && !failed; ++i) {
+        if (!mbar_wait(&full[s], ph, s_abort)) {
+          failed = true;
+          break;
+        }
+        const int buf = seg % C::NB;
+        if (seg_first && seg >= C::NB) {
+          // the epilogue of the segment that used this buffer last must have read it
+          if (!mbar_wait(&acc_empty[buf], ((seg / C::NB) - 1) & 1, s_abort)) {
+            failed = true;
+            break;
+          }
+        }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + buf * C::kDColsPad;
+        const uint32_t sfa = tmem_sfa + 4 * s;
+        const uint64_t adesc = adesc0 + static_cast<uint64_t>((s * C::kABytes) >> 4);
+        const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((s * C::kTokBytes) >> 4);
+        if (issuer) {
+          tmem_cp_32x128b_x4(sfa, sfdesc0 + static_cast<uint64_t>((s * kMxTileScaleBytes) >> 4));
+#pragma unroll
+          for (int k = 0; k < kBlockK / 32; ++k) {
+            // scale byte k of the stage's four columns belongs to elements 32k .. 32k+31
+            umma_mxf8f6f4(d_tmem, adesc + 2 * k, bdesc + 2 * k, umma_idesc_mx_e2m1_e4m3(BM, k, 0),
+                          sfa + (static_cast<uint32_t>(k) << 30), tmem_sfb, (!seg_first || k > 0) ? 1u : 0u);
+          }
+        }
+        const bool seg_last = (kb + 1 == p.kblocks) || (i + 1 == nunits);
+        if (issuer) {
+          umma_commit(&empty[s]);
+          if (seg_last) umma_commit(&acc_full[buf]);
+        }
+        __syncwarp();
+        seg_first = seg_last;
+        if (seg_last) ++seg;
+        if (++kb == p.kblocks) kb = 0;
+        if (++s == C::NS) {
+          s = 0;
+          ph ^= 1;
+        }
+      }
+      if (failed) {
+        if (issuer) {
+          raise_error(p, s_abort, kErrMma);
+          umma_commit(drain_bar);  // let the MMAs already issued finish before TMEM is released
+        }
+        uint32_t spin = 0;
+        while (!mbar_try_wait(drain_bar, 0) && ++spin < kSpinLimit) {
+        }
+      }
+      __syncwarp();
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int row = warp * 32 + lane;  // output channel within the tile = TMEM lane
+    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    constexpr int EC = BM <= 32 ? 4 : (BM <= 128 ? 8 : 16);  // columns per step
+    bool failed = !ok_start;
+
+    // Every thread walks every segment and executes the same named-barrier sequence whether or not it
+    // has failed, so a bounded wait that ran out can never leave others stuck at a hardware barrier.
+    int seg = 0;
+    for (int us = u0; us < u1; ++seg) {
+      const int tile = us / p.kblocks;
+      const int ue = min(u1, (tile + 1) * p.kblocks);
+      const int n = (tile % p.n_tiles) * kTileN + row;
+      const bool n_ok = n < p.N;
+      const int buf = seg % C::NB;
+      const uint32_t t_lane = tmem_base + buf * C::kDColsPad + lane_base;
+
+      float cs = 1.0f;
+      uint64_t u[8];  // the channel's U row, each value in both halves of a packed pair
+#pragma unroll
+      for (int e = 0; e < 8; ++e) u[e] = 0ull;
+      if (n_ok) cs = __ldg(p.scale + n);
+      if (p.r == 8 && n_ok) {
+        const uint4 h = __ldg(reinterpret_cast<const uint4*>(p.U + static_cast<int64_t>(n) * 8));
+        const uint32_t hw[4] = {h.x, h.y, h.z, h.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __half2 h2;
+          *reinterpret_cast<uint32_t*>(&h2) = hw[e];
+          const float2 f = __half22float2(h2);
+          u[2 * e] = pack2(f.x, f.x);
+          u[2 * e + 1] = pack2(f.y, f.y);
+        }
+      }
+      if (!failed) {
+        if (!mbar_wait_warp(&acc_full[buf], (seg / C::NB) & 1, s_abort)) {
+          raise_error(p, s_abort, kErrEpilogue);
+          failed = true;
+        }
+        tc_fence_after_sync();
+      }
+
+      const bool whole_tile = (ue - us) == p.kblocks;
+      if (whole_tile) {
+        if (!failed) {
+          // the next step's accumulator columns are in flight while this step's are finished
+          float nxt[EC];
+          tmem_ld_issue<EC>(t_lane, nxt);
+#pragma unroll 1
+          for (int c = 0; c < BM; c += EC) {
+            float v[EC];
+            tmem_ld_wait_regs<EC>(nxt);
+#pragma unroll
+            for (int e = 0; e < EC; ++e) v[e] = nxt[e];
+            if (c + EC < BM) tmem_ld_issue<EC>(t_lane + c + EC, nxt);
+            if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t);
+          }
+        }
+      } else if (p.atomic_y) {
+        // Several CTAs share this tile and y was zeroed before the launch: every CTA scales its share
+        // and adds it; the first contributor also adds the LoRC term.  No fence, ticket or second pass.
+        int first, count;
+        contributors(p, tile, &first, &count);
+        const bool lorc = static_cast<int>(blockIdx.x) == first;
+        if (!failed) {
+#pragma unroll 1
+          for (int c = 0; c < BM; c += EC) {
+            float v[EC];
+            tmem_ld_cols<EC>(t_lane + c, v);
+            if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t, true, lorc);
+          }
+        }
+      } else {
+        // Several CTAs share this tile: leave the raw partial sums in the workspace; the CTA that
+        // arrives last adds all of them in contributor order (deterministic) and finishes the tile.
+        int first, count;
+        contributors(p, tile, &first, &count);
+        const int my_j = p.stream ? static_cast<int>(blockIdx.x) - first : static_cast<int>(blockIdx.x) / p.tiles;
+        float* my_partial = p.partials + partial_slot(p, tile, first, my_j) * (BM * kTileN);
+        if (!failed) {
+#pragma unroll 1
+          for (int c = 0; c < BM; c += EC) {
+            float v[EC];
+            tmem_ld_cols<EC>(t_lane + c, v);
+#pragma unroll
+            for (int e = 0; e < EC; ++e) my_partial[(c + e) * kTileN + row] = v[e];
+          }
+        }
+        __threadfence();
+        named_bar_sync(1, C::kEpiThreads);
+        if (threadIdx.x == 0) {
+          const int ticket = (*s_abort) ? -1 : atomicAdd(p.counters + tile, 1);
+          *s_last = (ticket == count - 1) ? 1 : 0;
+          if (ticket == count - 1) p.counters[tile] = 0;  // ready for the next call
+        }
+        named_bar_sync(1, C::kEpiThreads);
+        if (*s_last) {
+          __threadfence();
+#pragma unroll 1
+          for (int c = 0; c < BM; c += EC) {
+            float v[EC];
+#pragma unroll
+            for (int e = 0; e < EC; ++e) v[e] = 0.0f;
+            for (int j = 0; j < count; ++j) {
+              const float* src = p.partials + partial_slot(p, tile, first, j) * (BM * kTileN) + c * kTileN + row;
+#pragma unroll
+              for (int e = 0; e < EC; ++e) v[e] += __ldcg(src + e * kTileN);
+            }
+            if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t);
+          }
+        }
+        named_bar_sync(1, C::kEpiThreads);  // s_last is reused by the next segment
+      }
+      // the accumulator buffer has been read: the MMA warp may reuse it
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[buf]);
+      us = ue;
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == C::kMmaWarp) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, C::kTmemCols);
+  }
+}
+
+// ---- host ------------------------------------------------------------------------------------------
+// The packed weight as a 3-D tensor of 4-bit elements [tiles][128 rows][128 elements]; the copy engine
+// expands a 128 x 128 box to the 16-byte-aligned FP4 form in shared memory, 128-byte swizzled.
+bool make_weight_map(CUtensorMap* m, const void* base, uint64_t tiles) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {kTileK, kTileRows, tiles};
+  const cuuint64_t strides[2] = {kTileK / 2, kMxTileBytes};
+  const cuuint32_t box[3] = {kTileK, kTileRows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BM>
+int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStream_t st) {
+  using C = MxCfg<BM>;
+  CUtensorMap tm_w, tm_q;
+  if (!make_weight_map(&tm_w, a.codes, static_cast<uint64_t>(plan.n_tiles) * static_cast<uint64_t>(p.kblocks)) ||
+      !make_map(&tm_q, a.q, static_cast<uint64_t>(a.K), static_cast<uint64_t>(a.M), kBlockK, BM,
+                CU_TENSOR_MAP_SWIZZLE_128B))
+    return ZQ_ERR_CUDA;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] {
+    attr_err = cudaFuncSetAttribute(w4a8_mx_gemm_kernel<BM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    C::kSmemBytes);
+  });
+  if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
+  if (p.atomic_y &&
+      cudaMemset2DAsync(a.y, static_cast<size_t>(a.ldy) * 4, 0, static_cast<size_t>(a.N) * 4, static_cast<size_t>(a.M),
+                        st) != cudaSuccess)
+    return ZQ_ERR_CUDA;
+  dim3 grid(static_cast<unsigned>(plan.ctas));
+  w4a8_mx_gemm_kernel<BM><<<grid, C::kThreads, C::kSmemBytes, st>>>(tm_w, tm_q, p);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
+  if (a.mode == ZQ_SCALE_NONE) return ZQ_ERR_MODE;
+  const GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode, ZQ_WEIGHTS_MX);
+  if (plan.partial_floats > a.partial_floats) return ZQ_ERR_WORKSPACE;
+  const Params p = make_params(a, plan);
+  switch (plan.bm) {
+    case 16: return launch_mx_cfg<16>(a, plan, p, st);
+    case 32: return launch_mx_cfg<32>(a, plan, p, st);
+    case 64: return launch_mx_cfg<64>(a, plan, p, st);
+    case 128: return launch_mx_cfg<128>(a, plan, p, st);
+    case 256: return launch_mx_cfg<256>(a, plan, p, st);
+  }
+  return ZQ_ERR_SHAPE;
+}
+
+}  // namespace zq

@@ -35,10 +35,21 @@ constexpr int kTileCodeBytes = kTileRows * kTileK / 2;
 constexpr int kTileShiftBytes = 2 * kTileRows;
 constexpr int kTileBytes = kTileCodeBytes + kTileShiftBytes;
 
+// Tiles for the tensor core's own FP4 operand (layout ZQ_WEIGHTS_MX, modes M1 / M2).  Same tiling and tile
+// order; a tile holds
+//   [0, 8192)    codes, row-major: row r at r * 64, element k of the K block in byte k / 2 (even k in the low
+//                nibble), a nibble being the plain E2M1 code (sign in bit 3)
+//   [8192, 8704) block scales, one E8M0 byte 127 - shift per row and 32 elements, in the order the tensor
+//                memory copy wants: byte 16 * (r % 32) + 4 * (r / 32) + s for row r, elements 32s .. 32s+31
+constexpr int kMxTileScaleBytes = 4 * kTileRows;
+constexpr int kMxTileBytes = kTileCodeBytes + kMxTileScaleBytes;
+
+inline size_t tile_bytes(int layout) { return layout == ZQ_WEIGHTS_MX ? kMxTileBytes : kTileBytes; }
+
 // ---- launchers implemented in the .cu files ------------------------------------------------------
 int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
                      const void* V, int r, float* t, cudaStream_t st);
-int launch_pack_weight(const float* W, int64_t N, int64_t K, int group, int mode, uint8_t* codes,
+int launch_pack_weight(const float* W, int64_t N, int64_t K, int group, int mode, int layout, uint8_t* codes,
                        uint8_t* shift, float* scale, cudaStream_t st);
 
 struct GemmArgs {
@@ -46,6 +57,7 @@ struct GemmArgs {
   const float* sx;       // [M]
   int64_t M, N, K;
   int group, mode;
+  int layout;            // ZQ_WEIGHTS_CAST or ZQ_WEIGHTS_MX
   const uint8_t* codes;  // tiled, see above
   const uint8_t* shift;  // [N, G] or NULL (not read by the GEMM: the tiles carry the shifts)
   const float* scale;    // [N] or [N, G]
@@ -71,8 +83,10 @@ struct GemmPlan {
   int base, rem;     // stream == 1: units per CTA (the first `rem` CTAs take one more)
   size_t partial_floats;
 };
-GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode);
-int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st);
+GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout);
+int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st);           // ZQ_WEIGHTS_CAST
+int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st);        // ZQ_WEIGHTS_MX
+int sm_count();
 
 #ifdef __CUDACC__
 // ---- device: bounded waits -----------------------------------------------------------------------
@@ -181,6 +195,15 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
       : "memory");
 }
 
+// The same for a 3-D tensor map (c0 innermost).
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m, int c0, int c1, int c2,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
 // Contiguous global -> shared copy of `bytes` (multiple of 16, both addresses 16-byte aligned).
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -223,6 +246,23 @@ __device__ __forceinline__ void umma_f8_tmem_a(uint32_t d_tmem, uint32_t a_tmem,
       "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], [%1], %2, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
+}
+// Block-scaled form: A and B are MX operands (here E2M1 x E4M3) whose 32-element blocks along K are
+// multiplied by the power-of-two (E8M0) scales found in tensor memory at sfa / sfb.
+__device__ __forceinline__ void umma_mxf8f6f4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                              uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%4], [%5], p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem), "r"(accumulate)
+      : "memory");
+}
+// Shared memory -> tensor memory: 32 rows of 16 bytes (described by `sdesc`) land in lanes 0..31 of four
+// consecutive columns and are repeated in the other three lane quarters.  Runs in order with the MMAs
+// issued by the same thread.
+__device__ __forceinline__ void tmem_cp_32x128b_x4(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 // Arrive once on `bar` when every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
@@ -317,6 +357,20 @@ __device__ __forceinline__ uint64_t umma_desc_k128(uint32_t smem_addr) {
   d |= uint64_t(1) << 46;                    // descriptor version of this architecture
   d |= uint64_t(2) << 61;                    // 128-byte swizzle
   return d;
+}
+// Shared-memory descriptor without swizzle: rows of 16 bytes, 8-row groups `group_stride` bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_rows16(uint32_t smem_addr, uint32_t group_stride) {
+  uint64_t d = 0;
+  d |= uint64_t((smem_addr >> 4) & 0x3FFF);
+  d |= uint64_t(group_stride >> 4) << 32;
+  d |= uint64_t(1) << 46;
+  return d;
+}
+// Instruction descriptor of the block-scaled MMA: A = E2M1, B = E4M3, E8M0 scales, both operands K-major,
+// D is 128 x n; sf_id selects which of the four scale bytes of a tensor-memory column this MMA uses.
+__device__ __forceinline__ uint32_t umma_idesc_mx_e2m1_e4m3(uint32_t n, uint32_t a_sf_id, uint32_t b_sf_id) {
+  return (b_sf_id << 4) | (5u << 7) | (0u << 10) | ((n >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) |
+         (a_sf_id << 29);
 }
 // Instruction descriptor: E4M3 x E4M3 -> FP32, both operands K-major, D is 128 x n.
 __device__ __forceinline__ uint32_t umma_idesc_e4m3(uint32_t n) {

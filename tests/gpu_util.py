@@ -24,10 +24,18 @@ def host(t):
     return None if t is None else t.cpu().numpy()
 
 
-def untile_codes(tiles: np.ndarray, N: int, K: int):
-    """Decodes the library's tiled weight format (include/zqfp.h) back to plain form:
-    returns (codes uint8 [N, K/2] with element 2b in the low nibble of byte b, shifts uint8 [N, K/64])."""
+def untile_codes(tiles: np.ndarray, N: int, K: int, layout=binding.WEIGHTS_CAST):
+    """Decodes either tiled weight format (include/zqfp.h) back to plain form:
+    returns (codes uint8 [N, K/2] with element 2b in the low nibble of byte b, shifts uint8 [N, K/32])."""
     nt, kb = (N + 127) // 128, K // 128
+    if layout == binding.WEIGHTS_MX:
+        t = np.ascontiguousarray(tiles, dtype=np.uint8).reshape(nt, kb, 8704)
+        codes = t[:, :, :8192].reshape(nt, kb, 128, 64).transpose(0, 2, 1, 3).reshape(nt * 128, K // 2)
+        sf = t[:, :, 8192:].reshape(nt, kb, 32, 4, 4)                   # [nt, kb, r % 32, r / 32, s]
+        sf = sf.transpose(0, 3, 2, 1, 4).reshape(nt * 128, kb * 4)      # [n, K / 32]
+        assert not codes[N:].any() and np.all(sf[N:] == 127), "padding rows: zero codes, unit scales"
+        assert np.all(sf <= 127) and np.all(sf >= 122)
+        return codes[:N], (127 - sf[:N]).astype(np.uint8)
     t = np.ascontiguousarray(tiles, dtype=np.uint8).reshape(nt, kb, 8448)
     words = t[:, :, :8192].copy().view(np.uint32).reshape(nt, kb, 4, 128, 4)     # [nt, kb, chunk, row, word]
     el = np.empty((nt, kb, 4, 128, 4, 8), dtype=np.uint8)                         # 4-bit codes per element
@@ -41,22 +49,23 @@ def untile_codes(tiles: np.ndarray, N: int, K: int):
     codes = (el[:, 0::2] | (el[:, 1::2] << 4)).astype(np.uint8)
     sh = t[:, :, 8192:].reshape(nt, kb, 128, 2).transpose(0, 2, 1, 3).reshape(nt * 128, kb * 2)
     assert not codes[N:].any() and not sh[N:].any(), "padding rows must be zero"
-    return codes[:N], sh[:N]
+    return codes[:N], np.repeat(sh[:N], 2, axis=1)
 
 
 def check_packed(pw, c_o, sh_o, sc_o, group):
     """Bit-exact comparison of a PackedWeight with the oracle's plain codes / shifts / scales."""
-    codes, sh64 = untile_codes(host(pw.codes), pw.N, pw.K)
+    codes, sh32 = untile_codes(host(pw.codes), pw.N, pw.K, pw.layout)
     assert np.array_equal(codes, c_o), "FP4 codes"
     if sh_o is not None:
         assert np.array_equal(host(pw.shift), sh_o), "shifts"
-        assert np.array_equal(sh64, np.repeat(sh_o, group // 64, axis=1)), "shift bytes inside the tiles"
+        assert np.array_equal(sh32, np.repeat(sh_o, group // 32, axis=1)), "shifts inside the tiles"
     else:
-        assert not sh64.any()
+        assert not sh32.any()
     assert np.array_equal(host(pw.scale).view(np.uint32), sc_o.view(np.uint32)), "scales"
 
 
-def check_linear(x_bits, W, U, V, group, mode, out_dtype=torch.float32, rows=None, fused_quant=False):
+def check_linear(x_bits, W, U, V, group, mode, out_dtype=torch.float32, rows=None, fused_quant=False,
+                 layout=binding.WEIGHTS_CAST):
     """Runs oracle and CUDA path on the same inputs; asserts bit-exact codes / scales and y within tolerance."""
     M, K = x_bits.shape
     N = W.shape[0]
@@ -67,7 +76,7 @@ def check_linear(x_bits, W, U, V, group, mode, out_dtype=torch.float32, rows=Non
 
     x = to_bf16(x_bits)
     Wd, Ud, Vd = up(W), up(U), up(V)
-    pw = binding.pack_weight_fp4(Wd, group, mode)
+    pw = binding.pack_weight_fp4(Wd, group, mode, layout)
     check_packed(pw, c_o, sh_o, sc_o, group)
     ws = binding.make_workspace(binding.linear_workspace_bytes(M, N, K, r))
     if fused_quant:

@@ -60,18 +60,20 @@ def test_validation_before_launch(L):
     assert L.zq_quantize_act_fp8(fake, 4, 64, 64, fake, fake, fake, 65, fake, null) == -2
     assert L.zq_quantize_act_fp8(fake, 0, 64, 64, fake, fake, null, 0, null, null) == 0
     # packer
-    assert L.zq_pack_weight_fp4(fake, 4, 256, 100, 1, fake, fake, fake, null) == -2
-    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 3, fake, fake, fake, null) == -4
-    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 1, fake, null, fake, null) == -1
-    assert L.zq_pack_weight_fp4(fake, 0, 256, 128, 1, fake, fake, fake, null) == 0
+    assert L.zq_pack_weight_fp4(fake, 4, 256, 100, 1, 0, fake, fake, fake, null) == -2
+    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 3, 0, fake, fake, fake, null) == -4
+    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 1, 2, fake, fake, fake, null) == -4   # unknown layout
+    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 0, 1, fake, fake, fake, null) == -4   # block scales need M1 / M2
+    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 1, 0, fake, null, fake, null) == -1
+    assert L.zq_pack_weight_fp4(fake, 0, 256, 128, 1, 1, fake, fake, fake, null) == 0
     # linear
-    args = dict(q=fake, sx=fake, x=null, ldx=0, M=4, N=128, K=256, group=128, mode=1, codes=fake, shift=fake,
+    args = dict(q=fake, sx=fake, x=null, ldx=0, M=4, N=128, K=256, group=128, mode=1, layout=0, codes=fake, shift=fake,
                 scale=fake, U=null, V=null, t=null, r=0, y=fake, ydt=0, ldy=128, ws=fake, wsb=1 << 30, st=null)
 
     def call(**kw):
         a = dict(args, **kw)
         return L.zq_w4a8_linear(a["q"], a["sx"], a["x"], a["ldx"], a["M"], a["N"], a["K"], a["group"], a["mode"],
-                                a["codes"], a["shift"], a["scale"], a["U"], a["V"], a["t"], a["r"], a["y"], a["ydt"],
+                                a["layout"], a["codes"], a["shift"], a["scale"], a["U"], a["V"], a["t"], a["r"], a["y"], a["ydt"],
                                 a["ldy"], a["ws"], a["wsb"], a["st"])
 
     assert call(K=192) == -2
@@ -84,6 +86,9 @@ def test_validation_before_launch(L):
     assert call(r=8, U=fake) == -1          # t missing
     assert call(ldy=64) == -2
     assert call(codes=C.c_void_p(0x1008)) == -3
+    assert call(layout=1, codes=C.c_void_p(0x1010)) == -3   # the 4-bit tensor map wants 32-byte alignment
+    assert call(layout=1, mode=0) == -4
+    assert call(layout=3) == -4
     assert call(ws=null) == -5
     assert call(wsb=1024) == -5
     assert call(M=0) == 0

@@ -1,0 +1,98 @@
+"""GPU parity of the layout in which the tensor core performs the cast FP4 -> FP8 (Section 3, "Casting the
+FP4 to FP8"): E2M1 codes as the MMA's own operand, the power-of-two group shift as its E8M0 block scale.
+Same oracle, same tolerances as the casting kernel: packed codes / shifts / scales bit-exact, outputs within
+1e-3 of max |y|, and exact where every product and sum is exactly representable."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2307_09782_b200 import binding, synth
+from tests.gpu_util import TOL_REL, check_linear, check_packed, host, to_bf16, up
+from tests.test_gpu_parity import _layer, _special_weights
+
+pytestmark = pytest.mark.gpu
+MX = binding.WEIGHTS_MX
+
+
+@pytest.mark.parametrize("mode", ["M1", "M2"])
+@pytest.mark.parametrize("group", [64, 128, 256])
+def test_pack_weight_mx_bit_exact(mode, group):
+    W = _special_weights(9, 1024, 31)
+    c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, group, mode)
+    check_packed(binding.pack_weight_fp4(up(W), group, mode, MX), c_o, sh_o, sc_o, group)
+
+
+def test_mx_layout_rejects_unconstrained_scales():
+    W = up(synth.make_w(1, 128, 256))
+    with pytest.raises(binding.ZqError) as e:
+        binding.pack_weight_fp4(W, 128, "none", MX)
+    assert e.value.status == -4
+
+
+@pytest.mark.parametrize("mode", ["M1", "M2"])
+@pytest.mark.parametrize("M", [1, 16, 17, 100, 130, 300])
+def test_linear_small(mode, M):
+    x_bits, W, U, V = _layer(40 + M, M, 384, 512, 8)
+    check_linear(x_bits, W, U, V, 128, mode, layout=MX)
+
+
+@pytest.mark.parametrize("M,N,K,r", [(3, 200, 256, 0), (33, 128, 128, 16), (64, 129, 1024, 8), (7, 1, 384, 8)])
+def test_linear_ragged_tiles(M, N, K, r):
+    x_bits, W, U, V = _layer(60 + M, M, N, K, r)
+    check_linear(x_bits, W, U, V, 128, "M2", layout=MX)
+
+
+@pytest.mark.parametrize("mode,group", [("M1", 64), ("M2", 256), ("M2", 64)])
+def test_linear_other_group_sizes(mode, group):
+    x_bits, W, U, V = _layer(71, 20, 256, 1024, 8)
+    check_linear(x_bits, W, U, V, group, mode, layout=MX)
+
+
+@pytest.mark.parametrize("M", [16, 40, 200])
+def test_linear_split_k_long_rows(M):
+    # few output tiles and a long K: several CTAs share an output tile (atomics or the workspace)
+    x_bits, W, U, V = _layer(81, M, 256, 8192, 8)
+    check_linear(x_bits, W, U, V, 128, "M1", layout=MX)
+
+
+def test_linear_many_tiles_per_cta():
+    # more output tiles than resident CTAs at 16 tokens: every CTA walks several segments, both accumulators
+    x_bits, W, U, V = _layer(83, 9, 128 * 40, 1024, 8)
+    rows = list(range(0, 9))
+    check_linear(x_bits, W, U, V, 128, "M2", layout=MX, rows=None)
+
+
+def test_linear_bf16_output_and_fused_quantizer():
+    x_bits, W, U, V = _layer(91, 48, 512, 1024, 8)
+    check_linear(x_bits, W, U, V, 128, "M2", out_dtype=torch.bfloat16, layout=MX)
+    check_linear(x_bits, W, U, V, 128, "M2", fused_quant=True, layout=MX)
+    check_linear(x_bits, W, None, None, 128, "M1", fused_quant=True, layout=MX)
+
+
+def test_linear_exact_on_power_of_two_data():
+    M, N, K = 16, 256, 512
+    rng = np.random.default_rng(5)
+    x = rng.choice([0.0, 0.25, 0.5, 1.0, -1.0, 2.0], (M, K)).astype(np.float32)
+    x[:, 0] = 7.0
+    W = rng.choice([0.0, 0.5, -1.0, 1.5, 3.0, -4.0], (N, K)).astype(np.float32)
+    W[:, ::128] = 6.0
+    W[3, 128:256] *= 0.125   # a group with shift 3
+    W[200, 256:] *= 0.25     # shift 2 over two groups
+    bits = synth.f32_to_bf16_bits(x)
+    for mode in ("M1", "M2"):
+        y, y_o = check_linear(bits, W, None, None, 128, mode, layout=MX)
+        assert np.array_equal(y, y_o), mode
+
+
+def test_both_layouts_agree():
+    # same codes, same products: the two kernels differ only in summation order
+    M, N, K, r = 64, 384, 2048, 8
+    x_bits, W, U, V = _layer(97, M, N, K, r)
+    x = to_bf16(x_bits)
+    q, sx, t = binding.quantize_act_fp8(x, up(V))
+    ys = []
+    for layout in (binding.WEIGHTS_CAST, MX):
+        pw = binding.pack_weight_fp4(up(W), 128, "M2", layout)
+        ys.append(host(binding.w4a8_linear(pw, q=q, sx=sx, t=t, U=up(U))))
+    assert np.abs(ys[0] - ys[1]).max() <= 1e-5 * np.abs(ys[0]).max()
