@@ -213,6 +213,7 @@ def run_ours(args):
     Ms = list(wl.Ms)
     shapes = list(wl.shapes)
     mode = MODE
+    layout = binding.LAYOUTS[args.layout]
     if args.case:
         parts = args.case.split(",")
         shapes = [synth.LayerShape(int(parts[0]), int(parts[1]), "case")]
@@ -227,7 +228,7 @@ def run_ours(args):
         x_bits = synth.make_x(wl.seed, Mmax, K, wl.n_outliers(K), wl.outlier_factor, row_offset=rank)
         x = torch.from_numpy(x_bits.view(np.int16)).to(dev).view(torch.bfloat16)
         W = torch.from_numpy(synth.make_w(wl.seed, N, K, wl.sigma_w)).to(dev)
-        pw = binding.pack_weight_fp4(W, GROUP, mode)
+        pw = binding.pack_weight_fp4(W, GROUP, mode, layout)
         del W
         U_h, V_h = synth.make_lorc(wl.seed, N, K, RANK)
         U, V = torch.from_numpy(U_h).to(dev), torch.from_numpy(V_h).to(dev)
@@ -262,7 +263,7 @@ def run_ours(args):
         rc = L.zq_quantize_act_fp8(vp(ly["x"]), M, K, K, vp(ly["q"]), vp(ly["sx"]), vp(ly["V"]), RANK, vp(ly["t"]), sp)
         if ev:
             ev[1].record(stream)
-        rc |= L.zq_w4a8_linear(vp(ly["q"]), vp(ly["sx"]), None, 0, M, N, K, GROUP, binding.MODES[mode], vp(codes),
+        rc |= L.zq_w4a8_linear(vp(ly["q"]), vp(ly["sx"]), None, 0, M, N, K, GROUP, binding.MODES[mode], layout, vp(codes),
                                vp(shift), vp(scale), vp(ly["U"]), None, vp(ly["t"]), RANK, vp(ly["y"]), 0, N,
                                vp(ly["ws"]), ly["ws"].numel(), sp)
         if ev:
@@ -328,17 +329,17 @@ def run_ours(args):
     big_flops = sum(2.0 * Mmax * ly["N"] * ly["K"] for ly in layers) / len(layers)
     big_us = statistics.mean(s["gemm_us"] for s in big)
     achieved = big_flops / (big_us * 1e-6) / 1e12
-    roofline = {"bound": "tensor", "kernel": "w4a8_gemm_kernel<256,false>", "achieved": round(achieved, 1),
+    roofline = {"bound": "tensor", "kernel": "w4a8_mx_gemm_kernel<256>" if layout else "w4a8_gemm_kernel<256,false>", "achieved": round(achieved, 1),
                 "peak": round(fp8_peak, 1), "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4), "traffic": None,
                 "peak_source": f"2 x bf16 sustained cuBLAS peak ({peaks['source']}); nominal dense FP8 4500"}
     dec = [s for s in sweep if s["M"] <= 16] or [sweep[0]]
-    roofline_decode = {"bound": "hbm", "kernel": "w4a8_gemm_kernel<16,false>",
+    roofline_decode = {"bound": "hbm", "kernel": "w4a8_mx_gemm_kernel<16>" if layout else "w4a8_gemm_kernel<16,false>",
                        "achieved": round(statistics.mean(s["gemm_gbs"] for s in dec), 1),
                        "peak": peaks["hbm_gbs"], "unit": "GB/s",
                        "frac": round(statistics.mean(s["frac_hbm"] for s in dec), 4), "traffic": None,
                        "peak_source": f"copy bandwidth ({peaks['source']}); nominal 7700-8000"}
     big_q = [s for s in sweep if s["M"] == Mmax and s["layer"].startswith("28672")] or [sweep[-1]]
-    roofline_quant = {"bound": "hbm", "kernel": "act_quant_kernel<true>", "achieved": big_q[0]["quant_gbs"],
+    roofline_quant = {"bound": "hbm", "kernel": "act_quant_rows_kernel<true>", "achieved": big_q[0]["quant_gbs"],
                       "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(big_q[0]["quant_gbs"] / peaks["hbm_gbs"], 4),
                       "traffic": None}
 
@@ -359,7 +360,7 @@ def run_ours(args):
                 ly = layers[li]
                 xh, yh, wsh = hosts[li]
                 codes, shift, scale = ly["copies"][(idx + ci // len(layers)) % N_WEIGHT_COPIES]
-                rc = L.zq_w4a8_linear_host(C.c_void_p(xh.data_ptr()), M, ly["N"], ly["K"], GROUP, binding.MODES[mode],
+                rc = L.zq_w4a8_linear_host(C.c_void_p(xh.data_ptr()), M, ly["N"], ly["K"], GROUP, binding.MODES[mode], layout,
                                            vp(codes), vp(shift), vp(scale), vp(ly["U"]), vp(ly["V"]), RANK,
                                            C.c_void_p(yh.data_ptr()), vp(wsh), wsh.numel(), sp)
                 if rc:
@@ -391,7 +392,7 @@ def run_ours(args):
             "warmup": args.warmup, "ms_per_step": round(ms_max / args.steps, 4), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f8e4m3 x f8e4m3 -> f32", "data": "synthetic",
             "config": {"workload": WORKLOAD if not args.case else f"case {args.case}",
-                       "layers": [f"{s.K}->{s.N}" for s in shapes], "M": Ms, "group": GROUP, "mode": mode, "lorc_rank": RANK, "multi_gpu": "independent replicas",
+                       "layers": [f"{s.K}->{s.N}" for s in shapes], "M": Ms, "group": GROUP, "mode": mode, "weight_layout": args.layout, "lorc_rank": RANK, "multi_gpu": "independent replicas",
                        "l2": f"inputs larger than L2: {N_WEIGHT_COPIES} weight copies per layer rotated, >300 MB "
                              "streamed between two reads of one buffer"},
             "roofline": roofline, "roofline_decode": roofline_decode, "roofline_quant": roofline_quant,
@@ -409,6 +410,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layout", default="mx", choices=["cast", "mx"],
+                    help="weight layout: the kernel casts FP4 to FP8 (cast) or the tensor core does (mx)")
     ap.add_argument("--case", default=None, metavar="K,N,M[,MODE]",
                     help="time one layer shape at one token count instead of the sweep (profiling aid)")
     args = ap.parse_args()

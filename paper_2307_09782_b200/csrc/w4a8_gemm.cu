@@ -123,7 +123,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     u0 = range_start(p, blockIdx.x);
     u1 = range_start(p, blockIdx.x + 1);
   } else {
-    const int z = blockIdx.x / p.tiles, tile = blockIdx.x % p.tiles;
+    const int z = blockIdx.x / p.tiles, tile = raster_tile(p, blockIdx.x % p.tiles);
     u0 = tile * p.kblocks + z * p.kb_per_split;
     u1 = min(u0 + p.kb_per_split, (tile + 1) * p.kblocks);
   }

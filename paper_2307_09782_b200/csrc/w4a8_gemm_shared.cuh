@@ -32,6 +32,7 @@ struct Params {
   //   stream == 0: CTA c = z * tiles + tile owns K blocks [z * kb_per_split, ...) of that tile
   //   stream == 1: the units of all tiles are dealt out evenly, base (+1 for the first rem CTAs) each
   int stream;
+  int m_group;   // stream == 0: CTAs are numbered through groups of this many token tiles (see raster_tile)
   int atomic_y;  // streaming launch with FP32 y: CTAs that share a tile add their share into a zeroed y
   int splits, kb_per_split;
   int base, rem;
@@ -59,6 +60,19 @@ __device__ __forceinline__ void named_bar_sync(int id, int count) {
 __device__ __forceinline__ void raise_error(const Params& p, volatile int* abort_flag, int detail) {
   *abort_flag = 1;
   if (atomicCAS(p.status, 0, ZQ_ERR_DEVICE_TIMEOUT) == 0) p.status[1] = detail;
+}
+
+// Launch order -> output tile.  CTAs that run at the same time should share operands in L2: numbering
+// them along N alone makes one wave read 148 different weight tiles against one token tile, and the whole
+// weight streams from HBM once per token tile.  Numbering through groups of m_group token tiles (N
+// outer, the group's token tiles inner) lets a wave share m_group token tiles and 1 / m_group as many
+// weight tiles, so the weight streams once per group.
+__device__ __forceinline__ int raster_tile(const Params& p, int idx) {
+  if (p.m_group <= 1) return idx;
+  const int per_group = p.m_group * p.n_tiles;
+  const int g = idx / per_group, within = idx - g * per_group;
+  const int gm = min(p.m_group, p.tiles / p.n_tiles - g * p.m_group);  // the last group may be smaller
+  return (g * p.m_group + within % gm) * p.n_tiles + within / gm;
 }
 
 __device__ __forceinline__ int range_start(const Params& p, int c) { return c * p.base + min(c, p.rem); }
@@ -208,6 +222,13 @@ inline Params make_params(const GemmArgs& a, const GemmPlan& plan) {
   p.n_tiles = plan.n_tiles;
   p.tiles = plan.n_tiles * plan.m_tiles;
   p.stream = plan.stream;
+  // as many token tiles per group as keep the group's tokens around 32 MB (they must stay in L2 while the
+  // group walks all of N), at most 8
+  if (!plan.stream && plan.m_tiles > 1) {
+    const int64_t tok_tile_bytes = static_cast<int64_t>(plan.bm) * a.K;
+    const int64_t fit = (int64_t(32) << 20) / tok_tile_bytes;
+    p.m_group = static_cast<int>(fit < 1 ? 1 : (fit > 8 ? 8 : fit));
+  }
   p.atomic_y = (plan.stream && a.ydt == ZQ_OUT_F32 && plan.partial_floats > 0) ? 1 : 0;
   p.splits = plan.splits;
   p.kb_per_split = plan.kb_per_split;
