@@ -32,9 +32,9 @@ inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // Largest split-K scratch any token count up to M can need at this (N, K), over both kernel families.
 size_t max_partial_floats(int64_t M, int64_t N, int64_t K) {
   size_t best = 0;
-  const int64_t cand[6] = {16, 32, 64, 128, 256, M};
+  const int64_t cand[7] = {16, 32, 64, 128, 192, 256, M};
   for (int variant = 0; variant < 3; ++variant)
-    for (int i = 0; i < 6; ++i) {
+    for (int i = 0; i < 7; ++i) {
       const int64_t m = cand[i] < M ? cand[i] : M;
       if (m <= 0) continue;
       const GemmPlan pl = plan_gemm(m, N, K, variant == 0 ? ZQ_SCALE_NONE : ZQ_SCALE_M1,

@@ -626,6 +626,9 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   const int bm_max = (mode == ZQ_SCALE_NONE) ? 64 : 256;
   int bm = 16;
   while (bm < bm_max && bm < M) bm *= 2;
+  // the block-scaled kernel also has a 192-token tile, the widest that leaves room for two accumulators:
+  // it serves every token count beyond one 256-token tile
+  if (mx && (M > 256 || (M > 128 && M <= 192))) bm = 192;
   pl.bm = bm;
   pl.m_tiles = static_cast<int>((M + bm - 1) / bm);
   pl.n_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
@@ -635,11 +638,21 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   const int ctas_per_sm = mx ? (bm <= 64 ? 2 : 1) : ((mode == ZQ_SCALE_NONE || bm > 128) ? 1 : (bm <= 16 ? 3 : 2));
   const int64_t resident = static_cast<int64_t>(ctas_per_sm) * sm_count();
   const int64_t units = tiles * kblocks;
-  if (mode != ZQ_SCALE_NONE && bm == 16 && pl.m_tiles == 1 && tiles <= kWsMaxTiles && units >= 8 &&
+  if (mx && pl.m_tiles > 1) {
+    // many tokens: one resident wave of CTAs walks whole tiles
+    pl.persist = 1;
+    pl.ctas = static_cast<int>(tiles < resident ? tiles : resident);
+    pl.splits = 1;
+    pl.kb_per_split = kblocks;
+    return pl;
+  }
+  if (mode != ZQ_SCALE_NONE && (mx || bm == 16) && pl.m_tiles == 1 && tiles <= kWsMaxTiles && units >= 8 &&
       units < (int64_t(1) << 30)) {
     // At most 16 tokens (decode): the weight streams exactly once and the per-tile epilogue is tiny, so deal
-    // the (tile, K block) units out evenly to one resident wave of CTAs, at least 4 units each.  (Wider
-    // token tiles measured slower this way: their shared tiles cost more atomics than the wave balance saves.)
+    // the (tile, K block) units out evenly to one resident wave of CTAs, at least 4 units each.  (In the casting
+    // kernel wider token tiles measured slower this way: their shared tiles cost more atomics than the wave
+    // balance saves.  The block-scaled kernel finishes one tile while it accumulates the next and does this
+    // for every single row of tiles.)
     int64_t g = resident < units / 4 ? resident : units / 4;
     if (g < 1) g = 1;
     pl.stream = 1;

@@ -32,6 +32,7 @@ struct Params {
   //   stream == 0: CTA c = z * tiles + tile owns K blocks [z * kb_per_split, ...) of that tile
   //   stream == 1: the units of all tiles are dealt out evenly, base (+1 for the first rem CTAs) each
   int stream;
+  int persist;   // CTAs walk whole tiles, every gridDim.x-th position of the launch order (block-scaled kernel)
   int m_group;   // stream == 0: CTAs are numbered through groups of this many token tiles (see raster_tile)
   int atomic_y;  // streaming launch with FP32 y: CTAs that share a tile add their share into a zeroed y
   int splits, kb_per_split;
@@ -222,6 +223,7 @@ inline Params make_params(const GemmArgs& a, const GemmPlan& plan) {
   p.n_tiles = plan.n_tiles;
   p.tiles = plan.n_tiles * plan.m_tiles;
   p.stream = plan.stream;
+  p.persist = plan.persist;
   // as many token tiles per group as keep the group's tokens around 32 MB (they must stay in L2 while the
   // group walks all of N), at most 8
   if (!plan.stream && plan.m_tiles > 1) {

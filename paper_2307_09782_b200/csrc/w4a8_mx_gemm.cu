@@ -17,8 +17,10 @@
 //   D        FP32 in tensor memory, two buffers where they fit, so that the epilogue of one output tile
 //            overlaps the main loop of the next.
 //
-// Orientation, work partition (units of one K block of one output tile, dealt out as contiguous ranges
-// or as split-K), the split-K hand-over and the epilogue are those of the casting kernel.
+// Orientation, the split-K hand-over and the epilogue are those of the casting kernel.  Work partition:
+// few tokens (one row of output tiles): the (tile, K block) units are dealt out evenly as contiguous ranges
+// to one resident wave of CTAs; many tokens: one CTA per SM walks whole 128 x 192 output tiles, every
+// gridDim.x-th one of the launch order, with both accumulator buffers in use.
 //
 // Warp roles: 0..3 epilogue (one TMEM lane quarter each), 4 producer (one lane issues all copies of a
 // stage onto one barrier), 5 TMEM allocation and MMA issue.
@@ -43,7 +45,7 @@ struct MxCfg {
   static constexpr int kStageTx = kTileCodeBytes + kMxTileScaleBytes + kTokBytes;  // bytes a stage's barrier counts
   static constexpr int kBudget = (kMinBlocks == 1 ? 220 : 110) * 1024 - BM * 36 - 512;
   static constexpr int NS = cmin(12, kBudget / (kABytes + kMxTileScaleBytes + kTokBytes));
-  static constexpr int NB = BM <= 128 ? 2 : 1;  // accumulator buffers
+  static constexpr int NB = BM <= 192 ? 2 : 1;  // accumulator buffers
   static constexpr int kDColsPad = BM < 32 ? 32 : BM;
   static constexpr int kSfaCol0 = NB * kDColsPad;
   static constexpr int kSfbCol0 = kSfaCol0 + 4 * NS;
@@ -62,6 +64,48 @@ struct MxCfg {
   static_assert(NS >= 3, "pipeline depth");
   static_assert(kTmemCols * kMinBlocks <= 512, "tensor memory");
   static_assert(kSmemBytes * kMinBlocks <= 226 * 1024, "shared memory");
+};
+
+// The output-tile segments of one CTA, in the order all three roles walk them.
+//   persist: whole tiles, every gridDim.x-th position of the launch order (see raster_tile), so that the CTAs
+//            running at one time work on neighbouring tiles;
+//   stream / split K: the contiguous unit range [us, u1), cut at tile boundaries.
+struct Segments {
+  int us, u1;
+  int idx, step;
+  bool persist;
+  __device__ __forceinline__ explicit Segments(const Params& p) {
+    persist = p.persist != 0;
+    idx = static_cast<int>(blockIdx.x);
+    step = static_cast<int>(gridDim.x);
+    us = u1 = 0;
+    if (p.stream) {
+      us = range_start(p, blockIdx.x);
+      u1 = range_start(p, blockIdx.x + 1);
+    } else if (!persist) {
+      const int z = blockIdx.x / p.tiles, tile = raster_tile(p, blockIdx.x % p.tiles);
+      us = tile * p.kblocks + z * p.kb_per_split;
+      u1 = min(us + p.kb_per_split, (tile + 1) * p.kblocks);
+    }
+  }
+  // next segment: K blocks [kb0, kb0 + nkb) of `tile`
+  __device__ __forceinline__ bool next(const Params& p, int& tile, int& kb0, int& nkb) {
+    if (persist) {
+      if (idx >= p.tiles) return false;
+      tile = raster_tile(p, idx);
+      idx += step;
+      kb0 = 0;
+      nkb = p.kblocks;
+      return true;
+    }
+    if (us >= u1) return false;
+    tile = us / p.kblocks;
+    kb0 = us - tile * p.kblocks;
+    const int ue = min(u1, (tile + 1) * p.kblocks);
+    nkb = ue - us;
+    us = ue;
+    return true;
+  }
 };
 
 template <int BM>
@@ -86,19 +130,6 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
   float* s_t = reinterpret_cast<float*>(smem + C::offT);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // this CTA's units [u0, u1)
-  int u0, u1;
-  if (p.stream) {
-    u0 = range_start(p, blockIdx.x);
-    u1 = range_start(p, blockIdx.x + 1);
-  } else {
-    const int z = blockIdx.x / p.tiles, tile = raster_tile(p, blockIdx.x % p.tiles);
-    u0 = tile * p.kblocks + z * p.kb_per_split;
-    u1 = min(u0 + p.kb_per_split, (tile + 1) * p.kblocks);
-  }
-  const int nunits = u1 - u0;
-  // all of a CTA's tiles share one token tile (streaming is only used with a single row of tiles)
-  const int m0 = ((u0 / p.kblocks) / p.n_tiles) * BM;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < C::NS; ++i) {
@@ -118,13 +149,6 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
   if (warp == C::kProducerWarp && lane == 0) {
     prefetch_tensormap(&tm_w);
     prefetch_tensormap(&tm_q);
-  }
-  if (warp < 4) {
-    // token scales and (rank 8) LoRC rows of this CTA's tokens, for the epilogue
-    for (int c = threadIdx.x; c < BM; c += 128) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
-    if (p.r == 8)
-      for (int c = threadIdx.x; c < BM * 8; c += 128)  // transposed: [j][BM]
-        s_t[(c & 7) * BM + (c >> 3)] = (m0 + (c >> 3) < p.M) ? __ldg(p.t + static_cast<int64_t>(m0) * 8 + c) : 0.0f;
   }
   if (warp == C::kMmaWarp) tmem_alloc(s_tmem, C::kTmemCols);
   tc_fence_before_sync();
@@ -146,35 +170,39 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
   __syncthreads();
   tc_fence_after_sync();
 
+  Segments sg(p);
+  int tile, kb0, nkb;
+
   if (warp == C::kProducerWarp) {
     // ------------------------------------------------------------------ producer
-    if (ok_start) {  // warp-uniform loop, one elected lane issues the copies
+    if (ok_start) {  // warp-uniform loops, one elected lane issues the copies
       const bool issuer = elect_one();
       int s = 0, issued = 0;
       uint32_t ph = 0;
-      int tile = u0 / p.kblocks, kb = u0 % p.kblocks;
-      for (int i = 0; i < nunits; ++i) {
-        if (!mbar_wait(&empty[s], ph ^ 1, s_abort)) {
-          if (issuer) raise_error(p, s_abort, kErrProducer);
-          break;
-        }
-        if (issuer) {
-          const int wt = (tile % p.n_tiles) * p.kblocks + kb;  // index of the weight tile
-          mbar_arrive_expect_tx(&full[s], C::kStageTx);
-          tma_load_3d(s_a + s * C::kABytes, &tm_w, 0, 0, wt, &full[s]);
-          bulk_load(s_sf + s * kMxTileScaleBytes, p.codes + static_cast<int64_t>(wt) * kMxTileBytes + kTileCodeBytes,
-                    kMxTileScaleBytes, &full[s]);
-          tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, kb * kBlockK, m0, &full[s]);
-        }
-        __syncwarp();
-        issued = i + 1;
-        if (++kb == p.kblocks) {
-          kb = 0;
-          ++tile;
-        }
-        if (++s == C::NS) {
-          s = 0;
-          ph ^= 1;
+      bool ok = true;
+      while (ok && sg.next(p, tile, kb0, nkb)) {
+        const int m0 = (tile / p.n_tiles) * BM;
+        const int wt0 = (tile % p.n_tiles) * p.kblocks;  // index of the output channels' first weight tile
+        for (int kb = kb0; kb < kb0 + nkb; ++kb) {
+          if (!mbar_wait(&empty[s], ph ^ 1, s_abort)) {
+            if (issuer) raise_error(p, s_abort, kErrProducer);
+            ok = false;
+            break;
+          }
+          if (issuer) {
+            mbar_arrive_expect_tx(&full[s], C::kStageTx);
+            tma_load_3d(s_a + s * C::kABytes, &tm_w, 0, 0, wt0 + kb, &full[s]);
+            bulk_load(s_sf + s * kMxTileScaleBytes,
+                      p.codes + static_cast<int64_t>(wt0 + kb) * kMxTileBytes + kTileCodeBytes, kMxTileScaleBytes,
+                      &full[s]);
+            tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, kb * kBlockK, m0, &full[s]);
+          }
+          __syncwarp();
+          ++issued;
+          if (++s == C::NS) {
+            s = 0;
+            ph ^= 1;
+          }
         }
       }
       // never leave with copies still in flight: wait (bounded) for the last phase issued per stage
@@ -186,57 +214,50 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
     }
   } else if (warp == C::kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
-    // The whole warp runs the loop (uniform control flow and addresses); one elected lane issues.
+    // The whole warp runs the loops (uniform control flow and addresses); one elected lane issues.
     if (ok_start) {
       const bool issuer = elect_one();
       const uint64_t adesc0 = umma_desc_k128(smem_u32(s_a));
       const uint64_t bdesc0 = umma_desc_k128(smem_u32(s_tok));
       const uint64_t sfdesc0 = umma_desc_rows16(smem_u32(s_sf), 128);
-      int s = 0;
+      int s = 0, seg = 0;
       uint32_t ph = 0;
-      int kb = u0 % p.kblocks, seg = 0;
-      bool seg_first = true;  // the next K block starts a segment (a new accumulation)
       bool failed = false;
-      for (int i = 0; i < nunits && !failed; ++i) {
-        if (!mbar_wait(&full[s], ph, s_abort)) {
+      while (!failed && sg.next(p, tile, kb0, nkb)) {
+        const int buf = seg % C::NB;
+        // the epilogue of the segment that used this accumulator buffer last must have read it
+        if (seg >= C::NB && !mbar_wait(&acc_empty[buf], ((seg / C::NB) - 1) & 1, s_abort)) {
           failed = true;
           break;
         }
-        const int buf = seg % C::NB;
-        if (seg_first && seg >= C::NB) {
-          // the epilogue of the segment that used this buffer last must have read it
-          if (!mbar_wait(&acc_empty[buf], ((seg / C::NB) - 1) & 1, s_abort)) {
+        const uint32_t d_tmem = tmem_base + buf * C::kDColsPad;
+        for (int i = 0; i < nkb; ++i) {
+          if (!mbar_wait(&full[s], ph, s_abort)) {
             failed = true;
             break;
           }
-        }
-        tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + buf * C::kDColsPad;
-        const uint32_t sfa = tmem_sfa + 4 * s;
-        const uint64_t adesc = adesc0 + static_cast<uint64_t>((s * C::kABytes) >> 4);
-        const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((s * C::kTokBytes) >> 4);
-        if (issuer) {
-          tmem_cp_32x128b_x4(sfa, sfdesc0 + static_cast<uint64_t>((s * kMxTileScaleBytes) >> 4));
+          tc_fence_after_sync();
+          const uint32_t sfa = tmem_sfa + 4 * s;
+          const uint64_t adesc = adesc0 + static_cast<uint64_t>((s * C::kABytes) >> 4);
+          const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((s * C::kTokBytes) >> 4);
+          if (issuer) {
+            tmem_cp_32x128b_x4(sfa, sfdesc0 + static_cast<uint64_t>((s * kMxTileScaleBytes) >> 4));
 #pragma unroll
-          for (int k = 0; k < kBlockK / 32; ++k) {
-            // scale byte k of the stage's four columns belongs to elements 32k .. 32k+31
-            umma_mxf8f6f4(d_tmem, adesc + 2 * k, bdesc + 2 * k, umma_idesc_mx_e2m1_e4m3(BM, k, 0),
-                          sfa + (static_cast<uint32_t>(k) << 30), tmem_sfb, (!seg_first || k > 0) ? 1u : 0u);
+            for (int k = 0; k < kBlockK / 32; ++k) {
+              // scale byte k of the stage's four columns belongs to elements 32k .. 32k+31
+              umma_mxf8f6f4(d_tmem, adesc + 2 * k, bdesc + 2 * k, umma_idesc_mx_e2m1_e4m3(BM, k, 0),
+                            sfa + (static_cast<uint32_t>(k) << 30), tmem_sfb, (i > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(&empty[s]);
+            if (i + 1 == nkb) umma_commit(&acc_full[buf]);
+          }
+          __syncwarp();
+          if (++s == C::NS) {
+            s = 0;
+            ph ^= 1;
           }
         }
-        const bool seg_last = (kb + 1 == p.kblocks) || (i + 1 == nunits);
-        if (issuer) {
-          umma_commit(&empty[s]);
-          if (seg_last) umma_commit(&acc_full[buf]);
-        }
-        __syncwarp();
-        seg_first = seg_last;
-        if (seg_last) ++seg;
-        if (++kb == p.kblocks) kb = 0;
-        if (++s == C::NS) {
-          s = 0;
-          ph ^= 1;
-        }
+        ++seg;
       }
       if (failed) {
         if (issuer) {
@@ -255,17 +276,28 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
     const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
     constexpr int EC = BM <= 32 ? 4 : (BM <= 128 ? 8 : 16);  // columns per step
     bool failed = !ok_start;
+    int m0_loaded = -1;
 
     // Every thread walks every segment and executes the same named-barrier sequence whether or not it
     // has failed, so a bounded wait that ran out can never leave others stuck at a hardware barrier.
-    int seg = 0;
-    for (int us = u0; us < u1; ++seg) {
-      const int tile = us / p.kblocks;
-      const int ue = min(u1, (tile + 1) * p.kblocks);
+    for (int seg = 0; sg.next(p, tile, kb0, nkb); ++seg) {
+      const int m0 = (tile / p.n_tiles) * BM;
       const int n = (tile % p.n_tiles) * kTileN + row;
       const bool n_ok = n < p.N;
       const int buf = seg % C::NB;
       const uint32_t t_lane = tmem_base + buf * C::kDColsPad + lane_base;
+
+      if (m0 != m0_loaded) {
+        // token scales and (rank 8) LoRC rows of this tile's tokens
+        named_bar_sync(2, C::kEpiThreads);  // the previous tile's reads are done
+        for (int c = threadIdx.x; c < BM; c += C::kEpiThreads) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
+        if (p.r == 8)
+          for (int c = threadIdx.x; c < BM * 8; c += C::kEpiThreads)  // transposed: [j][BM]
+            s_t[(c & 7) * BM + (c >> 3)] =
+                (m0 + (c >> 3) < p.M) ? __ldg(p.t + static_cast<int64_t>(m0) * 8 + c) : 0.0f;
+        named_bar_sync(2, C::kEpiThreads);
+        m0_loaded = m0;
+      }
 
       float cs = 1.0f;
       uint64_t u[8];  // the channel's U row, each value in both halves of a packed pair
@@ -292,8 +324,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
         tc_fence_after_sync();
       }
 
-      const bool whole_tile = (ue - us) == p.kblocks;
-      if (whole_tile) {
+      if (nkb == p.kblocks) {
         if (!failed) {
           // the next step's accumulator columns are in flight while this step's are finished
           float nxt[EC];
@@ -367,7 +398,6 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[buf]);
-      us = ue;
     }
   }
 
@@ -431,6 +461,7 @@ int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
     case 32: return launch_mx_cfg<32>(a, plan, p, st);
     case 64: return launch_mx_cfg<64>(a, plan, p, st);
     case 128: return launch_mx_cfg<128>(a, plan, p, st);
+    case 192: return launch_mx_cfg<192>(a, plan, p, st);
     case 256: return launch_mx_cfg<256>(a, plan, p, st);
   }
   return ZQ_ERR_SHAPE;

@@ -77,6 +77,7 @@ struct GemmPlan {
   int bm;      // tokens per tile (the MMA's N extent)
   int m_tiles, n_tiles;
   int stream;  // 1: the (tile, K block) units are dealt out evenly to `ctas` CTAs; 0: tiles x splits CTAs
+  int persist; // 1: `ctas` CTAs walk whole tiles, every ctas-th one (neither stream nor split K)
   int ctas;
   int splits;        // stream == 0: split-K factor
   int kb_per_split;  // stream == 0: 128-element K blocks per split

@@ -50,22 +50,31 @@ def _run_layer(wl, shape, modes, Ms, rows_per_case, lorc_variants=(True,)):
     ws = binding.make_workspace(binding.linear_workspace_bytes(Mmax, N, K, r))
     for mode in modes:
         c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, wl.group, mode)
-        pw = binding.pack_weight_fp4(W_d, wl.group, mode)
-        check_packed(pw, c_o, sh_o, sc_o, wl.group)
+        # both weight layouts for the constrained modes: the kernel that casts and the block-scaled one
+        layouts = [binding.WEIGHTS_CAST] + ([binding.WEIGHTS_MX] if mode != "none" else [])
+        pws = []
+        for layout in layouts:
+            pw = binding.pack_weight_fp4(W_d, wl.group, mode, layout)
+            check_packed(pw, c_o, sh_o, sc_o, wl.group)
+            pws.append(pw)
         for M in Ms:
             for with_lorc in lorc_variants:
                 use = bool(r) and with_lorc
-                y = binding.w4a8_linear(pw, x=x_d[:M], U=U_d if use else None, V=V_d if use else None, workspace=ws)
-                assert binding.device_status(ws) == (0, 0)
                 bm = 16
                 while bm < 256 and bm < M:
                     bm *= 2
-                rows = _sample_rows(M, bm, rows_per_case, 1000 + M)
+                rows = sorted(set(_sample_rows(M, bm, rows_per_case, 1000 + M)) |
+                              {r_ for r_ in (191, 192) if r_ < M})
                 y_o = oracle.w4a8_linear(q_o[:M], sx_o[:M], c_o, sh_o, sc_o, wl.group, mode, U if use else None,
                                          t_o[:M] if use else None, rows=rows)
-                err = np.abs(host(y[rows]).astype(np.float64) - y_o).max()
-                assert err <= TOL_REL * np.abs(y_o).max(), (shape, mode, M, use, err, np.abs(y_o).max())
-                del y
+                for pw in pws:
+                    y = binding.w4a8_linear(pw, x=x_d[:M], U=U_d if use else None, V=V_d if use else None,
+                                            workspace=ws)
+                    assert binding.device_status(ws) == (0, 0)
+                    err = np.abs(host(y[rows]).astype(np.float64) - y_o).max()
+                    assert err <= TOL_REL * np.abs(y_o).max(), (shape, mode, pw.layout, M, use, err, np.abs(y_o).max())
+                    del y
+        del pws
 
 
 def test_config_opt125m():

@@ -37,7 +37,9 @@ def test_linear_small(mode, M):
     check_linear(x_bits, W, U, V, 128, mode, layout=MX)
 
 
-@pytest.mark.parametrize("M,N,K,r", [(3, 200, 256, 0), (33, 128, 128, 16), (64, 129, 1024, 8), (7, 1, 384, 8)])
+@pytest.mark.parametrize("M,N,K,r", [(3, 200, 256, 0), (33, 128, 128, 16), (64, 129, 1024, 8), (7, 1, 384, 8),
+                                     (192, 256, 512, 8), (200, 300, 512, 8), (256, 128, 256, 0),
+                                     (700, 1000, 1024, 8), (1153, 2000, 256, 8)])
 def test_linear_ragged_tiles(M, N, K, r):
     x_bits, W, U, V = _layer(60 + M, M, N, K, r)
     check_linear(x_bits, W, U, V, 128, "M2", layout=MX)
@@ -59,8 +61,15 @@ def test_linear_split_k_long_rows(M):
 def test_linear_many_tiles_per_cta():
     # more output tiles than resident CTAs at 16 tokens: every CTA walks several segments, both accumulators
     x_bits, W, U, V = _layer(83, 9, 128 * 40, 1024, 8)
-    rows = list(range(0, 9))
-    check_linear(x_bits, W, U, V, 128, "M2", layout=MX, rows=None)
+    check_linear(x_bits, W, U, V, 128, "M2", layout=MX)
+
+
+def test_linear_many_token_tiles_per_cta():
+    # more 192-token tiles than SMs: the persistent CTAs walk several tiles with different tokens, and the
+    # launch order runs through groups of token tiles
+    x_bits, W, U, V = _layer(85, 192 * 11 + 5, 128 * 20, 256, 8)
+    rows = [0, 191, 192, 383, 1000, 192 * 8 - 1, 192 * 8, 192 * 11, 192 * 11 + 4]
+    check_linear(x_bits, W, U, V, 128, "M1", layout=MX, rows=rows)
 
 
 def test_linear_bf16_output_and_fused_quantizer():
