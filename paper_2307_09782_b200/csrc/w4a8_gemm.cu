@@ -638,15 +638,16 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   const int ctas_per_sm = mx ? (bm <= 64 ? 2 : 1) : ((mode == ZQ_SCALE_NONE || bm > 128) ? 1 : (bm <= 16 ? 3 : 2));
   const int64_t resident = static_cast<int64_t>(ctas_per_sm) * sm_count();
   const int64_t units = tiles * kblocks;
-  if (mx && pl.m_tiles > 1) {
-    // many tokens: one resident wave of CTAs walks whole tiles
+  if (mx && pl.m_tiles > 1 && (tiles >= 4 * resident || tiles > kWsMaxTiles)) {
+    // many tokens: one resident wave of CTAs walks whole tiles (with fewer than four tiles per CTA the
+    // uneven last round would cost too much: those shapes take the contiguous unit ranges below)
     pl.persist = 1;
     pl.ctas = static_cast<int>(tiles < resident ? tiles : resident);
     pl.splits = 1;
     pl.kb_per_split = kblocks;
     return pl;
   }
-  if (mode != ZQ_SCALE_NONE && (mx || bm == 16) && pl.m_tiles == 1 && tiles <= kWsMaxTiles && units >= 8 &&
+  if (mode != ZQ_SCALE_NONE && (mx || (bm == 16 && pl.m_tiles == 1)) && tiles <= kWsMaxTiles && units >= 8 &&
       units < (int64_t(1) << 30)) {
     // At most 16 tokens (decode): the weight streams exactly once and the per-tile epilogue is tiny, so deal
     // the (tile, K block) units out evenly to one resident wave of CTAs, at least 4 units each.  (In the casting

@@ -33,7 +33,7 @@ struct Params {
   //   stream == 1: the units of all tiles are dealt out evenly, base (+1 for the first rem CTAs) each
   int stream;
   int persist;   // CTAs walk whole tiles, every gridDim.x-th position of the launch order (block-scaled kernel)
-  int m_group;   // stream == 0: CTAs are numbered through groups of this many token tiles (see raster_tile)
+  int m_group;   // the launch order runs through groups of this many token tiles (see raster_tile)
   int atomic_y;  // streaming launch with FP32 y: CTAs that share a tile add their share into a zeroed y
   int splits, kb_per_split;
   int base, rem;
@@ -226,7 +226,7 @@ inline Params make_params(const GemmArgs& a, const GemmPlan& plan) {
   p.persist = plan.persist;
   // as many token tiles per group as keep the group's tokens around 32 MB (they must stay in L2 while the
   // group walks all of N), at most 8
-  if (!plan.stream && plan.m_tiles > 1) {
+  if (plan.m_tiles > 1) {
     const int64_t tok_tile_bytes = static_cast<int64_t>(plan.bm) * a.K;
     const int64_t fit = (int64_t(32) << 20) / tok_tile_bytes;
     p.m_group = static_cast<int>(fit < 1 ? 1 : (fit > 8 ? 8 : fit));

@@ -83,27 +83,29 @@ struct Segments {
       us = range_start(p, blockIdx.x);
       u1 = range_start(p, blockIdx.x + 1);
     } else if (!persist) {
-      const int z = blockIdx.x / p.tiles, tile = raster_tile(p, blockIdx.x % p.tiles);
-      us = tile * p.kblocks + z * p.kb_per_split;
-      u1 = min(us + p.kb_per_split, (tile + 1) * p.kblocks);
+      const int z = blockIdx.x / p.tiles, pos = blockIdx.x % p.tiles;
+      us = pos * p.kblocks + z * p.kb_per_split;
+      u1 = min(us + p.kb_per_split, (pos + 1) * p.kblocks);
     }
   }
-  // next segment: K blocks [kb0, kb0 + nkb) of `tile`
-  __device__ __forceinline__ bool next(const Params& p, int& tile, int& kb0, int& nkb) {
+  // next segment: K blocks [kb0, kb0 + nkb) of the output tile at position `pos` of the launch order,
+  // which is tile `tile` (m_tile * n_tiles + n_tile); split-K bookkeeping goes by position
+  __device__ __forceinline__ bool next(const Params& p, int& pos, int& tile, int& kb0, int& nkb) {
     if (persist) {
       if (idx >= p.tiles) return false;
-      tile = raster_tile(p, idx);
+      pos = idx;
       idx += step;
       kb0 = 0;
       nkb = p.kblocks;
-      return true;
+    } else {
+      if (us >= u1) return false;
+      pos = us / p.kblocks;
+      kb0 = us - pos * p.kblocks;
+      const int ue = min(u1, (pos + 1) * p.kblocks);
+      nkb = ue - us;
+      us = ue;
     }
-    if (us >= u1) return false;
-    tile = us / p.kblocks;
-    kb0 = us - tile * p.kblocks;
-    const int ue = min(u1, (tile + 1) * p.kblocks);
-    nkb = ue - us;
-    us = ue;
+    tile = raster_tile(p, pos);
     return true;
   }
 };
@@ -171,7 +173,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
   tc_fence_after_sync();
 
   Segments sg(p);
-  int tile, kb0, nkb;
+  int pos, tile, kb0, nkb;
 
   if (warp == C::kProducerWarp) {
     // ------------------------------------------------------------------ producer
@@ -180,7 +182,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       int s = 0, issued = 0;
       uint32_t ph = 0;
       bool ok = true;
-      while (ok && sg.next(p, tile, kb0, nkb)) {
+      while (ok && sg.next(p, pos, tile, kb0, nkb)) {
         const int m0 = (tile / p.n_tiles) * BM;
         const int wt0 = (tile % p.n_tiles) * p.kblocks;  // index of the output channels' first weight tile
         for (int kb = kb0; kb < kb0 + nkb; ++kb) {
@@ -223,7 +225,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       int s = 0, seg = 0;
       uint32_t ph = 0;
       bool failed = false;
-      while (!failed && sg.next(p, tile, kb0, nkb)) {
+      while (!failed && sg.next(p, pos, tile, kb0, nkb)) {
         const int buf = seg % C::NB;
         // the epilogue of the segment that used this accumulator buffer last must have read it
         if (seg >= C::NB && !mbar_wait(&acc_empty[buf], ((seg / C::NB) - 1) & 1, s_abort)) {
@@ -280,7 +282,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
 
     // Every thread walks every segment and executes the same named-barrier sequence whether or not it
     // has failed, so a bounded wait that ran out can never leave others stuck at a hardware barrier.
-    for (int seg = 0; sg.next(p, tile, kb0, nkb); ++seg) {
+    for (int seg = 0; sg.next(p, pos, tile, kb0, nkb); ++seg) {
       const int m0 = (tile / p.n_tiles) * BM;
       const int n = (tile % p.n_tiles) * kTileN + row;
       const bool n_ok = n < p.N;
@@ -343,7 +345,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
         // Several CTAs share this tile and y was zeroed before the launch: every CTA scales its share
         // and adds it; the first contributor also adds the LoRC term.  No fence, ticket or second pass.
         int first, count;
-        contributors(p, tile, &first, &count);
+        contributors(p, pos, &first, &count);
         const bool lorc = static_cast<int>(blockIdx.x) == first;
         if (!failed) {
 #pragma unroll 1
@@ -357,9 +359,9 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
         // Several CTAs share this tile: leave the raw partial sums in the workspace; the CTA that
         // arrives last adds all of them in contributor order (deterministic) and finishes the tile.
         int first, count;
-        contributors(p, tile, &first, &count);
+        contributors(p, pos, &first, &count);
         const int my_j = p.stream ? static_cast<int>(blockIdx.x) - first : static_cast<int>(blockIdx.x) / p.tiles;
-        float* my_partial = p.partials + partial_slot(p, tile, first, my_j) * (BM * kTileN);
+        float* my_partial = p.partials + partial_slot(p, pos, first, my_j) * (BM * kTileN);
         if (!failed) {
 #pragma unroll 1
           for (int c = 0; c < BM; c += EC) {
@@ -372,9 +374,9 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
         __threadfence();
         named_bar_sync(1, C::kEpiThreads);
         if (threadIdx.x == 0) {
-          const int ticket = (*s_abort) ? -1 : atomicAdd(p.counters + tile, 1);
+          const int ticket = (*s_abort) ? -1 : atomicAdd(p.counters + pos, 1);
           *s_last = (ticket == count - 1) ? 1 : 0;
-          if (ticket == count - 1) p.counters[tile] = 0;  // ready for the next call
+          if (ticket == count - 1) p.counters[pos] = 0;  // ready for the next call
         }
         named_bar_sync(1, C::kEpiThreads);
         if (*s_last) {
@@ -385,7 +387,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
 #pragma unroll
             for (int e = 0; e < EC; ++e) v[e] = 0.0f;
             for (int j = 0; j < count; ++j) {
-              const float* src = p.partials + partial_slot(p, tile, first, j) * (BM * kTileN) + c * kTileN + row;
+              const float* src = p.partials + partial_slot(p, pos, first, j) * (BM * kTileN) + c * kTileN + row;
 #pragma unroll
               for (int e = 0; e < EC; ++e) v[e] += __ldcg(src + e * kTileN);
             }

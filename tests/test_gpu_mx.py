@@ -72,6 +72,15 @@ def test_linear_many_token_tiles_per_cta():
     check_linear(x_bits, W, U, V, 128, "M1", layout=MX, rows=rows)
 
 
+def test_linear_several_token_tiles_dealt_out_as_unit_ranges():
+    # fewer 192-token tiles than four per SM: contiguous unit ranges across token tiles, shared tiles added
+    # with atomics (FP32 y) or handed over through the workspace (bf16 y)
+    x_bits, W, U, V = _layer(87, 500, 640, 2048, 8)
+    rows = [0, 191, 192, 383, 384, 499]
+    check_linear(x_bits, W, U, V, 128, "M2", layout=MX, rows=rows)
+    check_linear(x_bits, W, U, V, 128, "M2", layout=MX, rows=rows, out_dtype=torch.bfloat16)
+
+
 def test_linear_bf16_output_and_fused_quantizer():
     x_bits, W, U, V = _layer(91, 48, 512, 1024, 8)
     check_linear(x_bits, W, U, V, 128, "M2", out_dtype=torch.bfloat16, layout=MX)
