@@ -181,89 +181,83 @@ act_quant_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, uint8_t* _
 
 // ---- many tokens: eight rows per CTA -------------------------------------------------------------
 // With one row per CTA every row re-reads all of V (r x K fp16) from L2, eight times the bytes of the
-// row itself at rank 8.  Here a thread converts its slice of V to FP32 once and applies it to eight
-// rows, so V costs no more than x.  Pass 1 streams the rows once from HBM for absmax and t; pass 2
-// reads them again (they are still in L2: 8 rows per CTA) for the cast.
+// row itself at rank 8, and spends eight FMAs per element on t = V x.  Here a CTA takes eight rows and
+// the LoRC product goes to the tensor cores: bf16 and fp16 values are exact TF32 numbers, so
+// mma.m16n8k8 (TF32 in, FP32 accumulate) computes exact products.  The MMA's A operand is V (its eight
+// rows in the upper half of the 16, the lower half zero), its B operand eight token rows; a lane loads
+// 16 bytes of "its" token row and 16 bytes of "its" V row at the same K offset and feeds them to four
+// MMAs, so no value is moved between lanes.  Pass 1 streams the rows once from HBM for absmax and t;
+// pass 2 reads them again (they are still in L2: 148 CTAs x 8 rows) for the cast.
 constexpr int kRows = 8;
-constexpr int kRowsThreads = 256;
+constexpr int kRowsThreads = 1024;
+constexpr int kRowsWarps = kRowsThreads / 32;
+constexpr int kRowsUnroll = 4;  // 32-element K slices a warp has in flight
+
+__device__ __forceinline__ void mma_tf32_16x8x8(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  // rows 8..15 of A (registers a1, a3) are zero
+  asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
 
 template <bool HAS_V>
-__global__ void __launch_bounds__(kRowsThreads)
+__global__ void __launch_bounds__(kRowsThreads, 1)
 act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec, uint8_t* __restrict__ q,
                       float* __restrict__ sx, const uint4* __restrict__ V, float* __restrict__ t) {
-  __shared__ float s_amax[kRowsThreads / 32][kRows];
-  __shared__ float s_acc[kRowsThreads / 32][kRows * 8];
+  __shared__ float s_amax[kRowsWarps][kRows];
+  __shared__ float s_acc[kRowsWarps][kRows * 8];
   __shared__ float s_inv[kRows];
   const int m0 = blockIdx.x * kRows;
   const int nrows = min(kRows, M - m0);
-  const int nvec = K / 8;
+  const int nvec = K / 8;  // 16-byte vectors per row
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, tig = lane & 3;  // g: token row of this lane, and its row of V
   const uint4* xr = x + static_cast<int64_t>(m0) * ldx_vec;
+  const uint4* xrow = xr + static_cast<int64_t>(g) * ldx_vec;
+  const uint4* vrow = V + static_cast<int64_t>(g) * nvec;
+  const bool row_ok = g < nrows;
 
-  float amax[kRows];
-  float acc[kRows][8];
+  float amax = 0.0f;
+  float d[4] = {0.0f, 0.0f, 0.0f, 0.0f};  // d[0], d[1]: t[token 2 tig, 2 tig + 1][j = g], partial over this warp's K
+  // a warp takes 32-element slices of K: slice index = (it * warps + warp) * unroll + i
+  for (int base = warp * kRowsUnroll * 4; base < nvec; base += kRowsWarps * kRowsUnroll * 4) {
+    uint4 xv[kRowsUnroll], vv[kRowsUnroll];
 #pragma unroll
-  for (int r = 0; r < kRows; ++r) {
-    amax[r] = 0.0f;
+    for (int i = 0; i < kRowsUnroll; ++i) {
+      const int u = base + i * 4 + tig;
+      const bool in = u < nvec;
+      xv[i] = (in && row_ok) ? __ldg(xrow + u) : make_uint4(0, 0, 0, 0);
+      if (HAS_V) vv[i] = in ? __ldg(vrow + u) : make_uint4(0, 0, 0, 0);
+    }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc[r][j] = 0.0f;
-  }
-  for (int u = tid; u < nvec; u += kRowsThreads) {
-    uint4 xv[kRows];
-#pragma unroll
-    for (int r = 0; r < kRows; ++r)
-      xv[r] = (r < nrows) ? __ldg(xr + r * ldx_vec + u) : make_uint4(0, 0, 0, 0);
-    float vf[8][8];
-    if (HAS_V) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const uint4 vv = __ldg(V + static_cast<int64_t>(j) * nvec + u);
-        const uint32_t vw[4] = {vv.x, vv.y, vv.z, vv.w};
+    for (int i = 0; i < kRowsUnroll; ++i) {
+      amax = absmax8(xv[i], amax);
+      if (HAS_V) {
+        const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w};
+        const uint32_t vw[4] = {vv[i].x, vv[i].y, vv[i].z, vv[i].w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           __half2 h;
           *reinterpret_cast<uint32_t*>(&h) = vw[e];
-          const float2 f = __half22float2(h);
-          vf[j][2 * e] = f.x;
-          vf[j][2 * e + 1] = f.y;
+          const float2 vf = __half22float2(h);
+          // elements 2e and 2e+1 of both 8-element pieces stand at MMA-K positions tig and tig + 4
+          mma_tf32_16x8x8(d, __float_as_uint(vf.x), __float_as_uint(vf.y), xw[e] << 16, xw[e] & 0xFFFF0000u);
         }
       }
     }
-#pragma unroll
-    for (int r = 0; r < kRows; ++r) {
-      const uint32_t w[4] = {xv[r].x, xv[r].y, xv[r].z, xv[r].w};
-      float xf[8];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        xf[2 * e] = bf16_lo(w[e]);
-        xf[2 * e + 1] = bf16_hi(w[e]);
-      }
-#pragma unroll
-      for (int e = 0; e < 8; ++e) amax[r] = fmaxf(amax[r], fabsf(xf[e]));
-      if (HAS_V) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-#pragma unroll
-          for (int e = 0; e < 8; ++e) acc[r][j] = fmaf(xf[e], vf[j][e], acc[r][j]);
-      }
-    }
   }
-#pragma unroll
-  for (int r = 0; r < kRows; ++r) {
-    const float a = warp_max(amax[r]);
-    if (lane == 0) s_amax[warp][r] = a;
-    if (HAS_V) {
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float v = warp_sum(acc[r][j]);
-        if (lane == 0) s_acc[warp][r * 8 + j] = v;
-      }
-    }
+  // the four lanes of a token row
+  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+  if (tig == 0) s_amax[warp][g] = amax;
+  if (HAS_V) {
+    s_acc[warp][(2 * tig) * 8 + g] = d[0];      // [token][j]
+    s_acc[warp][(2 * tig + 1) * 8 + g] = d[1];
   }
   __syncthreads();
   if (tid < kRows) {
     float a = s_amax[0][tid];
-    for (int w = 1; w < kRowsThreads / 32; ++w) a = fmaxf(a, s_amax[w][tid]);
+    for (int w = 1; w < kRowsWarps; ++w) a = fmaxf(a, s_amax[w][tid]);
     float s = 1.0f, inv = 1.0f;
     if (a != 0.0f) {
       s = __fdiv_rn(a, 448.0f);
@@ -272,21 +266,19 @@ act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec
     s_inv[tid] = inv;
     if (tid < nrows) sx[m0 + tid] = s;
   }
-  if (HAS_V && tid < kRows * 8 && (tid >> 3) < nrows) {
+  if (HAS_V && tid >= 64 && tid < 64 + kRows * 8 && ((tid - 64) >> 3) < nrows) {
     float v = 0.0f;
-    for (int w = 0; w < kRowsThreads / 32; ++w) v += s_acc[w][tid];
-    t[static_cast<int64_t>(m0) * 8 + tid] = v;
+    for (int w = 0; w < kRowsWarps; ++w) v += s_acc[w][tid - 64];
+    t[static_cast<int64_t>(m0) * 8 + (tid - 64)] = v;
   }
   __syncthreads();
   const int nunits = K / kUnit;
-  for (int r = 0; r < nrows; ++r) {
+  for (int idx = tid; idx < nrows * nunits; idx += kRowsThreads) {
+    const int r = idx / nunits, u = idx - r * nunits;
     const float inv = s_inv[r];
     const uint4* row = xr + r * ldx_vec;
-    uint4* qrow = reinterpret_cast<uint4*>(q + static_cast<int64_t>(m0 + r) * K);
-    for (int u = tid; u < nunits; u += kRowsThreads) {
-      const uint2 lo = cast8(__ldg(row + 2 * u), inv), hi = cast8(__ldg(row + 2 * u + 1), inv);
-      qrow[u] = make_uint4(lo.x, lo.y, hi.x, hi.y);
-    }
+    const uint2 lo = cast8(__ldg(row + 2 * u), inv), hi = cast8(__ldg(row + 2 * u + 1), inv);
+    reinterpret_cast<uint4*>(q + static_cast<int64_t>(m0 + r) * K)[u] = make_uint4(lo.x, lo.y, hi.x, hi.y);
   }
 }
 
