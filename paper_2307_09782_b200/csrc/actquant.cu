@@ -192,6 +192,7 @@ constexpr int kRows = 8;
 constexpr int kRowsThreads = 1024;
 constexpr int kRowsWarps = kRowsThreads / 32;
 constexpr int kRowsUnroll = 4;  // 32-element K slices a warp has in flight
+constexpr int kRowsMinTokens = 384;
 
 __device__ __forceinline__ void mma_tf32_16x8x8(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
   // rows 8..15 of A (registers a1, a3) are zero
@@ -398,8 +399,9 @@ act_quant_cluster_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, ui
 int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
                      const void* V, int r, float* t, cudaStream_t st) {
   if (M == 0) return ZQ_OK;
-  // enough rows to fill the GPU with eight-row CTAs, and the rank the row kernel is written for
-  if (M >= 8 * 148 && (V == nullptr || r == 8)) {
+  // enough rows for the eight-row CTAs to beat one row per CTA (measured: from about 50 CTAs on), and the
+  // rank the row kernel is written for
+  if (M >= kRowsMinTokens && (V == nullptr || r == 8)) {
     dim3 grid(static_cast<unsigned>((M + kRows - 1) / kRows));
     if (V)
       act_quant_rows_kernel<true><<<grid, kRowsThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(M),
@@ -412,7 +414,7 @@ int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* 
     return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
   }
   // fewer tokens than the eight-row kernel needs, rows long enough to be worth sharing: a cluster of eight CTAs per row
-  if (M < 8 * 148 && (M <= 256 || K >= 16384) && K >= 2048 &&
+  if (M < kRowsMinTokens && (M <= 256 || K >= 16384) && K >= 2048 &&
       K / kUnit <= kClusterSize * kClusterThreads * kClusterVpt) {
     dim3 grid(kClusterSize, static_cast<unsigned>(M));
     act_quant_cluster_kernel<<<grid, kClusterThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(K),

@@ -19,7 +19,7 @@ constexpr int kBlockK = 128;  // K elements per pipeline step
 constexpr int kAStageCols = kBlockK / 4;  // TMEM columns of one widened 128 x 128 tile (4 bytes per column)
 
 // error detail codes written to status[1]
-enum { kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6 };
+enum { kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6, kErrZero = 7 };
 
 struct Params {
   int M, N, K;
@@ -35,6 +35,7 @@ struct Params {
   int persist;   // CTAs walk whole tiles, every gridDim.x-th position of the launch order (block-scaled kernel)
   int m_group;   // the launch order runs through groups of this many token tiles (see raster_tile)
   int atomic_y;  // streaming launch with FP32 y: CTAs that share a tile add their share into a zeroed y
+  int coop_zero; // cooperative launch: the kernel zeroes y itself and holds every output back until all CTAs have
   int splits, kb_per_split;
   int base, rem;
   const uint8_t* codes;  // tiled weight

@@ -280,6 +280,26 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
     bool failed = !ok_start;
     int m0_loaded = -1;
 
+    // Cooperative launch (all CTAs resident at once): instead of a memset before the kernel, every CTA
+    // clears its share of y now, while the first tiles are in flight, and announces it; outputs are
+    // held back until all CTAs have.
+    bool y_ready = p.coop_zero == 0;
+    if (p.coop_zero) {
+      float* y = static_cast<float*>(p.y);
+      const int64_t stride = static_cast<int64_t>(gridDim.x) * C::kEpiThreads;
+      const int64_t first = static_cast<int64_t>(blockIdx.x) * C::kEpiThreads + threadIdx.x;
+      if ((p.N & 3) == 0 && (p.ldy & 3) == 0 && (reinterpret_cast<uintptr_t>(y) & 15u) == 0) {
+        const int n4 = p.N >> 2;
+        for (int64_t i = first; i < static_cast<int64_t>(p.M) * n4; i += stride)
+          *reinterpret_cast<float4*>(y + (i / n4) * p.ldy + (i % n4) * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+      } else {
+        for (int64_t i = first; i < static_cast<int64_t>(p.M) * p.N; i += stride) y[(i / p.N) * p.ldy + i % p.N] = 0.0f;
+      }
+      __threadfence();
+      named_bar_sync(2, C::kEpiThreads);
+      if (threadIdx.x == 0) atomicAdd(p.status + kWsZeroArrive, 1);
+    }
+
     // Every thread walks every segment and executes the same named-barrier sequence whether or not it
     // has failed, so a bounded wait that ran out can never leave others stuck at a hardware barrier.
     for (int seg = 0; sg.next(p, pos, tile, kb0, nkb); ++seg) {
@@ -324,6 +344,23 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
           failed = true;
         }
         tc_fence_after_sync();
+      }
+      if (!y_ready) {
+        // every CTA has cleared its share of y (bounded wait; the CTAs of a cooperative launch all run)
+        if (threadIdx.x == 0) {
+          const uint64_t t0 = global_timer_ns();
+          volatile int* arrived = p.status + kWsZeroArrive;
+          bool ok = false;
+          for (uint32_t spin = 0; spin < kSpinLimit && !ok; ++spin) {
+            ok = *arrived >= static_cast<int>(gridDim.x);
+            if (!ok && (spin & 63u) == 63u && global_timer_ns() - t0 > kWaitLimitNs) break;
+          }
+          if (!ok) raise_error(p, s_abort, kErrZero);
+          __threadfence();
+        }
+        named_bar_sync(2, C::kEpiThreads);
+        y_ready = true;
+        if (*s_abort) failed = true;
       }
 
       if (nkb == p.kblocks) {
@@ -401,6 +438,13 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[buf]);
     }
+    if (p.coop_zero && threadIdx.x == 0) {
+      // this CTA is past the hand-over; the last CTA to get here leaves both counters at zero for the next call
+      if (atomicAdd(p.status + kWsZeroDone, 1) == static_cast<int>(gridDim.x) - 1) {
+        p.status[kWsZeroArrive] = 0;
+        p.status[kWsZeroDone] = 0;
+      }
+    }
   }
 
   tc_fence_before_sync();
@@ -441,11 +485,24 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
                                     C::kSmemBytes);
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
-  if (p.atomic_y &&
-      cudaMemset2DAsync(a.y, static_cast<size_t>(a.ldy) * 4, 0, static_cast<size_t>(a.N) * 4, static_cast<size_t>(a.M),
-                        st) != cudaSuccess)
-    return ZQ_ERR_CUDA;
   dim3 grid(static_cast<unsigned>(plan.ctas));
+  if (p.atomic_y) {
+    // y must be zero before the first CTA adds into it.  A cooperative launch (all CTAs resident, which the
+    // plan's grid is sized for) lets the kernel clear y itself; if the device cannot hold the grid at once,
+    // clear y with a memset and launch normally.
+    Params pc = p;
+    pc.coop_zero = 1;
+    void* args[3] = {&tm_w, &tm_q, &pc};
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM>), grid, dim3(C::kThreads),
+                                    args, C::kSmemBytes, st) == cudaSuccess) {
+      count_launch();
+      return ZQ_OK;
+    }
+    (void)cudaGetLastError();  // not launched; fall back
+    if (cudaMemset2DAsync(a.y, static_cast<size_t>(a.ldy) * 4, 0, static_cast<size_t>(a.N) * 4,
+                          static_cast<size_t>(a.M), st) != cudaSuccess)
+      return ZQ_ERR_CUDA;
+  }
   w4a8_mx_gemm_kernel<BM><<<grid, C::kThreads, C::kSmemBytes, st>>>(tm_w, tm_q, p);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;

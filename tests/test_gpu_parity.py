@@ -26,7 +26,8 @@ def test_act_quant_bit_exact(M, K):
     assert np.abs(host(t) - t_o).max() <= 1e-4 * np.abs(t_o).max()
 
 
-@pytest.mark.parametrize("M,K,lorc", [(1187, 768, True), (1184, 2048, False), (2500, 256, True)])
+@pytest.mark.parametrize("M,K,lorc", [(1187, 768, True), (1184, 2048, False), (2500, 256, True), (385, 4096, True),
+                                      (384, 48, True), (300, 16384, True)])
 def test_act_quant_many_rows_kernel(M, K, lorc):
     """Token counts large enough for the eight-rows-per-CTA kernel, with a ragged last CTA."""
     x_bits = synth.make_x(300 + M, M, K, max(1, K // 100), 20.0)
