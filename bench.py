@@ -30,6 +30,8 @@ from paper_2307_09782_b200 import synth  # noqa: E402
 
 WORKLOAD = "opt30b"
 GROUP, MODE, RANK = 128, "M2", 8
+# ncu, one pass, the bench's own M = 8192 launches of w4a8_mx_gemm_kernel<192> (profiles/): 1625.3 MB and 1795.9 MB
+DOMINANT_TRAFFIC = 1710.6e6
 METRIC = "w4a8_linear_tflops"
 UNIT = "TFLOP/s"
 N_WEIGHT_COPIES = 2  # per layer; rotated so that > 2x the L2 size streams between two reads of one buffer
@@ -155,13 +157,13 @@ def run_reference(args):
     state = None
     times, fl = [], 0.0
     for i in range(args.warmup + args.steps):
-        dt, fl, state = oracle_sample_step(wl, state, M_s=4)
+        dt, fl, state = oracle_sample_step(wl, state, M_s=2)
         if i >= args.warmup:
             times.append(dt)
     total = sum(times)
     value = fl * len(times) / total / 1e12
     shape = wl.shapes[0]
-    sample = (f"each step: {wl.name} {shape.K}->{shape.N}, first 4 tokens, all outputs (quantizer + LoRC + FP64 "
+    sample = (f"each step: {wl.name} {shape.K}->{shape.N}, first 2 tokens, all outputs (quantizer + LoRC + FP64 "
               f"linear); a bounded sample of the sweep")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
@@ -330,7 +332,9 @@ def run_ours(args):
     big_us = statistics.mean(s["gemm_us"] for s in big)
     achieved = big_flops / (big_us * 1e-6) / 1e12
     roofline = {"bound": "tensor", "kernel": "w4a8_mx_gemm_kernel<256>" if layout else "w4a8_gemm_kernel<256,false>", "achieved": round(achieved, 1),
-                "peak": round(fp8_peak, 1), "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4), "traffic": None,
+                "peak": round(fp8_peak, 1), "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4),
+                "traffic": DOMINANT_TRAFFIC if (layout and not args.case) else None,
+                "traffic_note": "DRAM bytes per launch (ncu dram__bytes_read + write, mean of the two M = 8192 launches)",
                 "peak_source": f"2 x bf16 sustained cuBLAS peak ({peaks['source']}); nominal dense FP8 4500"}
     dec = [s for s in sweep if s["M"] <= 16] or [sweep[0]]
     roofline_decode = {"bound": "hbm", "kernel": "w4a8_mx_gemm_kernel<16>" if layout else "w4a8_gemm_kernel<16,false>",
@@ -405,8 +409,8 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
