@@ -32,6 +32,8 @@ WORKLOAD = "opt30b"
 GROUP, MODE, RANK = 128, "M2", 8
 # ncu, one pass, the bench's own M = 8192 launches of w4a8_mx_gemm_kernel<192> (profiles/): 1625.3 MB and 1795.9 MB
 DOMINANT_TRAFFIC = 1710.6e6
+# ncu --set full, w4a8_mx_gemm_kernel<16> at 7168->28672, M = 8 (profiles/): read + write of the two captured launches
+DECODE_TRAFFIC = 116.8e6
 METRIC = "w4a8_linear_tflops"
 UNIT = "TFLOP/s"
 N_WEIGHT_COPIES = 2  # per layer; rotated so that > 2x the L2 size streams between two reads of one buffer
@@ -331,7 +333,7 @@ def run_ours(args):
     big_flops = sum(2.0 * Mmax * ly["N"] * ly["K"] for ly in layers) / len(layers)
     big_us = statistics.mean(s["gemm_us"] for s in big)
     achieved = big_flops / (big_us * 1e-6) / 1e12
-    roofline = {"bound": "tensor", "kernel": "w4a8_mx_gemm_kernel<256>" if layout else "w4a8_gemm_kernel<256,false>", "achieved": round(achieved, 1),
+    roofline = {"bound": "tensor", "kernel": "w4a8_mx_gemm_kernel<192>" if layout else "w4a8_gemm_kernel<256,false>", "achieved": round(achieved, 1),
                 "peak": round(fp8_peak, 1), "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4),
                 "traffic": DOMINANT_TRAFFIC if (layout and not args.case) else None,
                 "traffic_note": "DRAM bytes per launch (ncu dram__bytes_read + write, mean of the two M = 8192 launches)",
@@ -340,7 +342,9 @@ def run_ours(args):
     roofline_decode = {"bound": "hbm", "kernel": "w4a8_mx_gemm_kernel<16>" if layout else "w4a8_gemm_kernel<16,false>",
                        "achieved": round(statistics.mean(s["gemm_gbs"] for s in dec), 1),
                        "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                       "frac": round(statistics.mean(s["frac_hbm"] for s in dec), 4), "traffic": None,
+                       "frac": round(statistics.mean(s["frac_hbm"] for s in dec), 4),
+                       "traffic": DECODE_TRAFFIC if (layout and not args.case) else None,
+                       "traffic_note": "DRAM bytes per launch (ncu, 7168->28672 at M = 8, mean of two launches)",
                        "peak_source": f"copy bandwidth ({peaks['source']}); nominal 7700-8000"}
     big_q = [s for s in sweep if s["M"] == Mmax and s["layer"].startswith("28672")] or [sweep[-1]]
     roofline_quant = {"bound": "hbm", "kernel": "act_quant_rows_kernel<true>", "achieved": big_q[0]["quant_gbs"],

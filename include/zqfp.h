@@ -147,9 +147,10 @@ int zq_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  * K % 128 == 0; group in {64, 128, 256}; r in {0, 8, 16, ..., 64}; q, codes 16-byte aligned (codes 32-byte
  * aligned with ZQ_WEIGHTS_MX).
  * M == 0 or N == 0 is a no-op.  Summation order over K depends on the launch shape, so FP32 results are
- * not bit-identical across token counts.  When all tokens fit one tile (M <= 256, constrained modes,
- * FP32 y) the K range of a tile is shared by CTAs that add into y with FP32 atomics (y is zeroed by the
- * call first): the last bit can then differ from run to run; other shapes are reproducible.
+ * not bit-identical across token counts.  Where the K range of an output tile is shared by several CTAs
+ * and y is FP32 (ZQ_WEIGHTS_CAST: M <= 16; ZQ_WEIGHTS_MX: up to 256 tokens, and larger token counts
+ * with fewer than about 600 output tiles of 128 x 192) the CTAs add into y with FP32 atomics (y is cleared by
+ * the call first): the last bit can then differ from run to run; other shapes, and bf16 y, are reproducible.
  */
 int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M,
                    int64_t N, int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout,
