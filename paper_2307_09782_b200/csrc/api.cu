@@ -32,19 +32,19 @@ inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // Largest split-K scratch any token count up to M can need at this (N, K), over both kernel families.
 size_t max_partial_floats(int64_t M, int64_t N, int64_t K) {
   size_t best = 0;
-  const int64_t cand[7] = {16, 32, 64, 128, 192, 256, M};
+  const int64_t cand[8] = {16, 32, 64, 128, 192, 224, 256, M};
   for (int variant = 0; variant < 3; ++variant)
-    for (int i = 0; i < 7; ++i) {
+    for (int i = 0; i < 8; ++i) {
       const int64_t m = cand[i] < M ? cand[i] : M;
       if (m <= 0) continue;
       const GemmPlan pl = plan_gemm(m, N, K, variant == 0 ? ZQ_SCALE_NONE : ZQ_SCALE_M1,
                                     variant == 2 ? ZQ_WEIGHTS_MX : ZQ_WEIGHTS_CAST);
       if (pl.partial_floats > best) best = pl.partial_floats;
     }
-  // Between 256 tokens and M the block-scaled kernel may deal 192-token tiles out as contiguous unit
+  // Between 256 tokens and M the block-scaled kernel may deal 192- or 224-token tiles out as contiguous unit
   // ranges to one CTA per SM, each of which leaves at most two partial tiles.
   if (M > 256) {
-    const size_t stream_192 = 2 * static_cast<size_t>(sm_count()) * 192 * 128;
+    const size_t stream_192 = 2 * static_cast<size_t>(sm_count()) * 224 * 128;
     if (stream_192 > best) best = stream_192;
   }
   return best;

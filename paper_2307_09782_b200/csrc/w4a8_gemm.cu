@@ -629,6 +629,11 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   // the block-scaled kernel also has a 192-token tile, the widest that leaves room for two accumulators:
   // it serves every token count beyond one 256-token tile
   if (mx && (M > 256 || (M > 128 && M <= 192))) bm = 192;
+  // 224 tokens still leave room for two accumulators and move fewer shared-memory bytes per flop (the
+  // bound of this kernel); taken when the padding of the last tile does not eat the gain
+  if (mx && M > 256 && ((M + 223) / 224) * 224 * 20 < ((M + 191) / 192) * 192 * 21 &&
+      ((M + 223) / 224) * ((N + kTileN - 1) / kTileN) >= 4 * static_cast<int64_t>(sm_count()))
+    bm = 224;
   // long rows: the epilogue is a small share of a tile, and a 256-token tile (one accumulator, no overlap)
   // moves fewer shared-memory bytes per flop
   if (mx && M > 256 && K >= 16384 &&

@@ -45,7 +45,7 @@ struct MxCfg {
   static constexpr int kStageTx = kTileCodeBytes + kMxTileScaleBytes + kTokBytes;  // bytes a stage's barrier counts
   static constexpr int kBudget = (kMinBlocks == 1 ? 220 : 110) * 1024 - BM * 36 - 512;
   static constexpr int NS = cmin(12, kBudget / (kABytes + kMxTileScaleBytes + kTokBytes));
-  static constexpr int NB = BM <= 192 ? 2 : 1;  // accumulator buffers
+  static constexpr int NB = BM <= 224 ? 2 : 1;  // accumulator buffers
   static constexpr int kDColsPad = BM < 32 ? 32 : BM;
   static constexpr int kSfaCol0 = NB * kDColsPad;
   static constexpr int kSfbCol0 = kSfaCol0 + 4 * NS;
@@ -521,6 +521,7 @@ int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
     case 64: return launch_mx_cfg<64>(a, plan, p, st);
     case 128: return launch_mx_cfg<128>(a, plan, p, st);
     case 192: return launch_mx_cfg<192>(a, plan, p, st);
+    case 224: return launch_mx_cfg<224>(a, plan, p, st);
     case 256: return launch_mx_cfg<256>(a, plan, p, st);
   }
   return ZQ_ERR_SHAPE;

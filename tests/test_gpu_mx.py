@@ -72,6 +72,15 @@ def test_linear_many_token_tiles_per_cta():
     check_linear(x_bits, W, U, V, 128, "M1", layout=MX, rows=rows)
 
 
+@pytest.mark.parametrize("M", [1120, 1000])
+def test_linear_persistent_whole_tiles(M):
+    # 600 output tiles, more than four per SM: every CTA walks whole tiles (224 or 192 tokens wide) of
+    # different token rows with both accumulator buffers
+    x_bits, W, U, V = _layer(89, M, 128 * 120, 256, 8)
+    rows = [0, 191, 192, 223, 224, 447, 448, 700, M - 1]
+    check_linear(x_bits, W, U, V, 128, "M2", layout=MX, rows=rows)
+
+
 def test_linear_several_token_tiles_dealt_out_as_unit_ranges():
     # fewer 192-token tiles than four per SM: contiguous unit ranges across token tiles, shared tiles added
     # with atomics (FP32 y) or handed over through the workspace (bf16 y)
