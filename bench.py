@@ -30,8 +30,8 @@ from paper_2307_09782_b200 import synth  # noqa: E402
 
 WORKLOAD = "opt30b"
 GROUP, MODE, RANK = 128, "M2", 8
-# ncu, one pass, the bench's own M = 8192 launches of w4a8_mx_gemm_kernel<192> (profiles/): 1625.3 MB and 1795.9 MB
-DOMINANT_TRAFFIC = 1710.6e6
+# ncu, one pass, the bench's own M = 8192 launches of w4a8_mx_gemm_kernel<224> / <256> (profiles/): 1505.4 MB and 1654.6 MB
+DOMINANT_TRAFFIC = 1580.0e6
 # ncu --set full, w4a8_mx_gemm_kernel<16> at 7168->28672, M = 8 (profiles/): read + write of the two captured launches
 DECODE_TRAFFIC = 116.8e6
 METRIC = "w4a8_linear_tflops"
@@ -333,7 +333,7 @@ def run_ours(args):
     big_flops = sum(2.0 * Mmax * ly["N"] * ly["K"] for ly in layers) / len(layers)
     big_us = statistics.mean(s["gemm_us"] for s in big)
     achieved = big_flops / (big_us * 1e-6) / 1e12
-    roofline = {"bound": "tensor", "kernel": "w4a8_mx_gemm_kernel<192>" if layout else "w4a8_gemm_kernel<256,false>", "achieved": round(achieved, 1),
+    roofline = {"bound": "tensor", "kernel": "w4a8_mx_gemm_kernel<224> (7168->28672), <256> (28672->7168)" if layout else "w4a8_gemm_kernel<256,false>", "achieved": round(achieved, 1),
                 "peak": round(fp8_peak, 1), "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4),
                 "traffic": DOMINANT_TRAFFIC if (layout and not args.case) else None,
                 "traffic_note": "DRAM bytes per launch (ncu dram__bytes_read + write, mean of the two M = 8192 launches)",
