@@ -41,10 +41,11 @@ size_t max_partial_floats(int64_t M, int64_t N, int64_t K) {
                                     variant == 2 ? ZQ_WEIGHTS_MX : ZQ_WEIGHTS_CAST);
       if (pl.partial_floats > best) best = pl.partial_floats;
     }
-  // Between 256 tokens and M the block-scaled kernel may deal 192- or 224-token tiles out as contiguous unit
-  // ranges to one CTA per SM, each of which leaves at most two partial tiles.
+  // Beyond 256 tokens the block-scaled kernel may deal tiles of up to 256 tokens out as contiguous unit
+  // ranges to one CTA per SM (all of them, or the last round of a persistent launch), each of which
+  // leaves at most two partial tiles.
   if (M > 256) {
-    const size_t stream_192 = 2 * static_cast<size_t>(sm_count()) * 224 * 128;
+    const size_t stream_192 = 2 * static_cast<size_t>(sm_count()) * 256 * 128;
     if (stream_192 > best) best = stream_192;
   }
   return best;

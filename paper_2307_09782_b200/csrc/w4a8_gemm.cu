@@ -652,9 +652,19 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
     // many tokens: one resident wave of CTAs walks whole tiles (with fewer than four tiles per CTA the
     // uneven last round would cost too much: those shapes take the contiguous unit ranges below)
     pl.persist = 1;
-    pl.ctas = static_cast<int>(tiles < resident ? tiles : resident);
+    const int64_t g = tiles < resident ? tiles : resident;
+    pl.ctas = static_cast<int>(g);
     pl.splits = 1;
     pl.kb_per_split = kblocks;
+    // whole rounds as whole tiles; the tiles of the last, incomplete round as unit ranges over all CTAs
+    // (they hand partial sums over through the workspace)
+    // ... when that saves more than the shared tiles' extra epilogues cost (about 60 K blocks' time)
+    int64_t tail_tiles = tiles <= kWsMaxTiles ? tiles % g : 0;
+    if ((g - tail_tiles) * kblocks < 60 * g) tail_tiles = 0;
+    pl.tail_pos0 = static_cast<int>(tiles - tail_tiles);
+    pl.base = static_cast<int>(tail_tiles * kblocks / g);
+    pl.rem = static_cast<int>(tail_tiles * kblocks % g);
+    pl.partial_floats = tail_tiles > 0 ? 2 * static_cast<size_t>(g) * bm * kTileN : 0;
     return pl;
   }
   if (mode != ZQ_SCALE_NONE && (mx || (bm == 16 && pl.m_tiles == 1)) && tiles <= kWsMaxTiles && units >= 8 &&

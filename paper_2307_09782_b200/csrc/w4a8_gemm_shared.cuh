@@ -32,7 +32,10 @@ struct Params {
   //   stream == 0: CTA c = z * tiles + tile owns K blocks [z * kb_per_split, ...) of that tile
   //   stream == 1: the units of all tiles are dealt out evenly, base (+1 for the first rem CTAs) each
   int stream;
-  int persist;   // CTAs walk whole tiles, every gridDim.x-th position of the launch order (block-scaled kernel)
+  int persist;   // CTAs walk whole tiles, every gridDim.x-th position of the launch order (block-scaled kernel),
+                 // up to position tail_pos0; the tiles from there on are dealt out as unit ranges like stream == 1
+  int tail_pos0;
+  int dealt0;    // first unit of the units that are dealt out as ranges (0 when stream == 1)
   int m_group;   // the launch order runs through groups of this many token tiles (see raster_tile)
   int atomic_y;  // streaming launch with FP32 y: CTAs that share a tile add their share into a zeroed y
   int coop_zero; // cooperative launch: the kernel zeroes y itself and holds every output back until all CTAs have
@@ -80,24 +83,25 @@ __device__ __forceinline__ int raster_tile(const Params& p, int idx) {
 __device__ __forceinline__ int range_start(const Params& p, int c) { return c * p.base + min(c, p.rem); }
 __device__ __forceinline__ int cta_of_unit(const Params& p, int u) {
   const int big = p.rem * (p.base + 1);
-  return u < big ? u / (p.base + 1) : p.rem + (u - big) / p.base;
+  return (u < big || p.base == 0) ? u / (p.base + 1) : p.rem + (u - big) / p.base;
 }
 // The CTAs that contribute partial sums to `tile`: first CTA and their number.
 __device__ __forceinline__ void contributors(const Params& p, int tile, int* first, int* count) {
-  if (p.stream) {
-    *first = cta_of_unit(p, tile * p.kblocks);
-    *count = cta_of_unit(p, tile * p.kblocks + p.kblocks - 1) - *first + 1;
+  if (p.stream || p.persist) {
+    const int u = tile * p.kblocks - p.dealt0;
+    *first = cta_of_unit(p, u);
+    *count = cta_of_unit(p, u + p.kblocks - 1) - *first + 1;
   } else {
     *first = 0;
     *count = p.splits;
   }
 }
-// Workspace slot of the partial sum that contributor j (CTA first + j) leaves for `tile`.  A streaming
-// CTA can leave two (for the tile its range starts in and for the one it ends in).
+// Workspace slot of the partial sum that contributor j (CTA first + j) leaves for `tile`.  A CTA with a
+// dealt-out range can leave two (for the tile its range starts in and for the one it ends in).
 __device__ __forceinline__ size_t partial_slot(const Params& p, int tile, int first, int j) {
-  if (!p.stream) return static_cast<size_t>(tile) * p.splits + j;
+  if (!(p.stream || p.persist)) return static_cast<size_t>(tile) * p.splits + j;
   const int c = first + j;
-  return 2 * static_cast<size_t>(c) + (range_start(p, c) / p.kblocks == tile ? 0 : 1);
+  return 2 * static_cast<size_t>(c) + ((p.dealt0 + range_start(p, c)) / p.kblocks == tile ? 0 : 1);
 }
 
 // Final arithmetic of NC consecutive tokens (tile columns c0 .. c0+NC-1) of one output channel, and the store.
@@ -225,6 +229,8 @@ inline Params make_params(const GemmArgs& a, const GemmPlan& plan) {
   p.tiles = plan.n_tiles * plan.m_tiles;
   p.stream = plan.stream;
   p.persist = plan.persist;
+  p.tail_pos0 = plan.tail_pos0;
+  p.dealt0 = plan.persist ? plan.tail_pos0 * p.kblocks : 0;
   // as many token tiles per group as keep the group's tokens around 32 MB (they must stay in L2 while the
   // group walks all of N), at most 8
   if (plan.m_tiles > 1) {

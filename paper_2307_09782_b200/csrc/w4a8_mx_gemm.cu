@@ -68,7 +68,8 @@ struct MxCfg {
 
 // The output-tile segments of one CTA, in the order all three roles walk them.
 //   persist: whole tiles, every gridDim.x-th position of the launch order (see raster_tile), so that the CTAs
-//            running at one time work on neighbouring tiles;
+//            running at one time work on neighbouring tiles; the positions of the last, incomplete round
+//            are then dealt out as unit ranges, so that no SM idles through a whole tile's time;
 //   stream / split K: the contiguous unit range [us, u1), cut at tile boundaries.
 struct Segments {
   int us, u1;
@@ -79,10 +80,10 @@ struct Segments {
     idx = static_cast<int>(blockIdx.x);
     step = static_cast<int>(gridDim.x);
     us = u1 = 0;
-    if (p.stream) {
-      us = range_start(p, blockIdx.x);
-      u1 = range_start(p, blockIdx.x + 1);
-    } else if (!persist) {
+    if (p.stream || persist) {
+      us = p.dealt0 + range_start(p, blockIdx.x);
+      u1 = p.dealt0 + range_start(p, blockIdx.x + 1);
+    } else {
       const int z = blockIdx.x / p.tiles, pos = blockIdx.x % p.tiles;
       us = pos * p.kblocks + z * p.kb_per_split;
       u1 = min(us + p.kb_per_split, (pos + 1) * p.kblocks);
@@ -91,13 +92,14 @@ struct Segments {
   // next segment: K blocks [kb0, kb0 + nkb) of the output tile at position `pos` of the launch order,
   // which is tile `tile` (m_tile * n_tiles + n_tile); split-K bookkeeping goes by position
   __device__ __forceinline__ bool next(const Params& p, int& pos, int& tile, int& kb0, int& nkb) {
-    if (persist) {
-      if (idx >= p.tiles) return false;
+    if (persist && idx < p.tail_pos0) {
       pos = idx;
       idx += step;
       kb0 = 0;
       nkb = p.kblocks;
     } else {
+      // unit range: all of a streaming CTA's work, or its share of the last, incomplete round of a
+      // persistent launch
       if (us >= u1) return false;
       pos = us / p.kblocks;
       kb0 = us - pos * p.kblocks;
@@ -284,7 +286,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
     // clears its share of y now, while the first tiles are in flight, and announces it; outputs are
     // held back until all CTAs have.
     bool y_ready = p.coop_zero == 0;
-    if (p.coop_zero) {
+    if (p.coop_zero == 1) {
       float* y = static_cast<float*>(p.y);
       const int64_t stride = static_cast<int64_t>(gridDim.x) * C::kEpiThreads;
       const int64_t first = static_cast<int64_t>(blockIdx.x) * C::kEpiThreads + threadIdx.x;
@@ -295,6 +297,20 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       } else {
         for (int64_t i = first; i < static_cast<int64_t>(p.M) * p.N; i += stride) y[(i / p.N) * p.ldy + i % p.N] = 0.0f;
       }
+    } else if (p.coop_zero == 2) {
+      // persistent launch: only the tiles of the last, incomplete round are shared (and added into);
+      // there are fewer of them than CTAs, so CTA c clears the c-th of them
+      const int tpos = p.tail_pos0 + static_cast<int>(blockIdx.x);
+      if (tpos < p.tiles) {
+        const int ttile = raster_tile(p, tpos);
+        const int tm0 = (ttile / p.n_tiles) * BM, tn = (ttile % p.n_tiles) * kTileN + static_cast<int>(threadIdx.x);
+        float* y = static_cast<float*>(p.y) + static_cast<int64_t>(tm0) * p.ldy + tn;
+        const int rows = min(BM, p.M - tm0);
+        if (tn < p.N)
+          for (int r = 0; r < rows; ++r) y[static_cast<int64_t>(r) * p.ldy] = 0.0f;
+      }
+    }
+    if (p.coop_zero) {
       __threadfence();
       named_bar_sync(2, C::kEpiThreads);
       if (threadIdx.x == 0) atomicAdd(p.status + kWsZeroArrive, 1);
@@ -345,7 +361,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
         }
         tc_fence_after_sync();
       }
-      if (!y_ready) {
+      if (!y_ready && (p.coop_zero == 1 || pos >= p.tail_pos0)) {  // tiles before the tail are never cleared
         // every CTA has cleared its share of y (bounded wait; the CTAs of a cooperative launch all run)
         if (threadIdx.x == 0) {
           const uint64_t t0 = global_timer_ns();
@@ -397,7 +413,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
         // arrives last adds all of them in contributor order (deterministic) and finishes the tile.
         int first, count;
         contributors(p, pos, &first, &count);
-        const int my_j = p.stream ? static_cast<int>(blockIdx.x) - first : static_cast<int>(blockIdx.x) / p.tiles;
+        const int my_j = (p.stream || p.persist) ? static_cast<int>(blockIdx.x) - first : static_cast<int>(blockIdx.x) / p.tiles;
         float* my_partial = p.partials + partial_slot(p, pos, first, my_j) * (BM * kTileN);
         if (!failed) {
 #pragma unroll 1
@@ -486,6 +502,21 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
   dim3 grid(static_cast<unsigned>(plan.ctas));
+  if (plan.persist && plan.tail_pos0 < p.tiles && a.ydt == ZQ_OUT_F32) {
+    // The tiles of the last round are shared by all CTAs.  In a cooperative launch the kernel clears
+    // their part of y at its start and the CTAs add into it; otherwise (below) they hand partial sums
+    // over through the workspace.
+    Params pc = p;
+    pc.coop_zero = 2;
+    pc.atomic_y = 1;
+    void* args[3] = {&tm_w, &tm_q, &pc};
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM>), grid, dim3(C::kThreads),
+                                    args, C::kSmemBytes, st) == cudaSuccess) {
+      count_launch();
+      return ZQ_OK;
+    }
+    (void)cudaGetLastError();  // not launched; fall back
+  }
   if (p.atomic_y) {
     // y must be zero before the first CTA adds into it.  A cooperative launch (all CTAs resident, which the
     // plan's grid is sized for) lets the kernel clear y itself; if the device cannot hold the grid at once,

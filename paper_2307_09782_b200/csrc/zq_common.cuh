@@ -80,7 +80,9 @@ struct GemmPlan {
   int bm;      // tokens per tile (the MMA's N extent)
   int m_tiles, n_tiles;
   int stream;  // 1: the (tile, K block) units are dealt out evenly to `ctas` CTAs; 0: tiles x splits CTAs
-  int persist; // 1: `ctas` CTAs walk whole tiles, every ctas-th one (neither stream nor split K)
+  int persist; // 1: `ctas` CTAs walk whole tiles, every ctas-th one, up to position tail_pos0 of the launch
+               //    order; the rest (less than one round) is dealt out as unit ranges (base, rem)
+  int tail_pos0;
   int ctas;
   int splits;        // stream == 0: split-K factor
   int kb_per_split;  // stream == 0: 128-element K blocks per split

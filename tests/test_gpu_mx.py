@@ -74,11 +74,22 @@ def test_linear_many_token_tiles_per_cta():
 
 @pytest.mark.parametrize("M", [1120, 1000])
 def test_linear_persistent_whole_tiles(M):
-    # 600 output tiles, more than four per SM: every CTA walks whole tiles (224 or 192 tokens wide) of
+    # 600 or 720 output tiles, more than four per SM: every CTA walks whole tiles (224 or 192 tokens wide) of
     # different token rows with both accumulator buffers
-    x_bits, W, U, V = _layer(89, M, 128 * 120, 256, 8)
-    rows = [0, 191, 192, 223, 224, 447, 448, 700, M - 1]
+    x_bits, W, U, V = _layer(89, M, 128 * 120, 512, 8)
+    rows = [0, 191, 192, 223, 224, 447, 448, 700, M - 2, M - 1]
     check_linear(x_bits, W, U, V, 128, "M2", layout=MX, rows=rows)
+
+
+@pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
+def test_linear_persistent_last_round_shared(out_dtype):
+    # 600 tiles of 72 K blocks on 148 SMs: four whole rounds, then the 8 tiles of the last round are dealt
+    # out as unit ranges to all CTAs (FP32 y: cleared in the kernel and added into; bf16 y: partial sums
+    # through the workspace)
+    M = 1120
+    x_bits, W, U, V = _layer(90, M, 128 * 120, 9216, 8)
+    rows = [0, 223, 224, 700, M - 1]
+    check_linear(x_bits, W, U, V, 128, "M2", layout=MX, rows=rows, out_dtype=out_dtype)
 
 
 def test_linear_several_token_tiles_dealt_out_as_unit_ranges():
