@@ -648,9 +648,12 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   const int ctas_per_sm = mx ? (bm <= 64 ? 2 : 1) : ((mode == ZQ_SCALE_NONE || bm > 128) ? 1 : (bm <= 16 ? 3 : 2));
   const int64_t resident = static_cast<int64_t>(ctas_per_sm) * sm_count();
   const int64_t units = tiles * kblocks;
-  if (mx && pl.m_tiles > 1 && (tiles >= 4 * resident || tiles > kWsMaxTiles)) {
+  if (mx && ((pl.m_tiles > 1 && (tiles >= 4 * resident || tiles > kWsMaxTiles)) ||
+             (pl.m_tiles == 1 && bm >= 128 && tiles >= resident))) {
     // many tokens: one resident wave of CTAs walks whole tiles (with fewer than four tiles per CTA the
-    // uneven last round would cost too much: those shapes take the contiguous unit ranges below)
+    // uneven last round would cost too much: those shapes take the contiguous unit ranges below).  Also one
+    // row of wide tiles with at least a tile per SM: sharing such tiles costs more (16 K atomic adds per
+    // CTA and tile) than the uneven second round does.
     pl.persist = 1;
     const int64_t g = tiles < resident ? tiles : resident;
     pl.ctas = static_cast<int>(g);
