@@ -159,6 +159,24 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
                    size_t workspace_bytes, void* stream);
 
 /*
+ * How zq_w4a8_linear would partition a problem on the current device (no launch; host only).  Not an
+ * operation of the paper: it exposes the launch plan so that its arithmetic can be checked without a GPU.
+ * Work is counted in units of one 128-element K block of one output tile (128 channels x bm tokens);
+ * positions of the launch order map to tiles through groups of m_group token tiles (N outer, the group's
+ * token tiles inner; m_group <= 1: along N only).
+ *   plan[0] bm, [1] m_tiles, [2] n_tiles, [3] ctas,
+ *   [4] stream  (1: the units are dealt out as contiguous ranges, base each, the first rem CTAs one more),
+ *   [5] persist (1: CTA c walks whole tiles at positions c, c + ctas, ... below tail_pos0; the units of the
+ *                tiles from tail_pos0 on are dealt out as ranges like stream),
+ *   [6] splits, [7] kb_per_split (neither stream nor persist: CTA z * tiles + pos takes K blocks
+ *                [z * kb_per_split, ...) of the tile at position pos),
+ *   [8] base, [9] rem, [10] tail_pos0, [11] m_group, [12] floats of partial-sum scratch, [13] SMs assumed.
+ */
+#define ZQ_PLAN_WORDS 14
+int zq_w4a8_linear_plan(int64_t M, int64_t N, int64_t K, zq_scale_mode mode, zq_weight_layout layout,
+                        int64_t* plan);
+
+/*
  * The same layer for callers whose activations live in HOST memory: copies x (bf16 [M, K] dense,
  * host, ideally pinned) to the device, runs quantizer + linear, copies y (FP32 [M, N] dense, host)
  * back and synchronizes the stream before returning.  Weights, U, V and the workspace stay on the

@@ -26,8 +26,10 @@ EXPORTS = [
     "zq_status_string", "zq_quantize_act_fp8", "zq_packed_weight_sizes", "zq_pack_weight_fp4",
     "zq_w4a8_linear_workspace_bytes", "zq_workspace_init", "zq_w4a8_linear",
     "zq_w4a8_linear_host_workspace_bytes", "zq_w4a8_linear_host", "zq_device_status", "zq_launch_count",
-    "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc",
+    "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc", "zq_w4a8_linear_plan",
 ]
+PLAN_FIELDS = ("bm", "m_tiles", "n_tiles", "ctas", "stream", "persist", "splits", "kb_per_split", "base", "rem",
+               "tail_pos0", "m_group", "partial_floats", "sms")
 
 
 class ZqError(RuntimeError):
@@ -66,6 +68,8 @@ def lib() -> C.CDLL:
                                      i64, vp, sz, vp]
         L.zq_w4a8_linear_host.restype = ci
         L.zq_w4a8_linear_host.argtypes = [vp, i64, i64, i64, ci, ci, ci, vp, vp, vp, vp, vp, ci, vp, vp, sz, vp]
+        L.zq_w4a8_linear_plan.restype = ci
+        L.zq_w4a8_linear_plan.argtypes = [i64, i64, i64, ci, ci, C.POINTER(i64)]
         L.zq_device_status.restype = ci
         L.zq_device_status.argtypes = [vp, C.POINTER(ci), vp]
         L.zq_launch_count.restype = i64
@@ -164,6 +168,13 @@ def pack_weight_fp4(W: torch.Tensor, group: int, mode, layout=WEIGHTS_CAST) -> P
     _check(lib().zq_pack_weight_fp4(_ptr(W), N, K, group, mode, layout, _ptr(codes), _ptr(shift), _ptr(scale),
                                     _stream()), "zq_pack_weight_fp4")
     return PackedWeight(codes, shift, scale, N, K, group, mode, layout)
+
+
+def linear_plan(M: int, N: int, K: int, mode, layout=WEIGHTS_CAST) -> dict:
+    """The launch plan ``zq_w4a8_linear`` would use (host only, nothing is launched)."""
+    out = (C.c_int64 * len(PLAN_FIELDS))()
+    _check(lib().zq_w4a8_linear_plan(M, N, K, _mode(mode), _layout(layout), out), "zq_w4a8_linear_plan")
+    return dict(zip(PLAN_FIELDS, [int(v) for v in out]))
 
 
 def linear_workspace_bytes(M: int, N: int, K: int, r: int) -> int:

@@ -222,6 +222,20 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
   return layout == ZQ_WEIGHTS_MX ? launch_w4a8_mx_gemm(a, st) : launch_w4a8_gemm(a, st);
 }
 
+int zq_w4a8_linear_plan(int64_t M, int64_t N, int64_t K, zq_scale_mode mode, zq_weight_layout layout,
+                        int64_t* plan) {
+  if (!plan) return ZQ_ERR_NULL;
+  if (!valid_mode(mode) || !valid_layout(layout, mode)) return ZQ_ERR_MODE;
+  if (M <= 0 || N <= 0 || K <= 0 || K % 128 || M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > (int64_t(1) << 30))
+    return ZQ_ERR_SHAPE;
+  const GemmPlan pl = plan_gemm(M, N, K, mode, layout);
+  const int64_t v[ZQ_PLAN_WORDS] = {pl.bm,   pl.m_tiles,     pl.n_tiles, pl.ctas, pl.stream,    pl.persist,
+                                    pl.splits, pl.kb_per_split, pl.base,  pl.rem,  pl.tail_pos0, pl.m_group,
+                                    static_cast<int64_t>(pl.partial_floats), sm_count()};
+  for (int i = 0; i < ZQ_PLAN_WORDS; ++i) plan[i] = v[i];
+  return ZQ_OK;
+}
+
 int zq_w4a8_linear_host(const void* x_host, int64_t M, int64_t N, int64_t K, int group, zq_scale_mode mode,
                         zq_weight_layout layout, const uint8_t* codes, const uint8_t* shift, const float* scale, const void* U,
                         const void* V, int r, float* y_host, void* workspace, size_t workspace_bytes,

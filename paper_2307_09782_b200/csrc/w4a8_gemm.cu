@@ -648,6 +648,12 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   const int ctas_per_sm = mx ? (bm <= 64 ? 2 : 1) : ((mode == ZQ_SCALE_NONE || bm > 128) ? 1 : (bm <= 16 ? 3 : 2));
   const int64_t resident = static_cast<int64_t>(ctas_per_sm) * sm_count();
   const int64_t units = tiles * kblocks;
+  // as many token tiles per group of the launch order as keep the group's tokens around 32 MB (they must
+  // stay in L2 while the group walks all of N), at most 8
+  if (pl.m_tiles > 1) {
+    const int64_t fit = (int64_t(32) << 20) / (static_cast<int64_t>(bm) * K);
+    pl.m_group = static_cast<int>(fit < 1 ? 1 : (fit > 8 ? 8 : fit));
+  }
   if (mx && ((pl.m_tiles > 1 && (tiles >= 4 * resident || tiles > kWsMaxTiles)) ||
              (pl.m_tiles == 1 && bm >= 128 && tiles >= resident))) {
     // many tokens: one resident wave of CTAs walks whole tiles (with fewer than four tiles per CTA the

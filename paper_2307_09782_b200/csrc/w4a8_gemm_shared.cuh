@@ -231,13 +231,7 @@ inline Params make_params(const GemmArgs& a, const GemmPlan& plan) {
   p.persist = plan.persist;
   p.tail_pos0 = plan.tail_pos0;
   p.dealt0 = plan.persist ? plan.tail_pos0 * p.kblocks : 0;
-  // as many token tiles per group as keep the group's tokens around 32 MB (they must stay in L2 while the
-  // group walks all of N), at most 8
-  if (plan.m_tiles > 1) {
-    const int64_t tok_tile_bytes = static_cast<int64_t>(plan.bm) * a.K;
-    const int64_t fit = (int64_t(32) << 20) / tok_tile_bytes;
-    p.m_group = static_cast<int>(fit < 1 ? 1 : (fit > 8 ? 8 : fit));
-  }
+  p.m_group = plan.m_group;
   p.atomic_y = (plan.stream && a.ydt == ZQ_OUT_F32 && plan.partial_floats > 0) ? 1 : 0;
   p.splits = plan.splits;
   p.kb_per_split = plan.kb_per_split;

@@ -87,6 +87,7 @@ struct GemmPlan {
   int splits;        // stream == 0: split-K factor
   int kb_per_split;  // stream == 0: 128-element K blocks per split
   int base, rem;     // stream == 1: units per CTA (the first `rem` CTAs take one more)
+  int m_group;       // the launch order runs through groups of this many token tiles (0 or 1: along N only)
   size_t partial_floats;
 };
 GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout);

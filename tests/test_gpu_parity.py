@@ -27,7 +27,8 @@ def test_act_quant_bit_exact(M, K):
 
 
 @pytest.mark.parametrize("M,K,lorc", [(1187, 768, True), (1184, 2048, False), (2500, 256, True), (385, 4096, True),
-                                      (384, 48, True), (300, 16384, True)])
+                                      (384, 48, True), (300, 16384, True), (1030, 7168, True), (520, 28672, True),
+                                      (400, 3584, False), (390, 14336, True), (386, 28704, True)])
 def test_act_quant_many_rows_kernel(M, K, lorc):
     """Token counts large enough for the eight-rows-per-CTA kernel, with a ragged last CTA."""
     x_bits = synth.make_x(300 + M, M, K, max(1, K // 100), 20.0)
