@@ -45,8 +45,8 @@ size_t max_partial_floats(int64_t M, int64_t N, int64_t K) {
   // ranges to one CTA per SM (all of them, or the last round of a persistent launch), each of which
   // leaves at most two partial tiles.
   if (M > 256) {
-    const size_t stream_192 = 2 * static_cast<size_t>(sm_count()) * 256 * 128;
-    if (stream_192 > best) best = stream_192;
+    const size_t dealt_bound = 2 * static_cast<size_t>(sm_count()) * 256 * 128;
+    if (dealt_bound > best) best = dealt_bound;
   }
   return best;
 }

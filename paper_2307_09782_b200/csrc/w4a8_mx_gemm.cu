@@ -17,10 +17,17 @@
 //   D        FP32 in tensor memory, two buffers where they fit, so that the epilogue of one output tile
 //            overlaps the main loop of the next.
 //
-// Orientation, the split-K hand-over and the epilogue are those of the casting kernel.  Work partition:
-// few tokens (one row of output tiles): the (tile, K block) units are dealt out evenly as contiguous ranges
-// to one resident wave of CTAs; many tokens: one CTA per SM walks whole 128 x 192 output tiles, every
-// gridDim.x-th one of the launch order, with both accumulator buffers in use.
+// Orientation, the split-K hand-over and the epilogue are those of the casting kernel.  Work partition
+// (plan_gemm): few tokens or few tiles: the (tile, K block) units are dealt out evenly as contiguous
+// ranges to one resident wave of CTAs; many tokens: one CTA per SM walks whole output tiles of 128
+// channels x 192 / 224 tokens (two accumulator buffers in use) or x 256 tokens (long rows, one buffer),
+// every gridDim.x-th one of the launch order, and the tiles of the last, incomplete round are dealt out
+// as unit ranges again.  Where tiles are shared and y is FP32 the launch is cooperative and the kernel
+// clears the shared part of y itself before anything is added into it.
+//
+// What bounds it: with many tokens, shared-memory bandwidth (the copy engine writes, and the tensor core
+// reads back, 16 KB of padded codes plus 128 bytes per token per K block); with few tokens, HBM
+// latency and the fixed cost of a short kernel, not instruction issue.
 //
 // Warp roles: 0..3 epilogue (one TMEM lane quarter each), 4 producer (one lane issues all copies of a
 // stage onto one barrier), 5 TMEM allocation and MMA issue.
