@@ -134,3 +134,36 @@ def test_both_layouts_agree():
         pw = binding.pack_weight_fp4(up(W), 128, "M2", layout)
         ys.append(host(binding.w4a8_linear(pw, q=q, sx=sx, t=t, U=up(U))))
     assert np.abs(ys[0] - ys[1]).max() <= 1e-5 * np.abs(ys[0]).max()
+
+
+def _fuzz_cases():
+    rng = np.random.default_rng(20230719)
+    cases = []
+    for i in range(28):
+        kind = i % 4
+        if kind == 0:      # decode-like: one narrow row of tiles, long K (unit ranges, shared tiles)
+            M, N, K = int(rng.integers(1, 65)), 128 * int(rng.integers(1, 12)) - int(rng.integers(0, 100)), \
+                128 * int(rng.integers(8, 72))
+        elif kind == 1:    # one row of wide tiles
+            M, N, K = int(rng.integers(65, 257)), 128 * int(rng.integers(1, 40)), 128 * int(rng.integers(1, 20))
+        elif kind == 2:    # several token tiles, few output tiles (unit ranges across token tiles)
+            M, N, K = int(rng.integers(257, 1500)), 128 * int(rng.integers(1, 6)) - int(rng.integers(0, 60)), \
+                128 * int(rng.integers(2, 40))
+        else:              # many tiles: persistent launch, with and without a shared last round
+            M, N, K = int(rng.integers(700, 2400)), 128 * int(rng.integers(60, 130)), 128 * int(rng.integers(1, 4))
+        N = max(N, 1)
+        cases.append((M, N, K, ["M1", "M2"][i % 2], [64, 128, 256][i % 3], [0, 8, 8, 16][i % 4],
+                      torch.float32 if i % 5 else torch.bfloat16))
+    return cases
+
+
+@pytest.mark.parametrize("M,N,K,mode,group,r,out_dtype", _fuzz_cases())
+def test_linear_seeded_random_shapes(M, N, K, mode, group, r, out_dtype):
+    """Seeded random shapes through every branch of the launch plan; sampled token rows against the oracle."""
+    if K % group:
+        K += group - K % group
+    x_bits, W, U, V = _layer(1000 + M + N, M, N, K, r)
+    rng = np.random.default_rng(M * 7 + N)
+    rows = sorted(set([0, M - 1] + [int(v) for v in rng.integers(0, M, 6)] +
+                      [b for b in (191, 192, 223, 224, 255, 256) if b < M]))
+    check_linear(x_bits, W, U, V, group, mode, layout=MX, rows=rows, out_dtype=out_dtype)
