@@ -149,8 +149,9 @@ int zq_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  * M == 0 or N == 0 is a no-op.  Summation order over K depends on the launch shape, so FP32 results are
  * not bit-identical across token counts.  Where the K range of an output tile is shared by several CTAs
  * and y is FP32 (ZQ_WEIGHTS_CAST: M <= 16; ZQ_WEIGHTS_MX: up to 256 tokens, and larger token counts
- * with fewer than about 600 output tiles of 128 x 192) the CTAs add into y with FP32 atomics (y is cleared by
- * the call first): the last bit can then differ from run to run; other shapes, and bf16 y, are reproducible.
+ * with fewer than about 600 output tiles of 128 x 192, and the last round of larger ones) the CTAs add
+ * their shares into y with FP32 atomics: the last bit can then differ from run to run; other shapes, and
+ * bf16 y, are reproducible.
  */
 int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M,
                    int64_t N, int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout,

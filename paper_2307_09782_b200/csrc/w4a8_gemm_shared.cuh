@@ -19,7 +19,7 @@ constexpr int kBlockK = 128;  // K elements per pipeline step
 constexpr int kAStageCols = kBlockK / 4;  // TMEM columns of one widened 128 x 128 tile (4 bytes per column)
 
 // error detail codes written to status[1]
-enum { kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6, kErrZero = 7 };
+enum { kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6, kErrHandover = 7 };
 
 struct Params {
   int M, N, K;
@@ -38,7 +38,8 @@ struct Params {
   int dealt0;    // first unit of the units that are dealt out as ranges (0 when stream == 1)
   int m_group;   // the launch order runs through groups of this many token tiles (see raster_tile)
   int atomic_y;  // streaming launch with FP32 y: CTAs that share a tile add their share into a zeroed y
-  int coop_zero; // cooperative launch: the kernel zeroes y itself and holds every output back until all CTAs have
+  int handover;  // cooperative launch: shared FP32 tiles are handed over through per-tile flags (one CTA stores,
+                 // the others wait for its flag and add), so y needs no clearing
   int splits, kb_per_split;
   int base, rem;
   const uint8_t* codes;  // tiled weight

@@ -22,8 +22,8 @@
 // ranges to one resident wave of CTAs; many tokens: one CTA per SM walks whole output tiles of 128
 // channels x 192 / 224 tokens (two accumulator buffers in use) or x 256 tokens (long rows, one buffer),
 // every gridDim.x-th one of the launch order, and the tiles of the last, incomplete round are dealt out
-// as unit ranges again.  Where tiles are shared and y is FP32 the launch is cooperative and the kernel
-// clears the shared part of y itself before anything is added into it.
+// as unit ranges again.  Where tiles are shared and y is FP32 the launch is cooperative and a shared tile
+// is handed over through a flag: its last contributor stores, the others wait for the flag and add.
 //
 // What bounds it: with many tokens, shared-memory bandwidth (the copy engine writes, and the tensor core
 // reads back, 16 KB of padded codes plus 128 bytes per token per K block); with few tokens, HBM
@@ -289,40 +289,6 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
     bool failed = !ok_start;
     int m0_loaded = -1;
 
-    // Cooperative launch (all CTAs resident at once): instead of a memset before the kernel, every CTA
-    // clears its share of y now, while the first tiles are in flight, and announces it; outputs are
-    // held back until all CTAs have.
-    bool y_ready = p.coop_zero == 0;
-    if (p.coop_zero == 1) {
-      float* y = static_cast<float*>(p.y);
-      const int64_t stride = static_cast<int64_t>(gridDim.x) * C::kEpiThreads;
-      const int64_t first = static_cast<int64_t>(blockIdx.x) * C::kEpiThreads + threadIdx.x;
-      if ((p.N & 3) == 0 && (p.ldy & 3) == 0 && (reinterpret_cast<uintptr_t>(y) & 15u) == 0) {
-        const int n4 = p.N >> 2;
-        for (int64_t i = first; i < static_cast<int64_t>(p.M) * n4; i += stride)
-          *reinterpret_cast<float4*>(y + (i / n4) * p.ldy + (i % n4) * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
-      } else {
-        for (int64_t i = first; i < static_cast<int64_t>(p.M) * p.N; i += stride) y[(i / p.N) * p.ldy + i % p.N] = 0.0f;
-      }
-    } else if (p.coop_zero == 2) {
-      // persistent launch: only the tiles of the last, incomplete round are shared (and added into);
-      // there are fewer of them than CTAs, so CTA c clears the c-th of them
-      const int tpos = p.tail_pos0 + static_cast<int>(blockIdx.x);
-      if (tpos < p.tiles) {
-        const int ttile = raster_tile(p, tpos);
-        const int tm0 = (ttile / p.n_tiles) * BM, tn = (ttile % p.n_tiles) * kTileN + static_cast<int>(threadIdx.x);
-        float* y = static_cast<float*>(p.y) + static_cast<int64_t>(tm0) * p.ldy + tn;
-        const int rows = min(BM, p.M - tm0);
-        if (tn < p.N)
-          for (int r = 0; r < rows; ++r) y[static_cast<int64_t>(r) * p.ldy] = 0.0f;
-      }
-    }
-    if (p.coop_zero) {
-      __threadfence();
-      named_bar_sync(2, C::kEpiThreads);
-      if (threadIdx.x == 0) atomicAdd(p.status + kWsZeroArrive, 1);
-    }
-
     // Every thread walks every segment and executes the same named-barrier sequence whether or not it
     // has failed, so a bounded wait that ran out can never leave others stuck at a hardware barrier.
     for (int seg = 0; sg.next(p, pos, tile, kb0, nkb); ++seg) {
@@ -368,24 +334,6 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
         }
         tc_fence_after_sync();
       }
-      if (!y_ready && (p.coop_zero == 1 || pos >= p.tail_pos0)) {  // tiles before the tail are never cleared
-        // every CTA has cleared its share of y (bounded wait; the CTAs of a cooperative launch all run)
-        if (threadIdx.x == 0) {
-          const uint64_t t0 = global_timer_ns();
-          volatile int* arrived = p.status + kWsZeroArrive;
-          bool ok = false;
-          for (uint32_t spin = 0; spin < kSpinLimit && !ok; ++spin) {
-            ok = *arrived >= static_cast<int>(gridDim.x);
-            if (!ok && (spin & 63u) == 63u && global_timer_ns() - t0 > kWaitLimitNs) break;
-          }
-          if (!ok) raise_error(p, s_abort, kErrZero);
-          __threadfence();
-        }
-        named_bar_sync(2, C::kEpiThreads);
-        y_ready = true;
-        if (*s_abort) failed = true;
-      }
-
       if (nkb == p.kblocks) {
         if (!failed) {
           // the next step's accumulator columns are in flight while this step's are finished
@@ -399,6 +347,47 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
             for (int e = 0; e < EC; ++e) v[e] = nxt[e];
             if (c + EC < BM) tmem_ld_issue<EC>(t_lane + c + EC, nxt);
             if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t);
+          }
+        }
+      } else if (p.atomic_y && p.handover) {
+        // Several CTAs share this tile (FP32 y, cooperative launch: all CTAs are resident).  The tile's last
+        // contributor in K order meets it as the first segment of its range, i.e. early: it STORES its
+        // share (with the LoRC term) and raises the tile's flag.  The others meet the tile at the end of
+        // their ranges: they wait for the flag (long set by then) and ADD their shares.  Nothing has to
+        // clear y first.  The adder that finds all others done leaves the flag at zero for the next call.
+        int first, count;
+        contributors(p, pos, &first, &count);
+        const bool storer = static_cast<int>(blockIdx.x) == first + count - 1;
+        int* flag = p.counters + pos;
+        if (!storer) {
+          if (threadIdx.x == 0) {
+            const uint64_t t0 = global_timer_ns();
+            bool ok = false;
+            for (uint32_t spin = 0; spin < kSpinLimit && !ok; ++spin) {
+              ok = *reinterpret_cast<volatile int*>(flag) != 0 || *s_abort != 0;
+              if (!ok && (spin & 63u) == 63u && global_timer_ns() - t0 > kWaitLimitNs) break;
+            }
+            if (!ok) raise_error(p, s_abort, kErrHandover);
+            __threadfence();
+          }
+          named_bar_sync(2, C::kEpiThreads);
+          if (*s_abort) failed = true;
+        }
+        if (!failed) {
+#pragma unroll 1
+          for (int c = 0; c < BM; c += EC) {
+            float v[EC];
+            tmem_ld_cols<EC>(t_lane + c, v);
+            if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t, !storer, storer);
+          }
+        }
+        __threadfence();  // this thread's stores / adds are performed before the flag moves
+        named_bar_sync(2, C::kEpiThreads);
+        if (threadIdx.x == 0 && !*s_abort) {
+          if (storer) {
+            atomicExch(flag, 1);
+          } else if (atomicAdd(flag, 1) == count - 1) {
+            atomicExch(flag, 0);  // storer + all other adders were counted before this one
           }
         }
       } else if (p.atomic_y) {
@@ -461,13 +450,6 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[buf]);
     }
-    if (p.coop_zero && threadIdx.x == 0) {
-      // this CTA is past the hand-over; the last CTA to get here leaves both counters at zero for the next call
-      if (atomicAdd(p.status + kWsZeroDone, 1) == static_cast<int>(gridDim.x) - 1) {
-        p.status[kWsZeroArrive] = 0;
-        p.status[kWsZeroDone] = 0;
-      }
-    }
   }
 
   tc_fence_before_sync();
@@ -509,13 +491,16 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
   dim3 grid(static_cast<unsigned>(plan.ctas));
-  if (plan.persist && plan.tail_pos0 < p.tiles && a.ydt == ZQ_OUT_F32) {
-    // The tiles of the last round are shared by all CTAs.  In a cooperative launch the kernel clears
-    // their part of y at its start and the CTAs add into it; otherwise (below) they hand partial sums
-    // over through the workspace.
+  const bool shared_f32 =
+      a.ydt == ZQ_OUT_F32 && (p.atomic_y || (plan.persist && plan.tail_pos0 < p.tiles));
+  if (shared_f32) {
+    // Output tiles are shared by CTAs that accumulate into FP32 y.  In a cooperative launch (all CTAs
+    // resident, which the plan's grid is sized for) they hand over through per-tile flags: one stores,
+    // the others wait for it and add.  If the device cannot hold the grid at once: unit ranges -> clear
+    // y with a memset and let every CTA add; persistent launch -> partial sums through the workspace.
     Params pc = p;
-    pc.coop_zero = 2;
     pc.atomic_y = 1;
+    pc.handover = 1;
     void* args[3] = {&tm_w, &tm_q, &pc};
     if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM>), grid, dim3(C::kThreads),
                                     args, C::kSmemBytes, st) == cudaSuccess) {
@@ -523,22 +508,8 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
       return ZQ_OK;
     }
     (void)cudaGetLastError();  // not launched; fall back
-  }
-  if (p.atomic_y) {
-    // y must be zero before the first CTA adds into it.  A cooperative launch (all CTAs resident, which the
-    // plan's grid is sized for) lets the kernel clear y itself; if the device cannot hold the grid at once,
-    // clear y with a memset and launch normally.
-    Params pc = p;
-    pc.coop_zero = 1;
-    void* args[3] = {&tm_w, &tm_q, &pc};
-    if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM>), grid, dim3(C::kThreads),
-                                    args, C::kSmemBytes, st) == cudaSuccess) {
-      count_launch();
-      return ZQ_OK;
-    }
-    (void)cudaGetLastError();  // not launched; fall back
-    if (cudaMemset2DAsync(a.y, static_cast<size_t>(a.ldy) * 4, 0, static_cast<size_t>(a.N) * 4,
-                          static_cast<size_t>(a.M), st) != cudaSuccess)
+    if (p.atomic_y && cudaMemset2DAsync(a.y, static_cast<size_t>(a.ldy) * 4, 0, static_cast<size_t>(a.N) * 4,
+                                        static_cast<size_t>(a.M), st) != cudaSuccess)
       return ZQ_ERR_CUDA;
   }
   w4a8_mx_gemm_kernel<BM><<<grid, C::kThreads, C::kSmemBytes, st>>>(tm_w, tm_q, p);

@@ -15,9 +15,7 @@ void count_launch(int n = 1);  // adds to the process-wide launch counter
 
 // Workspace head: status words the kernels may write (256 bytes), then the split-K tile counters.
 constexpr size_t kWsStatusBytes = 256;
-// status[0] error code, status[1] detail; two counters of the grid-wide hand-over in a cooperative launch
-constexpr int kWsZeroArrive = 8;  // CTAs that have zeroed their share of y
-constexpr int kWsZeroDone = 9;    // CTAs that have finished (the last one clears both)
+// status[0] error code, status[1] detail
 constexpr int kWsMaxTiles = 16384;  // counters: one int per output tile
 constexpr size_t kWsCounterBytes = size_t(kWsMaxTiles) * 4;
 constexpr size_t kWsHeadBytes = kWsStatusBytes + kWsCounterBytes;
