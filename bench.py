@@ -30,10 +30,10 @@ from paper_2307_09782_b200 import synth  # noqa: E402
 
 WORKLOAD = "opt30b"
 GROUP, MODE, RANK = 128, "M2", 8
-# ncu, one pass, the bench's own M = 8192 launches of w4a8_mx_gemm_kernel<224> / <256> (profiles/): 1510.2 MB and 1657.5 MB
-DOMINANT_TRAFFIC = 1583.9e6
+# ncu, one pass, the bench's own M = 8192 launches of w4a8_mx_gemm_kernel<224> / <256> (profiles/): 1510.6 MB and 1655.4 MB
+DOMINANT_TRAFFIC = 1583.0e6
 # ncu --set full, w4a8_mx_gemm_kernel<16> at 7168->28672, M = 8 (profiles/): read + write of the two captured launches
-DECODE_TRAFFIC = 116.8e6
+DECODE_TRAFFIC = 114.6e6
 METRIC = "w4a8_linear_tflops"
 UNIT = "TFLOP/s"
 N_WEIGHT_COPIES = 2  # per layer; rotated so that > 2x the L2 size streams between two reads of one buffer
