@@ -182,7 +182,10 @@ int zq_w4a8_linear_plan(int64_t M, int64_t N, int64_t K, zq_scale_mode mode, zq_
  * host, ideally pinned) to the device, runs quantizer + linear, copies y (FP32 [M, N] dense, host)
  * back and synchronizes the stream before returning.  Weights, U, V and the workspace stay on the
  * device.  The workspace must have zq_w4a8_linear_host_workspace_bytes(M, N, K, r) bytes and must
- * have been zeroed once with zq_workspace_init.
+ * have been zeroed once with zq_workspace_init.  Calls with more than 1024 tokens are cut into row chunks
+ * (token rows are independent) whose upload, kernels and download overlap on two copy streams that the
+ * library creates on first use, per device, and keeps; the kernels still run on `stream`, and everything
+ * has completed when the call returns.
  */
 size_t zq_w4a8_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int r);
 int zq_w4a8_linear_host(const void* x_bf16_host, int64_t M, int64_t N, int64_t K, int group,

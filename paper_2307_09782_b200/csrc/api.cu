@@ -1,6 +1,7 @@
 // C-ABI entry points of libzqfp: argument validation, workspace carving, kernel dispatch.
 // The operations themselves are defined in include/zqfp.h next to their citations.
 #include <atomic>
+#include <mutex>
 
 #include "zq_common.cuh"
 
@@ -236,9 +237,41 @@ int zq_w4a8_linear_plan(int64_t M, int64_t N, int64_t K, zq_scale_mode mode, zq_
   return ZQ_OK;
 }
 
+namespace {
+
+// Copy streams and events of the host-buffer entry point, one set per device, created on first use and
+// kept until the process exits.  Large calls are cut into row chunks so that the upload of chunk i + 1,
+// the kernels of chunk i and the download of chunk i - 1 overlap (token rows are independent).
+constexpr int kHostMaxChunks = 32;
+constexpr int64_t kHostChunkRows = 1024;
+struct HostPipe {
+  bool ok = false;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t entry = nullptr, up[kHostMaxChunks] = {}, done[kHostMaxChunks] = {};
+};
+HostPipe* host_pipe() {
+  static HostPipe pipes[64];
+  static std::once_flag once[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::call_once(once[dev], [dev] {
+    HostPipe& p = pipes[dev];
+    bool ok = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.entry, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < kHostMaxChunks; ++i)
+      ok = cudaEventCreateWithFlags(&p.up[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&p.done[i], cudaEventDisableTiming) == cudaSuccess;
+    p.ok = ok;
+  });
+  return pipes[dev].ok ? &pipes[dev] : nullptr;
+}
+
+}  // namespace
+
 int zq_w4a8_linear_host(const void* x_host, int64_t M, int64_t N, int64_t K, int group, zq_scale_mode mode,
-                        zq_weight_layout layout, const uint8_t* codes, const uint8_t* shift, const float* scale, const void* U,
-                        const void* V, int r, float* y_host, void* workspace, size_t workspace_bytes,
+                        zq_weight_layout layout, const uint8_t* codes, const uint8_t* shift, const float* scale,
+                        const void* U, const void* V, int r, float* y_host, void* workspace, size_t workspace_bytes,
                         void* stream) {
   if (M < 0 || N < 0 || K <= 0 || r < 0) return ZQ_ERR_SHAPE;
   if (M == 0 || N == 0) return ZQ_OK;
@@ -248,16 +281,56 @@ int zq_w4a8_linear_host(const void* x_host, int64_t M, int64_t N, int64_t K, int
   if (workspace_bytes < w.total) return ZQ_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  void* x_dev = ws + w.off_x;
+  uint8_t* x_dev = ws + w.off_x;
   float* y_dev = reinterpret_cast<float*>(ws + w.off_y);
-  if (cudaMemcpyAsync(x_dev, x_host, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+  const uint8_t* xh = static_cast<const uint8_t*>(x_host);
+
+  // chunks of at least kHostChunkRows rows, at most kHostMaxChunks of them
+  int64_t rows = kHostChunkRows;
+  if ((M + rows - 1) / rows > kHostMaxChunks) rows = (M + kHostMaxChunks - 1) / kHostMaxChunks;
+  rows = (rows + 63) / 64 * 64;
+  HostPipe* hp = M > rows ? host_pipe() : nullptr;
+  if (!hp) {
+    // one piece, everything on the caller's stream
+    if (cudaMemcpyAsync(x_dev, xh, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return ZQ_ERR_CUDA;
+    const int e = zq_w4a8_linear(nullptr, nullptr, x_dev, K, M, N, K, group, mode, layout, codes, shift, scale, U, V,
+                                 nullptr, r, y_dev, ZQ_OUT_F32, N, workspace, w.off_x, stream);
+    if (e) return e;
+    if (cudaMemcpyAsync(y_host, y_dev, static_cast<size_t>(M) * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+      return ZQ_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+  }
+
+  // uploads wait for whatever the caller queued before this call
+  if (cudaEventRecord(hp->entry, st) != cudaSuccess || cudaStreamWaitEvent(hp->in, hp->entry, 0) != cudaSuccess)
     return ZQ_ERR_CUDA;
-  const int e = zq_w4a8_linear(nullptr, nullptr, x_dev, K, M, N, K, group, mode, layout, codes, shift, scale, U, V, nullptr,
-                               r, y_dev, ZQ_OUT_F32, N, workspace, w.off_x, stream);
-  if (e) return e;
-  if (cudaMemcpyAsync(y_host, y_dev, static_cast<size_t>(M) * N * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
-    return ZQ_ERR_CUDA;
-  return cudaStreamSynchronize(st) == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+  int rc = ZQ_OK;
+  int c = 0;
+  for (int64_t m0 = 0; m0 < M && rc == ZQ_OK; m0 += rows, ++c) {
+    const int64_t mc = M - m0 < rows ? M - m0 : rows;
+    uint8_t* xd = x_dev + static_cast<size_t>(m0) * K * 2;
+    float* yd = y_dev + static_cast<size_t>(m0) * N;
+    if (cudaMemcpyAsync(xd, xh + static_cast<size_t>(m0) * K * 2, static_cast<size_t>(mc) * K * 2,
+                        cudaMemcpyHostToDevice, hp->in) != cudaSuccess ||
+        cudaEventRecord(hp->up[c], hp->in) != cudaSuccess || cudaStreamWaitEvent(st, hp->up[c], 0) != cudaSuccess) {
+      rc = ZQ_ERR_CUDA;
+      break;
+    }
+    rc = zq_w4a8_linear(nullptr, nullptr, xd, K, mc, N, K, group, mode, layout, codes, shift, scale, U, V, nullptr, r, yd,
+                        ZQ_OUT_F32, N, workspace, w.off_x, stream);
+    if (rc) break;
+    if (cudaEventRecord(hp->done[c], st) != cudaSuccess || cudaStreamWaitEvent(hp->out, hp->done[c], 0) != cudaSuccess ||
+        cudaMemcpyAsync(y_host + static_cast<size_t>(m0) * N, yd, static_cast<size_t>(mc) * N * 4,
+                        cudaMemcpyDeviceToHost, hp->out) != cudaSuccess)
+      rc = ZQ_ERR_CUDA;
+  }
+  // the call is synchronous: nothing of it is left in flight, also after an error
+  const bool s1 = cudaStreamSynchronize(hp->in) == cudaSuccess;
+  const bool s2 = cudaStreamSynchronize(st) == cudaSuccess;
+  const bool s3 = cudaStreamSynchronize(hp->out) == cudaSuccess;
+  if (rc) return rc;
+  return (s1 && s2 && s3) ? ZQ_OK : ZQ_ERR_CUDA;
 }
 
 int zq_device_status(void* workspace, int* detail, void* stream) {

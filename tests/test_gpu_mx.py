@@ -167,3 +167,26 @@ def test_linear_seeded_random_shapes(M, N, K, mode, group, r, out_dtype):
     rows = sorted(set([0, M - 1] + [int(v) for v in rng.integers(0, M, 6)] +
                       [b for b in (191, 192, 223, 224, 255, 256) if b < M]))
     check_linear(x_bits, W, U, V, group, mode, layout=MX, rows=rows, out_dtype=out_dtype)
+
+
+@pytest.mark.parametrize("layout", [binding.WEIGHTS_CAST, MX])
+def test_host_buffer_entry_point_in_row_chunks(layout):
+    # more than 1024 tokens: the host entry uploads, computes and downloads in overlapping row chunks
+    M, N, K, r = 2600, 384, 512, 8
+    x_bits, W, U, V = _layer(96, M, N, K, r)
+    pw = binding.pack_weight_fp4(up(W), 128, "M2", layout)
+    ws = binding.make_workspace(binding.linear_host_workspace_bytes(M, N, K, r))
+    xh = torch.from_numpy(x_bits.view(np.int16)).view(torch.bfloat16).pin_memory()
+    yh = torch.full((M, N), float("nan"), dtype=torch.float32).pin_memory()
+    for _ in range(2):   # the second call reuses the copy streams
+        binding.w4a8_linear_host(xh, yh, pw, U=up(U), V=up(V), workspace=ws)
+    assert binding.device_status(ws) == (0, 0)
+    q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
+    c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, 128, "M2")
+    rows = [0, 1023, 1024, 2047, 2048, 2599] + list(range(1000, 1100, 7))
+    y_o = oracle.w4a8_linear(q_o, sx_o, c_o, sh_o, sc_o, 128, "M2", U, t_o, rows=rows)
+    assert not np.isnan(yh.numpy()).any()
+    assert np.abs(yh.numpy()[rows] - y_o).max() <= TOL_REL * np.abs(y_o).max()
+    # the same numbers as the device entry point up to summation order
+    y_d = host(binding.w4a8_linear(pw, x=to_bf16(x_bits), U=up(U), V=up(V)))
+    assert np.abs(yh.numpy() - y_d).max() <= 1e-5 * np.abs(y_d).max()
