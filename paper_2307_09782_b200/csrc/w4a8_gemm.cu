@@ -655,11 +655,13 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
     pl.m_group = static_cast<int>(fit < 1 ? 1 : (fit > 8 ? 8 : fit));
   }
   if (mx && ((pl.m_tiles > 1 && (tiles >= 4 * resident || tiles > kWsMaxTiles)) ||
-             (pl.m_tiles == 1 && bm >= 128 && tiles >= resident))) {
+             (pl.m_tiles == 1 && bm >= 128 && tiles >= resident) ||
+             (pl.m_tiles == 1 && bm < 128 && 4 * tiles >= 3 * resident))) {
     // many tokens: one resident wave of CTAs walks whole tiles (with fewer than four tiles per CTA the
     // uneven last round would cost too much: those shapes take the contiguous unit ranges below).  Also one
-    // row of wide tiles with at least a tile per SM: sharing such tiles costs more (16 K atomic adds per
-    // CTA and tile) than the uneven second round does.
+    // row of tiles that fills at least three quarters of a resident wave (a full one for wide tiles): a CTA
+    // that shares tiles runs two epilogues and a hand-over, which measured dearer than the idle slots
+    // (7168 -> 28672: 31.6 -> 26.7 us at 8 tokens, 41 -> 29 us at 32, 60 -> 47 us at 128).
     pl.persist = 1;
     const int64_t g = tiles < resident ? tiles : resident;
     pl.ctas = static_cast<int>(g);
