@@ -52,7 +52,7 @@ typedef enum {
 const char* zq_status_string(int status);
 
 /*
- * Token-wise FP8 activation quantization (Section 3: "token-wise quantization for activation";
+ * Token-wise FP8 activation quantization (Section 3, the activation quantizer of the W4A8 scheme;
  * Appendix A; symmetric, i.e. Eq. 1 with Z = 0, in the E4M3 format of Section 2 / 4).
  *
  *   a_m = max_k |x[m,k]| ;  sx[m] = a_m / 448 ;  q[m,k] = RNE_E4M3( fl32( x[m,k] * fl32(448 / a_m) ) )
@@ -218,15 +218,19 @@ int zq_device_status(void* workspace, int* detail, void* stream);
  * tiles are not split and always fit; so do the M <= 128 cases of layers up to 28672 x 28672.
  * The first call on a device looks up the array's device address (once per device, with that device
  * current); make that first call outside any stream capture.
- * Every call on a device shares the one array: the call clears the status words and counters it needs
- * at zero, but two calls that overlap on the GPU race on it, so issue them on one stream or
- * serialize them yourself.
+ * Every call on a device shares the one array: the call clears the counters it needs at zero, but two
+ * calls that overlap on the GPU race on it, so issue them on one stream or serialize them yourself.
+ * The workspace of zq_device_status does not exist here; zq_w4a8_linear_noalloc_status is its counterpart:
+ * it synchronizes `stream`, reads the status words at the head of the array on the current device and
+ * clears them; ZQ_OK, or ZQ_ERR_DEVICE_TIMEOUT with `detail` (host, may be NULL) naming the wait that ran
+ * out in some call since the last query (that call's y is invalid).  It allocates nothing either.
  */
 size_t zq_w4a8_linear_noalloc_max_scratch_bytes(void);
 int zq_w4a8_linear_noalloc(const uint8_t* q, const float* sx, int64_t M, int64_t N, int64_t K, int group,
                            zq_scale_mode mode, const uint8_t* codes, const uint8_t* shift,
                            const float* scale, const void* U_f16, const float* t, int r, void* y,
                            zq_out_dtype ydt, int64_t ldy, void* stream);
+int zq_w4a8_linear_noalloc_status(int* detail, void* stream);
 
 /* Number of kernels of this library launched by the calling process so far (all entry points). */
 int64_t zq_launch_count(void);

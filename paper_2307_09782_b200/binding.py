@@ -26,7 +26,7 @@ EXPORTS = [
     "zq_status_string", "zq_quantize_act_fp8", "zq_packed_weight_sizes", "zq_pack_weight_fp4",
     "zq_w4a8_linear_workspace_bytes", "zq_workspace_init", "zq_w4a8_linear",
     "zq_w4a8_linear_host_workspace_bytes", "zq_w4a8_linear_host", "zq_device_status", "zq_launch_count",
-    "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc", "zq_w4a8_linear_plan",
+    "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc", "zq_w4a8_linear_noalloc_status", "zq_w4a8_linear_plan",
 ]
 PLAN_FIELDS = ("bm", "m_tiles", "n_tiles", "ctas", "stream", "persist", "splits", "kb_per_split", "base", "rem",
                "tail_pos0", "m_group", "partial_floats", "sms")
@@ -78,6 +78,8 @@ def lib() -> C.CDLL:
         L.zq_w4a8_linear_noalloc_max_scratch_bytes.argtypes = []
         L.zq_w4a8_linear_noalloc.restype = ci
         L.zq_w4a8_linear_noalloc.argtypes = [vp, vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, ci, vp, ci, i64, vp]
+        L.zq_w4a8_linear_noalloc_status.restype = ci
+        L.zq_w4a8_linear_noalloc_status.argtypes = [C.POINTER(ci), vp]
         _lib = L
     return _lib
 
@@ -228,6 +230,13 @@ def w4a8_linear_noalloc(w: PackedWeight, *, q, sx, t=None, U=None, y=None, out_d
                                         _ptr(scale), _ptr(U), _ptr(t), r, _ptr(y), ydt, ldy, _stream()),
            "zq_w4a8_linear_noalloc")
     return y
+
+
+def noalloc_status():
+    """Synchronizes the current stream; returns (status, detail) of the fixed scratch array and clears them."""
+    d = C.c_int(0)
+    st = lib().zq_w4a8_linear_noalloc_status(C.byref(d), _stream())
+    return int(st), int(d.value)
 
 
 def w4a8_linear_host(x_host: torch.Tensor, y_host: torch.Tensor, w: PackedWeight, *, U=None, V=None,

@@ -10,17 +10,17 @@ namespace zq {
 static std::atomic<int64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
-namespace {
-
-inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
-
 int check_device_sm100() {
   int dev = 0, major = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return ZQ_ERR_CUDA;
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return ZQ_ERR_CUDA;
   return major == 10 ? ZQ_OK : ZQ_ERR_ARCH;
 }
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 bool valid_mode(int mode) { return mode == ZQ_SCALE_NONE || mode == ZQ_SCALE_M1 || mode == ZQ_SCALE_M2; }
 bool valid_group(int g) { return g == 64 || g == 128 || g == 256; }
@@ -29,25 +29,40 @@ bool valid_layout(int layout, int mode) {
   return layout == ZQ_WEIGHTS_CAST || (layout == ZQ_WEIGHTS_MX && mode != ZQ_SCALE_NONE);
 }
 inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
+// the sizes every linear entry point and size query accepts (the group size is checked where it is known)
+bool valid_linear_shape(int64_t M, int64_t N, int64_t K, int r) {
+  return M >= 0 && N >= 0 && K > 0 && K % 128 == 0 && r >= 0 && r <= 64 && r % 8 == 0 && M <= 0x7FFFFFFF &&
+         N <= 0x7FFFFFFF && K <= (int64_t(1) << 30);
+}
 
 // Largest split-K scratch any token count up to M can need at this (N, K), over both kernel families.
+// The plan depends on the token count only through the tile width and the number of token tiles, i.e.
+// through ceil(m / 192), ceil(m / 224), ceil(m / 256) and a few thresholds up to 256: it is evaluated on
+// both sides of every such breakpoint up to 65536 tokens; beyond that an upper bound of every plan is
+// taken as well (no plan has more than 4 x SMs contributors of a 256 x 128 tile).
 size_t max_partial_floats(int64_t M, int64_t N, int64_t K) {
   size_t best = 0;
-  const int64_t cand[8] = {16, 32, 64, 128, 192, 224, 256, M};
-  for (int variant = 0; variant < 3; ++variant)
-    for (int i = 0; i < 8; ++i) {
-      const int64_t m = cand[i] < M ? cand[i] : M;
-      if (m <= 0) continue;
+  if (M <= 0 || N <= 0) return 0;
+  auto probe = [&](int64_t m) {
+    if (m <= 0 || m > M) return;
+    for (int variant = 0; variant < 3; ++variant) {
       const GemmPlan pl = plan_gemm(m, N, K, variant == 0 ? ZQ_SCALE_NONE : ZQ_SCALE_M1,
                                     variant == 2 ? ZQ_WEIGHTS_MX : ZQ_WEIGHTS_CAST);
       if (pl.partial_floats > best) best = pl.partial_floats;
     }
-  // Beyond 256 tokens the block-scaled kernel may deal tiles of up to 256 tokens out as contiguous unit
-  // ranges to one CTA per SM (all of them, or the last round of a persistent launch), each of which
-  // leaves at most two partial tiles.
-  if (M > 256) {
-    const size_t dealt_bound = 2 * static_cast<size_t>(sm_count()) * 256 * 128;
-    if (dealt_bound > best) best = dealt_bound;
+  };
+  const int64_t small[10] = {16, 32, 64, 128, 129, 192, 193, 224, 256, M};
+  for (int i = 0; i < 10; ++i) probe(small[i]);
+  const int64_t top = M < 65536 ? M : 65536;
+  const int widths[3] = {192, 224, 256};
+  for (int w = 0; w < 3; ++w)
+    for (int64_t m = widths[w]; m <= top; m += widths[w]) {
+      probe(m);
+      probe(m + 1);
+    }
+  if (M > 65536) {
+    const size_t bound = 4 * static_cast<size_t>(sm_count()) * 256 * 128;
+    if (bound > best) best = bound;
   }
   return best;
 }
@@ -139,12 +154,12 @@ int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale
 }
 
 size_t zq_w4a8_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int r) {
-  if (M < 0 || N < 0 || K <= 0 || r < 0) return 0;
+  if (!valid_linear_shape(M, N, K, r)) return 0;
   return ws_layout(M, N, K, r, false).total;
 }
 
 size_t zq_w4a8_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K, int r) {
-  if (M < 0 || N < 0 || K <= 0 || r < 0) return 0;
+  if (!valid_linear_shape(M, N, K, r)) return 0;
   return ws_layout(M, N, K, r, true).total;
 }
 
@@ -162,9 +177,7 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
                    void* y, zq_out_dtype ydt, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
   if (!valid_mode(mode) || !valid_layout(layout, mode) || (ydt != ZQ_OUT_F32 && ydt != ZQ_OUT_BF16))
     return ZQ_ERR_MODE;
-  if (M < 0 || N < 0 || K <= 0 || K % 128 || !valid_group(group) || K % group || r < 0 || r > 64 || r % 8 ||
-      ldy < N || M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > (int64_t(1) << 30))
-    return ZQ_ERR_SHAPE;
+  if (!valid_linear_shape(M, N, K, r) || !valid_group(group) || K % group || ldy < N) return ZQ_ERR_SHAPE;
   if (M == 0 || N == 0) return ZQ_OK;
   if (!codes || !scale || !y || (r > 0 && !U)) return ZQ_ERR_NULL;
   if (x_bf16) {
@@ -273,7 +286,8 @@ int zq_w4a8_linear_host(const void* x_host, int64_t M, int64_t N, int64_t K, int
                         zq_weight_layout layout, const uint8_t* codes, const uint8_t* shift, const float* scale,
                         const void* U, const void* V, int r, float* y_host, void* workspace, size_t workspace_bytes,
                         void* stream) {
-  if (M < 0 || N < 0 || K <= 0 || r < 0) return ZQ_ERR_SHAPE;
+  if (!valid_mode(mode) || !valid_layout(layout, mode)) return ZQ_ERR_MODE;
+  if (!valid_linear_shape(M, N, K, r) || !valid_group(group) || K % group) return ZQ_ERR_SHAPE;
   if (M == 0 || N == 0) return ZQ_OK;
   if (!x_host || !y_host) return ZQ_ERR_NULL;
   if (!workspace) return ZQ_ERR_WORKSPACE;

@@ -71,13 +71,16 @@ int zq_w4a8_linear_noalloc(const uint8_t* q, const float* sx, int64_t M, int64_t
   const GemmPlan pl = plan_gemm(M, N, K, mode, ZQ_WEIGHTS_CAST);
   if (pl.partial_floats > kScratchPartialFloats || pl.ctas <= 0) return ZQ_ERR_WORKSPACE;
 
+  if (int e = check_device_sm100()) return e;
   void* scratch = nullptr;
   if (int e = scratch_address(&scratch)) return e;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // the array keeps whatever the last call left: the status words and tile counters must start at zero
-  if (cudaMemsetAsync(scratch, 0, kWsHeadBytes, st) != cudaSuccess) return ZQ_ERR_CUDA;
-
   unsigned char* base = static_cast<unsigned char*>(scratch);
+  // The array keeps whatever the last call left: the tile counters must start at zero.  The status words
+  // are left alone, so that an error recorded by an earlier call stays readable until
+  // zq_w4a8_linear_noalloc_status fetches (and clears) it.
+  if (cudaMemsetAsync(base + kWsStatusBytes, 0, kWsCounterBytes, st) != cudaSuccess) return ZQ_ERR_CUDA;
+
   GemmArgs a{};
   a.q = q;
   a.sx = sx;
@@ -100,6 +103,19 @@ int zq_w4a8_linear_noalloc(const uint8_t* q, const float* sx, int64_t M, int64_t
   a.partials = reinterpret_cast<float*>(base + kWsHeadBytes);
   a.partial_floats = kScratchPartialFloats;
   return launch_w4a8_gemm(a, st);
+}
+
+int zq_w4a8_linear_noalloc_status(int* detail, void* stream) {
+  void* scratch = nullptr;
+  if (int e = scratch_address(&scratch)) return e;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int words[2] = {0, 0};
+  if (cudaMemcpyAsync(words, scratch, sizeof(words), cudaMemcpyDeviceToHost, st) != cudaSuccess) return ZQ_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return ZQ_ERR_CUDA;
+  if (detail) *detail = words[1];
+  if (words[0] == 0) return ZQ_OK;
+  if (cudaMemsetAsync(scratch, 0, 8, st) != cudaSuccess) return ZQ_ERR_CUDA;
+  return ZQ_ERR_DEVICE_TIMEOUT;
 }
 
 }  // extern "C"

@@ -644,6 +644,7 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   pl.n_tiles = static_cast<int>((N + kTileN - 1) / kTileN);
   const int64_t tiles = static_cast<int64_t>(pl.m_tiles) * pl.n_tiles;
   const int kblocks = static_cast<int>(K / kBlockK);
+  if (tiles <= 0 || kblocks <= 0) return pl;  // nothing to do: an empty plan (ctas == 0)
   // CTAs per SM the kernel family is sized for at this tile
   const int ctas_per_sm = mx ? (bm <= 64 ? 2 : 1) : ((mode == ZQ_SCALE_NONE || bm > 128) ? 1 : (bm <= 16 ? 3 : 2));
   const int64_t resident = static_cast<int64_t>(ctas_per_sm) * sm_count();

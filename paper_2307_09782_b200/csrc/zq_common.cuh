@@ -12,6 +12,7 @@ namespace zq {
 
 // ---- host-side bookkeeping ---------------------------------------------------------------------
 void count_launch(int n = 1);  // adds to the process-wide launch counter
+int check_device_sm100();      // ZQ_OK when the current device is compute capability 10.x
 
 // Workspace head: status words the kernels may write (256 bytes), then the split-K tile counters.
 constexpr size_t kWsStatusBytes = 256;

@@ -47,6 +47,27 @@ def test_size_queries(L):
     assert small >= 256 + 4 * 16384
     assert binding.linear_workspace_bytes(8192, 28672, 7168, 8) >= 8192 * 7168
     assert binding.linear_host_workspace_bytes(16, 768, 768, 0) >= small + 16 * 768 * 2 + 16 * 768 * 4
+    # sizes the linear entry points refuse give 0, and degenerate ones do not crash the host process
+    for fn in (binding.linear_workspace_bytes, binding.linear_host_workspace_bytes):
+        assert fn(16, 128, 64, 0) == 0       # K below one 128-element block
+        assert fn(16, 128, 192, 0) == 0      # K not a multiple of 128
+        assert fn(16, 128, 256, 12) == 0     # rank not a multiple of 8
+        assert fn(-1, 128, 256, 0) == 0
+        assert fn(16, 0, 128, 0) >= 256 + 4 * 16384    # N == 0 is a no-op of the linear call: head only
+        assert fn(0, 128, 128, 0) >= 256 + 4 * 16384
+
+
+def test_workspace_serves_every_smaller_token_count(L):
+    # a workspace sized for M tokens must hold the split-K scratch of every plan up to M tokens
+    for (N, K) in [(7552, 1024), (7168, 28672), (2048, 8192), (640, 4096)]:
+        big = binding.linear_workspace_bytes(8192, N, K, 8)
+        for M in [1, 16, 17, 100, 128, 129, 192, 193, 256, 257, 448, 449, 1280, 1281, 2047, 4097, 8191]:
+            assert binding.linear_workspace_bytes(M, N, K, 8) <= big, (N, K, M)
+            for mode, layout in (("none", "cast"), ("M1", "cast"), ("M1", "mx")):
+                pl = binding.linear_plan(M, N, K, mode, layout)
+                # head + partial sums + q + sx + t for M tokens fit the 8192-token workspace
+                need = 256 + 4 * 16384 + 4 * pl["partial_floats"] + M * K + 4 * M + 32 * M
+                assert need <= big, (N, K, M, mode, layout)
 
 
 def test_validation_before_launch(L):
@@ -92,5 +113,16 @@ def test_validation_before_launch(L):
     assert call(ws=null) == -5
     assert call(wsb=1024) == -5
     assert call(M=0) == 0
+    assert call(N=0, ldy=0) == 0
+    # the host-buffer entry point validates the same way
+    def host_call(**kw):
+        a = dict(args, **kw)
+        return L.zq_w4a8_linear_host(fake, a["M"], a["N"], a["K"], a["group"], a["mode"], a["layout"], a["codes"],
+                                     a["shift"], a["scale"], a["U"], a["V"], a["r"], fake, a["ws"], a["wsb"], a["st"])
+    assert host_call(K=64) == -2
+    assert host_call(N=0) == 0
+    assert host_call(group=96) == -2
+    assert host_call(mode=9) == -4
+    assert host_call(ws=null) == -5
     assert L.zq_workspace_init(null, 1 << 20, null) == -1
     assert L.zq_workspace_init(fake, 16, null) == -5

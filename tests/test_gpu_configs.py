@@ -1,9 +1,13 @@
 """GPU parity at the full sizes of the five workload configurations, in the launch shapes bench.py times.
 
 Every packed FP4 code, shift, scale, FP8 activation code and token scale is compared bit for bit with the
-oracle on the whole tensor.  Outputs are compared on sampled token rows (first, last, tile boundaries, a few
-seeded random rows; all N columns of each) within 1e-3 * max|y| over the sampled rows, because the FP64
-oracle needs about a second per row at these sizes.
+oracle on the whole tensor.  Outputs are compared on sampled token rows, all N columns of each, within
+1e-3 * max|y| over the sampled rows, because the FP64 oracle needs a fraction of a second per row at these
+sizes.  The sample of a case is built from the token-tile width the launch plan really picks for each weight
+layout (asked from zq_w4a8_linear_plan): the first and the last row, both rows at every tile boundary, one
+seeded row inside every token tile, and 32 further seeded rows; up to 64 tokens every row is compared.
+The LoRC-off variant of a case runs the same kernels with another epilogue branch, so it takes the
+boundaries of the first two and the last tile plus 8 seeded rows.
 """
 import numpy as np
 import pytest
@@ -16,19 +20,27 @@ from gpu_util import TOL_REL, check_packed, host, to_bf16, up
 pytestmark = pytest.mark.gpu
 
 
-def _sample_rows(M, bm, k, seed):
-    rows = {0, M - 1}
-    for b in (bm, 2 * bm):
-        for r in (b - 1, b):
-            if 0 <= r < M:
-                rows.add(r)
+def _sample_rows(M, bms, seed, full=True):
+    """Token rows to compare: see the module docstring.  `bms`: tile widths in use (one per weight layout)."""
+    if M <= 64:
+        return list(range(M))
     rng = np.random.default_rng(seed)
-    while len(rows) < min(k, M):
-        rows.add(int(rng.integers(0, M)))
-    return sorted(rows)[:max(k, 1)] if M > k else sorted(rows)
+    rows = {0, M - 1}
+    for bm in bms:
+        n_tiles = (M + bm - 1) // bm
+        tiles = range(n_tiles) if full else sorted({0, 1, n_tiles - 1})
+        for ti in tiles:
+            lo, hi = ti * bm, min((ti + 1) * bm, M)
+            rows.update((lo, hi - 1))
+            if lo > 0:
+                rows.add(lo - 1)
+            if full:
+                rows.add(int(rng.integers(lo, hi)))
+    rows.update(int(v) for v in rng.integers(0, M, size=32 if full else 8))
+    return sorted(rows)
 
 
-def _run_layer(wl, shape, modes, Ms, rows_per_case, lorc_variants=(True,)):
+def _run_layer(wl, shape, modes, Ms, lorc_variants=(True,)):
     K, N = shape.K, shape.N
     Mmax = max(Ms)
     x_bits = synth.make_x(wl.seed, Mmax, K, wl.n_outliers(K), wl.outlier_factor)
@@ -60,11 +72,8 @@ def _run_layer(wl, shape, modes, Ms, rows_per_case, lorc_variants=(True,)):
         for M in Ms:
             for with_lorc in lorc_variants:
                 use = bool(r) and with_lorc
-                bm = 16
-                while bm < 256 and bm < M:
-                    bm *= 2
-                rows = sorted(set(_sample_rows(M, bm, rows_per_case, 1000 + M)) |
-                              {r_ for r_ in (191, 192) if r_ < M})
+                bms = sorted({binding.linear_plan(M, N, K, mode, pw.layout)["bm"] for pw in pws})
+                rows = _sample_rows(M, bms, 1000 + M, full=with_lorc or not r)
                 y_o = oracle.w4a8_linear(q_o[:M], sx_o[:M], c_o, sh_o, sc_o, wl.group, mode, U if use else None,
                                          t_o[:M] if use else None, rows=rows)
                 for pw in pws:
@@ -79,28 +88,28 @@ def _run_layer(wl, shape, modes, Ms, rows_per_case, lorc_variants=(True,)):
 
 def test_config_opt125m():
     wl = synth.WORKLOADS["opt125m"]
-    _run_layer(wl, wl.shapes[0], wl.modes, wl.Ms, rows_per_case=16)
+    _run_layer(wl, wl.shapes[0], wl.modes, wl.Ms)
 
 
 @pytest.mark.parametrize("i", [0, 1, 2])
 def test_config_opt1_3b(i):
     wl = synth.WORKLOADS["opt1.3b"]
-    _run_layer(wl, wl.shapes[i], wl.modes, wl.Ms, rows_per_case=8)
+    _run_layer(wl, wl.shapes[i], wl.modes, wl.Ms)
 
 
 @pytest.mark.parametrize("i", [0, 1, 2])
 def test_config_llama7b(i):
     wl = synth.WORKLOADS["llama7b"]
-    _run_layer(wl, wl.shapes[i], wl.modes, wl.Ms, rows_per_case=5)
+    _run_layer(wl, wl.shapes[i], wl.modes, wl.Ms)
 
 
 @pytest.mark.parametrize("i", [0, 1])
 def test_config_llama30b(i):
     wl = synth.WORKLOADS["llama30b"]
-    _run_layer(wl, wl.shapes[i], wl.modes, wl.Ms, rows_per_case=4)
+    _run_layer(wl, wl.shapes[i], wl.modes, wl.Ms)
 
 
 @pytest.mark.parametrize("i", [0, 1])
 def test_config_opt30b(i):
     wl = synth.WORKLOADS["opt30b"]
-    _run_layer(wl, wl.shapes[i], wl.modes, wl.Ms, rows_per_case=5, lorc_variants=(True, False))
+    _run_layer(wl, wl.shapes[i], wl.modes, wl.Ms, lorc_variants=(True, False))
