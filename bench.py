@@ -1,13 +1,19 @@
 """Benchmark of the W4A8 quantized linear layer (FP4 weights, FP8 activations, LoRC) on B200.
 
-A step is one pass of the whole hot path (token-wise FP8 quantization with the LoRC down-projection,
+A step is SWEEPS passes of the whole hot path (token-wise FP8 quantization with the LoRC down-projection,
 then the W4A8 GEMM with its scale + LoRC epilogue) over the OPT-30B-shaped sweep: the two MLP layers
-(7168 -> 28672 and 28672 -> 7168), each at M in {1, 8, 32, 128, 512, 2048, 8192} tokens, constraint M2,
-group 128, LoRC rank 8.  Weights are packed once before the timed region.
+(7168 -> 28672 and 28672 -> 7168), each at M in {8192, 2048, 512, 128, 32, 8, 1} tokens, constraint M2,
+group 128, LoRC rank 8.  Weights are packed once before the timed region.  A layer call is
+zq_w4a8_linear on raw bf16 activations (the library runs its quantizer and then the GEMM); the calls at the
+largest token count are issued as quantizer call + GEMM call so that CUDA events can bracket the dominant
+GEMM kernel inside the timed region.  The sweep runs from many tokens to few: a decode-size call right
+after the 8192-token GEMM would be timed while that kernel's 235 MB of output is still being written back
+from L2 (measured: 35 us instead of 27 us for the same launch).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-cpu-baseline]
 
 Prints one JSON line.  `--impl reference` times the CPU oracle on a bounded sample of the same workload.
+With --gpus N > 1 outside a torchrun environment the script starts the N ranks itself.
 """
 from __future__ import annotations
 
@@ -30,10 +36,12 @@ from paper_2307_09782_b200 import synth  # noqa: E402
 
 WORKLOAD = "opt30b"
 GROUP, MODE, RANK = 128, "M2", 8
-# ncu, one pass, the bench's own M = 8192 launches of w4a8_mx_gemm_kernel<224> / <256> (profiles/): 1510.6 MB and 1655.4 MB
-DOMINANT_TRAFFIC = 1583.0e6
-# ncu --set full, w4a8_mx_gemm_kernel<16> at 7168->28672, M = 8 (profiles/): read + write of the two captured launches
-DECODE_TRAFFIC = 114.6e6
+NOMINAL_FP8_TFLOPS = 4500.0  # public dense FP8 figure of the part, for context
+# DRAM bytes per launch from the ncu captures summarised under profiles/ (null when the kernel changed since)
+DOMINANT_TRAFFIC = None
+DECODE_TRAFFIC = None
+# LLaMA-7B-shaped rows outside the timed step: (scale mode, weight layout)
+EXTRA_LLAMA7B = (("none", "cast"), ("M2", "mx"))
 METRIC = "w4a8_linear_tflops"
 UNIT = "TFLOP/s"
 N_WEIGHT_COPIES = 2  # per layer; rotated so that > 2x the L2 size streams between two reads of one buffer
@@ -43,13 +51,18 @@ def flops(M, N, K, r):
     return 2.0 * M * N * K + 2.0 * M * r * (K + N)
 
 
-def algorithmic_bytes(M, N, K, r, group=GROUP):
-    """Bytes the fused path must move (M1/M2, FP32 y): codes, shifts, channel scales, x, y, U, V."""
-    return N * K / 2 + N * K / group + 4 * N + 2 * M * K + 4 * M * N + 2 * r * (N + K)
-
-
 def weight_bytes(N, K, group=GROUP):
     return N * K / 2 + N * K / group + 4 * N
+
+
+def layer_bytes(M, N, K, r, group=GROUP):
+    """Bytes the whole layer must move (M1 / M2, FP32 y): codes, shifts, channel scales, x, y, U, V."""
+    return weight_bytes(N, K, group) + 2 * M * K + 4 * M * N + 2 * r * (N + K)
+
+
+def gemm_bytes(M, N, K, r, group=GROUP):
+    """Bytes of the GEMM alone on pre-quantized activations: weights, q, sx, t, y, U."""
+    return weight_bytes(N, K, group) + M * K + 4 * M + 4 * M * r + 4 * M * N + 2 * r * N
 
 
 def load_peaks():
@@ -139,6 +152,12 @@ def oracle_sample_step(wl, state=None, M_s=8):
     return dt, flops(M_s, shape.N, shape.K, RANK), state
 
 
+def base_config(args, shapes, Ms, mode):
+    return {"workload": WORKLOAD if not args.case else f"case {args.case}",
+            "layers": [f"{s.K}->{s.N}" for s in shapes], "M": Ms, "group": GROUP, "mode": mode,
+            "weight_layout": args.layout, "lorc_rank": RANK}
+
+
 def cpu_baseline(wl):
     import oracle
 
@@ -170,7 +189,7 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "group": GROUP, "mode": MODE, "lorc_rank": RANK},
+            "config": base_config(args, list(wl.shapes), sorted(wl.Ms, reverse=True), MODE),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -195,6 +214,146 @@ def reduce_over_ranks(local_ms: float, local_units: float, dist):
     return float(t.item()), float(u.item())
 
 
+def fp8_peak_for(peaks, timed_seconds, clocks):
+    """The tensor roofline's denominator: the measured bf16 cuBLAS peak times the nominal FP8 : bf16 ratio (2).
+    The burst figure when the timed region is short or the sampled clock stayed at its maximum, the sustained
+    (power-capped) one for a long region whose clock dropped."""
+    at_max = bool(clocks and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and
+                  clocks["sm_mhz"] >= 0.97 * clocks["sm_max_mhz"])
+    regime = "burst" if (timed_seconds < 2.0 or at_max) else "sustained"
+    return 2.0 * peaks["bf16_" + regime], regime
+
+
+class Bench:
+    """Device buffers of the layers and the calls into the C ABI."""
+
+    def __init__(self, dev, rank):
+        import ctypes as C
+
+        import torch
+
+        from paper_2307_09782_b200 import binding
+
+        self.C, self.torch, self.binding = C, torch, binding
+        self.L = binding.lib()  # fails loudly if the CUDA library is missing
+        self.dev, self.rank = dev, rank
+        self.stream = torch.cuda.current_stream()
+        self.sp = C.c_void_p(self.stream.cuda_stream)
+        self.w_cache = {}
+
+    def vp(self, t):
+        return None if t is None else self.C.c_void_p(t.data_ptr())
+
+    def make_layer(self, wl, shape, Mmax, mode, layout, rank_lorc=RANK, copies=N_WEIGHT_COPIES):
+        torch, binding = self.torch, self.binding
+        K, N = shape.K, shape.N
+        # replicas draw their own activations (row_offset = rank); weights are the same model on every rank
+        x_bits = synth.make_x(wl.seed, Mmax, K, wl.n_outliers(K), wl.outlier_factor, row_offset=self.rank)
+        x = torch.from_numpy(x_bits.view(np.int16)).to(self.dev).view(torch.bfloat16)
+        key = (wl.seed, N, K, wl.sigma_w)
+        if key not in self.w_cache:  # the host-side draw of a large weight takes seconds
+            self.w_cache[key] = synth.make_w(wl.seed, N, K, wl.sigma_w)
+        W = torch.from_numpy(self.w_cache[key]).to(self.dev)
+        pw = binding.pack_weight_fp4(W, GROUP, mode, layout)
+        del W
+        U = V = None
+        if rank_lorc:
+            U_h, V_h = synth.make_lorc(wl.seed, N, K, rank_lorc)
+            U, V = torch.from_numpy(U_h).to(self.dev), torch.from_numpy(V_h).to(self.dev)
+        cps = [(pw.codes, pw.shift, pw.scale)]
+        for _ in range(copies - 1):
+            c = pw.clone()
+            cps.append((c.codes, c.shift, c.scale))
+        ws = binding.make_workspace(binding.linear_workspace_bytes(Mmax, N, K, rank_lorc), self.dev)
+        return dict(K=K, N=N, r=rank_lorc, mode=binding.MODES[mode], layout=binding.LAYOUTS[layout], x=x, x_bits=x_bits,
+                    U=U, V=V, copies=cps, ws=ws,
+                    q=torch.empty((Mmax, K), dtype=torch.uint8, device=self.dev),
+                    sx=torch.empty((Mmax,), dtype=torch.float32, device=self.dev),
+                    t=torch.empty((Mmax, max(rank_lorc, 1)), dtype=torch.float32, device=self.dev),
+                    y=torch.empty((Mmax, N), dtype=torch.float32, device=self.dev))
+
+    def layer_call(self, ly, M, copy):
+        """The whole layer through one call on raw activations."""
+        vp, K, N = self.vp, ly["K"], ly["N"]
+        codes, shift, scale = ly["copies"][copy % len(ly["copies"])]
+        rc = self.L.zq_w4a8_linear(None, None, vp(ly["x"]), K, M, N, K, GROUP, ly["mode"], ly["layout"], vp(codes),
+                                   vp(shift), vp(scale), vp(ly["U"]), vp(ly["V"]), None, ly["r"], vp(ly["y"]), 0, N,
+                                   vp(ly["ws"]), ly["ws"].numel(), self.sp)
+        if rc:
+            raise RuntimeError(f"zq_w4a8_linear failed: {rc}")
+
+    def quant_call(self, ly, M):
+        vp, K = self.vp, ly["K"]
+        rc = self.L.zq_quantize_act_fp8(vp(ly["x"]), M, K, K, vp(ly["q"]), vp(ly["sx"]), vp(ly["V"]), ly["r"],
+                                        vp(ly["t"]) if ly["r"] else None, self.sp)
+        if rc:
+            raise RuntimeError(f"zq_quantize_act_fp8 failed: {rc}")
+
+    def gemm_call(self, ly, M, copy):
+        vp, K, N = self.vp, ly["K"], ly["N"]
+        codes, shift, scale = ly["copies"][copy % len(ly["copies"])]
+        rc = self.L.zq_w4a8_linear(vp(ly["q"]), vp(ly["sx"]), None, 0, M, N, K, GROUP, ly["mode"], ly["layout"],
+                                   vp(codes), vp(shift), vp(scale), vp(ly["U"]), None,
+                                   vp(ly["t"]) if ly["r"] else None, ly["r"], vp(ly["y"]), 0, N, vp(ly["ws"]),
+                                   ly["ws"].numel(), self.sp)
+        if rc:
+            raise RuntimeError(f"zq_w4a8_linear failed: {rc}")
+
+    def split_call(self, ly, M, copy, ev=None):
+        """The same layer as quantizer call + GEMM call, with optional events (start, between, end)."""
+        if ev:
+            ev[0].record(self.stream)
+        self.quant_call(ly, M)
+        if ev:
+            ev[1].record(self.stream)
+        self.gemm_call(ly, M, copy)
+        if ev:
+            ev[2].record(self.stream)
+
+    def time_shape(self, ly, M, n, batches=3):
+        """Steady-state times of one (layer, M) in microseconds: the one-call layer, the quantizer alone and
+        the GEMM alone on pre-quantized activations.  Each figure is one event pair around n back-to-back
+        launches, divided by n (launch gaps included; an event pair around a single launch adds about 4 us of
+        its own, measured with an empty kernel); the median of `batches` such batches."""
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def timed(fn):
+            res = []
+            for b in range(batches + 1):  # the first batch warms up
+                e0.record(self.stream)
+                for i in range(n):
+                    fn(b * n + i)
+                e1.record(self.stream)
+                torch.cuda.synchronize()
+                res.append(e0.elapsed_time(e1) * 1e3 / n)
+            return statistics.median(res[1:])
+
+        t_layer = timed(lambda i: self.layer_call(ly, M, i))
+        t_quant = timed(lambda i: self.quant_call(ly, M))
+        t_gemm = timed(lambda i: self.gemm_call(ly, M, i))
+        st = self.binding.device_status(ly["ws"])
+        if st[0] != 0:
+            raise RuntimeError(f"device status {st}")
+        return t_layer, t_quant, t_gemm
+
+
+def shape_row(name, M, N, K, r, t_layer, t_quant, t_gemm, peaks, fp8_peak, extra=None):
+    row = {"layer": name, "M": M, "layer_us": round(t_layer, 2), "quant_us": round(t_quant, 2),
+           "gemm_us": round(t_gemm, 2),
+           "layer_tflops": round(flops(M, N, K, r) / (t_layer * 1e-6) / 1e12, 2),
+           "gemm_tflops": round(2.0 * M * N * K / (t_gemm * 1e-6) / 1e12, 2),
+           "weight_gbs": round(weight_bytes(N, K) / (t_gemm * 1e-6) / 1e9, 1),
+           "quant_gbs": round(3.0 * M * K / (t_quant * 1e-6) / 1e9, 1),
+           "gemm_frac_fp8_peak": round(2.0 * M * N * K / (t_gemm * 1e-6) / 1e12 / fp8_peak, 4),
+           "gemm_frac_fp8_nominal": round(2.0 * M * N * K / (t_gemm * 1e-6) / 1e12 / NOMINAL_FP8_TFLOPS, 4),
+           "gemm_frac_hbm": round(gemm_bytes(M, N, K, r) / (t_gemm * 1e-6) / 1e9 / peaks["hbm_gbs"], 4),
+           "layer_frac_hbm": round(layer_bytes(M, N, K, r) / (t_layer * 1e-6) / 1e9 / peaks["hbm_gbs"], 4)}
+    if extra:
+        row.update(extra)
+    return row
+
+
 def run_ours(args):
     import torch
 
@@ -211,13 +370,13 @@ def run_ours(args):
         dist = dist_mod
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    binding.lib()  # fails loudly if the CUDA library is missing
+    B = Bench(dev, rank)
 
     wl = synth.WORKLOADS[WORKLOAD]
-    Ms = list(wl.Ms)
+    Ms = sorted(wl.Ms, reverse=True)
     shapes = list(wl.shapes)
     mode = MODE
-    layout = binding.LAYOUTS[args.layout]
+    sweeps = args.sweeps
     if args.case:
         parts = args.case.split(",")
         shapes = [synth.LayerShape(int(parts[0]), int(parts[1]), "case")]
@@ -225,69 +384,34 @@ def run_ours(args):
         if len(parts) > 3:
             mode = parts[3]
     Mmax = max(Ms)
-    layers = []
-    for shape in shapes:
-        K, N = shape.K, shape.N
-        # replicas draw their own activations (row_offset = rank); weights are the same model on every rank
-        x_bits = synth.make_x(wl.seed, Mmax, K, wl.n_outliers(K), wl.outlier_factor, row_offset=rank)
-        x = torch.from_numpy(x_bits.view(np.int16)).to(dev).view(torch.bfloat16)
-        W = torch.from_numpy(synth.make_w(wl.seed, N, K, wl.sigma_w)).to(dev)
-        pw = binding.pack_weight_fp4(W, GROUP, mode, layout)
-        del W
-        U_h, V_h = synth.make_lorc(wl.seed, N, K, RANK)
-        U, V = torch.from_numpy(U_h).to(dev), torch.from_numpy(V_h).to(dev)
-        copies = [(pw.codes, pw.shift, pw.scale)]
-        for _ in range(N_WEIGHT_COPIES - 1):
-            c = pw.clone()
-            copies.append((c.codes, c.shift, c.scale))
-        ws = binding.make_workspace(binding.linear_workspace_bytes(Mmax, N, K, RANK), dev)
-        layers.append(dict(K=K, N=N, x=x, x_bits=x_bits, U=U, V=V, copies=copies, ws=ws,
-                           q=torch.empty((Mmax, K), dtype=torch.uint8, device=dev),
-                           sx=torch.empty((Mmax,), dtype=torch.float32, device=dev),
-                           t=torch.empty((Mmax, RANK), dtype=torch.float32, device=dev),
-                           y=torch.empty((Mmax, N), dtype=torch.float32, device=dev)))
+    layers = [B.make_layer(wl, shape, Mmax, mode, args.layout) for shape in shapes]
     torch.cuda.synchronize()
-
-    L = binding.lib()
-    import ctypes as C
-
-    def vp(t):
-        return None if t is None else C.c_void_p(t.data_ptr())
-
-    stream = torch.cuda.current_stream()
-    sp = C.c_void_p(stream.cuda_stream)
+    stream = B.stream
     calls = [(li, M) for M in Ms for li in range(len(layers))]
+    n_big = sum(1 for _, M in calls if M == Mmax)
 
-    def one_call(li, M, copy, ev=None):
-        ly = layers[li]
-        K, N = ly["K"], ly["N"]
-        codes, shift, scale = ly["copies"][copy]
-        if ev:
-            ev[0].record(stream)
-        rc = L.zq_quantize_act_fp8(vp(ly["x"]), M, K, K, vp(ly["q"]), vp(ly["sx"]), vp(ly["V"]), RANK, vp(ly["t"]), sp)
-        if ev:
-            ev[1].record(stream)
-        rc |= L.zq_w4a8_linear(vp(ly["q"]), vp(ly["sx"]), None, 0, M, N, K, GROUP, binding.MODES[mode], layout, vp(codes),
-                               vp(shift), vp(scale), vp(ly["U"]), None, vp(ly["t"]), RANK, vp(ly["y"]), 0, N,
-                               vp(ly["ws"]), ly["ws"].numel(), sp)
-        if ev:
-            ev[2].record(stream)
-        if rc:
-            raise RuntimeError(f"zqfp call failed: {rc}")
-
-    def step(idx, events=None):
+    def sweep(idx, events=None):
+        """One pass over all (layer, M).  `events`: one triple per call at the largest token count."""
+        b = 0
         for ci, (li, M) in enumerate(calls):
-            one_call(li, M, (idx + ci // len(layers)) % N_WEIGHT_COPIES, events[ci] if events else None)
+            copy = idx + ci // len(layers)
+            if M == Mmax:
+                B.split_call(layers[li], M, copy, events[b] if events else None)
+                b += 1
+            else:
+                B.layer_call(layers[li], M, copy)
 
     for i in range(args.warmup):
-        step(i)
+        for s in range(sweeps):
+            sweep(i * sweeps + s)
     torch.cuda.synchronize()
     for ly in layers:
         st = binding.device_status(ly["ws"])
         if st[0] != 0:
             raise RuntimeError(f"device status {st}")
 
-    events = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in calls] for _ in range(args.steps)]
+    n_sw = args.steps * sweeps
+    events = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_big)] for _ in range(n_sw)]
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
@@ -298,8 +422,8 @@ def run_ours(args):
     launches0 = binding.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for i in range(args.steps):
-        step(args.warmup + i, events[i])
+    for i in range(n_sw):
+        sweep(args.warmup * sweeps + i, events[i])
     e1.record(stream)
     torch.cuda.synchronize()
     if dist:
@@ -307,53 +431,96 @@ def run_ours(args):
     launches = binding.launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     total_ms = e0.elapsed_time(e1)
-    step_flops = sum(flops(M, layers[li]["N"], layers[li]["K"], RANK) for li, M in calls)
-    ms_max, flops_all = reduce_over_ranks(total_ms, step_flops * args.steps, dist)
+    sweep_flops = sum(flops(M, layers[li]["N"], layers[li]["K"], RANK) for li, M in calls)
+    ms_max, flops_all = reduce_over_ranks(total_ms, sweep_flops * n_sw, dist)
     value = flops_all / (ms_max * 1e-3) / 1e12
 
-    # ---- per-call table from the events of the timed region
+    # ---- dominant kernel: the GEMM at the largest token count, from the events inside the timed region
     peaks = load_peaks()
-    fp8_peak = 2.0 * peaks["bf16_sustained"]
-    sweep = []
-    for ci, (li, M) in enumerate(calls):
-        ly = layers[li]
-        K, N = ly["K"], ly["N"]
-        tq = statistics.mean(events[s][ci][0].elapsed_time(events[s][ci][1]) for s in range(args.steps)) * 1e3
-        tg = statistics.mean(events[s][ci][1].elapsed_time(events[s][ci][2]) for s in range(args.steps)) * 1e3
-        gemm_bytes = weight_bytes(N, K) + M * K + 4 * M + 4 * M * N + 2 * RANK * N + 4 * M * RANK
-        sweep.append({"layer": f"{K}->{N}", "M": M, "quant_us": round(tq, 2), "gemm_us": round(tg, 2),
-                      "gemm_tflops": round(2.0 * M * N * K / (tg * 1e-6) / 1e12, 2),
-                      "weight_gbs": round(weight_bytes(N, K) / (tg * 1e-6) / 1e9, 1),
-                      "gemm_gbs": round(gemm_bytes / (tg * 1e-6) / 1e9, 1),
-                      "quant_gbs": round(3.0 * M * K / (tq * 1e-6) / 1e9, 1),
-                      "frac_fp8_peak": round(2.0 * M * N * K / (tg * 1e-6) / 1e12 / fp8_peak, 4),
-                      "frac_hbm": round(gemm_bytes / (tg * 1e-6) / 1e9 / peaks["hbm_gbs"], 4)})
-    # dominant kernel: the GEMM at the largest M (both layers)
-    big = [s for s in sweep if s["M"] == Mmax]
-    big_flops = sum(2.0 * Mmax * ly["N"] * ly["K"] for ly in layers) / len(layers)
-    big_us = statistics.mean(s["gemm_us"] for s in big)
-    achieved = big_flops / (big_us * 1e-6) / 1e12
-    roofline = {"bound": "tensor", "kernel": "w4a8_mx_gemm_kernel<224> (7168->28672), <256> (28672->7168)" if layout else "w4a8_gemm_kernel<256,false>", "achieved": round(achieved, 1),
-                "peak": round(fp8_peak, 1), "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4),
-                "traffic": DOMINANT_TRAFFIC if (layout and not args.case) else None,
-                "traffic_note": "DRAM bytes per launch (ncu dram__bytes_read + write, mean of the two M = 8192 launches)",
-                "peak_source": f"2 x bf16 sustained cuBLAS peak ({peaks['source']}); nominal dense FP8 4500"}
-    dec = [s for s in sweep if s["M"] <= 16] or [sweep[0]]
-    roofline_decode = {"bound": "hbm", "kernel": "w4a8_mx_gemm_kernel<16>" if layout else "w4a8_gemm_kernel<16,false>",
-                       "achieved": round(statistics.mean(s["gemm_gbs"] for s in dec), 1),
-                       "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                       "frac": round(statistics.mean(s["frac_hbm"] for s in dec), 4),
-                       "traffic": DECODE_TRAFFIC if (layout and not args.case) else None,
-                       "traffic_note": "DRAM bytes per launch (ncu, 7168->28672 at M = 8, mean of two launches)",
-                       "peak_source": f"copy bandwidth ({peaks['source']}); nominal 7700-8000"}
-    big_q = [s for s in sweep if s["M"] == Mmax and s["layer"].startswith("28672")] or [sweep[-1]]
-    roofline_quant = {"bound": "hbm", "kernel": "act_quant_rows_kernel<true>", "achieved": big_q[0]["quant_gbs"],
-                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(big_q[0]["quant_gbs"] / peaks["hbm_gbs"], 4),
-                      "traffic": None}
+    fp8_peak, regime = fp8_peak_for(peaks, total_ms * 1e-3, clocks)
+    big_layers = [li for li, M in calls if M == Mmax]
+    per_layer_us = []
+    for b, li in enumerate(big_layers):
+        per_layer_us.append(statistics.mean(events[s][b][1].elapsed_time(events[s][b][2]) for s in range(n_sw)) * 1e3)
+    bound = "tensor" if Mmax >= 512 else "hbm"
+    kfam = "w4a8_mx_gemm_kernel" if args.layout == "mx" else "w4a8_gemm_kernel"
+    bms = {li: binding.linear_plan(Mmax, layers[li]["N"], layers[li]["K"], mode, args.layout)["bm"] for li in big_layers}
+    kname = ", ".join(f"{kfam}<{bms[li]}> ({layers[li]['K']}->{layers[li]['N']}, {per_layer_us[b]:.1f} us)"
+                      for b, li in enumerate(big_layers))
+    big_us = statistics.mean(per_layer_us)
+    if bound == "tensor":
+        big_flops = statistics.mean(2.0 * Mmax * layers[li]["N"] * layers[li]["K"] for li in big_layers)
+        achieved = big_flops / (big_us * 1e-6) / 1e12
+        roofline = {"bound": "tensor", "kernel": kname, "achieved": round(achieved, 1), "peak": round(fp8_peak, 1),
+                    "unit": "TFLOP/s", "frac": round(achieved / fp8_peak, 4),
+                    "peak_source": f"2 x bf16 cuBLAS peak, {regime} figure ({peaks['source']}): timed region "
+                                   f"{total_ms * 1e-3:.2f} s",
+                    "frac_of_burst_peak": round(achieved / (2.0 * peaks["bf16_burst"]), 4),
+                    "frac_of_sustained_peak": round(achieved / (2.0 * peaks["bf16_sustained"]), 4),
+                    "frac_of_nominal_4500": round(achieved / NOMINAL_FP8_TFLOPS, 4),
+                    "traffic": DOMINANT_TRAFFIC if (args.layout == "mx" and not args.case) else None,
+                    "launches_timed": n_sw * len(big_layers)}
+    else:
+        big_bytes = statistics.mean(gemm_bytes(Mmax, layers[li]["N"], layers[li]["K"], RANK) for li in big_layers)
+        achieved = big_bytes / (big_us * 1e-6) / 1e9
+        roofline = {"bound": "hbm", "kernel": kname, "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": round(achieved / peaks["hbm_gbs"], 4),
+                    "peak_source": f"copy bandwidth ({peaks['source']})", "traffic": None,
+                    "launches_timed": n_sw * len(big_layers),
+                    "note": "single launches between event pairs: each figure carries about 4 us of event overhead"}
+
+    # ---- per (layer, M): steady-state times of each shape by itself, after the timed region
+    table = []
+    if not args.no_sweep_table:
+        for li, M in calls:
+            ly = layers[li]
+            tl, tq, tg = B.time_shape(ly, M, n=20 if M <= 2048 else 6)
+            table.append(shape_row(f"{ly['K']}->{ly['N']}", M, ly["N"], ly["K"], RANK, tl, tq, tg, peaks, fp8_peak))
+    dec = [s for s in table if s["M"] <= 16]
+    roofline_decode = None
+    if dec:
+        roofline_decode = {"bound": "hbm", "kernel": f"{kfam}<16>",
+                           "what": "the GEMM alone on pre-quantized activations at M <= 16: algorithmic bytes / gemm_us",
+                           "achieved": round(statistics.mean(s["gemm_frac_hbm"] for s in dec) * peaks["hbm_gbs"], 1),
+                           "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                           "frac": round(statistics.mean(s["gemm_frac_hbm"] for s in dec), 4),
+                           "frac_whole_layer": round(statistics.mean(s["layer_frac_hbm"] for s in dec), 4),
+                           "traffic": DECODE_TRAFFIC if (args.layout == "mx" and not args.case) else None,
+                           "peak_source": f"copy bandwidth ({peaks['source']}); nominal 7700-8000"}
+    big_q = [s for s in table if s["M"] == Mmax and s["layer"].startswith("28672")] or table[:1]
+    roofline_quant = None
+    if big_q:
+        roofline_quant = {"bound": "hbm", "kernel": "activation quantizer at [%d, %s]" % (big_q[0]["M"], big_q[0]["layer"].split("->")[0]),
+                          "achieved": big_q[0]["quant_gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                          "frac": round(big_q[0]["quant_gbs"] / peaks["hbm_gbs"], 4), "traffic": None}
+
+    # ---- further rows the configurations ask for (not part of the timed step)
+    extra_rows = []
+    if not args.case and not args.no_extra:
+        def extra(wl_, shape, M, md, lay, r_):
+            ly = B.make_layer(wl_, shape, M, md, lay, rank_lorc=r_)
+            tl, tq, tg = B.time_shape(ly, M, n=20 if M <= 2048 else 6)
+            extra_rows.append(shape_row(f"{shape.K}->{shape.N}", M, shape.N, shape.K, r_, tl, tq, tg, peaks, fp8_peak,
+                                        {"workload": wl_.name, "mode": md, "layout": lay, "lorc_rank": r_}))
+            del ly
+
+        other = "cast" if args.layout == "mx" else "mx"
+        for shape in shapes:
+            for M in (8, Mmax):  # the sweep's workload without LoRC
+                extra(wl, shape, M, mode, args.layout, 0)
+            for M in (1, 8, Mmax):  # the other kernel family (cast: kind::f8f6f4, E4M3 x E4M3, the kernel casts)
+                extra(wl, shape, M, mode, other, RANK)
+        wl7 = synth.WORKLOADS["llama7b"]  # unconstrained scales (per-group FP32 promotion) at 2048 tokens
+        for shape in wl7.shapes:
+            for md, lay in EXTRA_LLAMA7B:
+                extra(wl7, shape, 2048, md, lay, RANK)
+        torch.cuda.empty_cache()
 
     # ---- end to end through the host-buffer entry point (host <-> device copies inside the timed region)
     e2e = None
     if not args.no_e2e:
+        import ctypes as C
+
         h2d = d2h = 0
         hosts = []
         for ly in layers:
@@ -363,61 +530,87 @@ def run_ours(args):
             wsh = binding.make_workspace(binding.linear_host_workspace_bytes(Mmax, N, K, RANK), dev)
             hosts.append((xh, yh, wsh))
 
-        def e2e_step(idx):
+        def e2e_sweep(idx):
             for ci, (li, M) in enumerate(calls):
                 ly = layers[li]
                 xh, yh, wsh = hosts[li]
                 codes, shift, scale = ly["copies"][(idx + ci // len(layers)) % N_WEIGHT_COPIES]
-                rc = L.zq_w4a8_linear_host(C.c_void_p(xh.data_ptr()), M, ly["N"], ly["K"], GROUP, binding.MODES[mode], layout,
-                                           vp(codes), vp(shift), vp(scale), vp(ly["U"]), vp(ly["V"]), RANK,
-                                           C.c_void_p(yh.data_ptr()), vp(wsh), wsh.numel(), sp)
+                rc = B.L.zq_w4a8_linear_host(C.c_void_p(xh.data_ptr()), M, ly["N"], ly["K"], GROUP, ly["mode"],
+                                             ly["layout"], B.vp(codes), B.vp(shift), B.vp(scale), B.vp(ly["U"]),
+                                             B.vp(ly["V"]), RANK, C.c_void_p(yh.data_ptr()), B.vp(wsh), wsh.numel(), B.sp)
                 if rc:
                     raise RuntimeError(f"zq_w4a8_linear_host failed: {rc}")
 
         for li, M in calls:
             h2d += 2 * M * layers[li]["K"]
             d2h += 4 * M * layers[li]["N"]
-        e2e_steps = max(1, min(args.steps, 5))
-        e2e_step(0)
+        e2e_sweeps = max(1, min(args.steps, 5))
+        e2e_sweep(0)
         torch.cuda.synchronize()
         if dist:
             dist.barrier()
         t0 = time.perf_counter()
-        for i in range(e2e_steps):
-            e2e_step(i + 1)
+        for i in range(e2e_sweeps):
+            e2e_sweep(i + 1)
         torch.cuda.synchronize()
         e2e_ms = (time.perf_counter() - t0) * 1e3
         if dist:
             dist.barrier()
-        e2e_ms_max, e2e_flops = reduce_over_ranks(e2e_ms, step_flops * e2e_steps, dist)
-        e2e = {"value": round(e2e_flops / (e2e_ms_max * 1e-3) / 1e12, 3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": round(e2e_ms_max / e2e_steps, 3),
+        e2e_ms_max, e2e_flops = reduce_over_ranks(e2e_ms, sweep_flops * e2e_sweeps, dist)
+        e2e = {"value": round(e2e_flops / (e2e_ms_max * 1e-3) / 1e12, 3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d * sweeps, "d2h_bytes_per_step": d2h * sweeps,
+               "sweeps_timed": e2e_sweeps, "ms_per_sweep": round(e2e_ms_max / e2e_sweeps, 3),
                "api": "zq_w4a8_linear_host (pinned host x -> device, quantizer + linear, y -> pinned host)"}
 
     if rank != 0:
         return
+    cfg = base_config(args, shapes, Ms, mode)
+    cfg.update({"sweeps_per_step": sweeps, "multi_gpu": "independent replicas",
+                "l2": f"inputs larger than L2: {N_WEIGHT_COPIES} weight copies per layer rotated, >300 MB "
+                      "streamed between two reads of one buffer"})
+    dtype = ("f4e2m1 (E8M0 block scale) x f8e4m3 -> f32" if args.layout == "mx"
+             else "f8e4m3 (cast from f4e2m1 in the kernel) x f8e4m3 -> f32")
     line = {"metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": round(ms_max / args.steps, 4), "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f8e4m3 x f8e4m3 -> f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD if not args.case else f"case {args.case}",
-                       "layers": [f"{s.K}->{s.N}" for s in shapes], "M": Ms, "group": GROUP, "mode": mode, "weight_layout": args.layout, "lorc_rank": RANK, "multi_gpu": "independent replicas",
-                       "l2": f"inputs larger than L2: {N_WEIGHT_COPIES} weight copies per layer rotated, >300 MB "
-                             "streamed between two reads of one buffer"},
+            "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic", "config": cfg,
+            "timed_region_s": round(ms_max * 1e-3, 3),
             "roofline": roofline, "roofline_decode": roofline_decode, "roofline_quant": roofline_quant,
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "sweep": sweep}
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+            "sweep_note": "per-shape rows: each (layer, M) timed by itself after the timed region: one event pair "
+                          "around n = 6-20 back-to-back launches (rotated weight copies), divided by n, median of 3 "
+                          "batches; layer_us = one zq_w4a8_linear call on raw x; quant_us / gemm_us = the quantizer "
+                          "kernel alone and the GEMM alone on pre-quantized activations",
+            "sweep": table, "extra_rows": extra_rows}
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(wl)
     print(json.dumps(line))
 
 
+def spawn_ranks(args) -> int:
+    """`--gpus N` without a torchrun environment: start the N ranks (one process per GPU) ourselves."""
+    import socket
+
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--sweeps", type=int, default=25,
+                    help="passes over the (layer, M) sweep per step (a step of about 0.1 s, so that 20 steps give "
+                         "a timed region of about 2 s and settled clocks)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the rows outside the timed step")
+    ap.add_argument("--no-sweep-table", action="store_true", help="skip the per-shape table")
     ap.add_argument("--layout", default="mx", choices=["cast", "mx"],
                     help="weight layout: the kernel casts FP4 to FP8 (cast) or the tensor core does (mx)")
     ap.add_argument("--case", default=None, metavar="K,N,M[,MODE]",
@@ -425,8 +618,10 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_ours(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
+    run_ours(args)
     if int(os.environ.get("WORLD_SIZE", "1")) > 1:
         import torch.distributed as dist
 

@@ -103,11 +103,13 @@ int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, 
  *             (b = 0..3);
  *           - byte 8192 + 2r + h = the shift of row r for elements 64h .. 64h+63 (0 in mode none).
  *         Rows of the last tile beyond N are zero.
- *         With ZQ_WEIGHTS_MX (M1 / M2 only; ZQ_ERR_MODE otherwise) a tile is 8704 bytes, 32-byte aligned:
- *           - [0, 8192): row r at r*64, element k of the K block in byte k/2, even k in the low nibble, a
- *             nibble being the E2M1 code s e1 e0 m;
- *           - byte 8192 + 16*(r % 32) + 4*(r / 32) + s = 127 - shift of row r for elements 32s .. 32s+31
- *             (the E8M0 encoding of 2^-shift), the order in which the tensor core's scale copy reads them.
+ *         With ZQ_WEIGHTS_MX (M1 / M2 only; ZQ_ERR_MODE otherwise; 32-byte aligned) a block of 128 output rows
+ *         takes (K/128) * 8704 bytes, the codes of all its K blocks first and their scales after:
+ *           - [kb*8192, +8192): K block kb; row r at r*64, element k of the K block in byte k/2, even k in
+ *             the low nibble, a nibble being the E2M1 code s e1 e0 m;
+ *           - byte (K/128)*8192 + kb*512 + 16*(r % 32) + 4*(r / 32) + s = 127 - shift of row r for elements
+ *             32s .. 32s+31 of K block kb (the E8M0 encoding of 2^-shift), the order in which the tensor
+ *             core's scale copy reads them.
  *         Rows beyond N have zero codes and scale bytes 127.
  * shift : out, u8 [N, G] (M1, M2), the same shifts in plain form; ignored (may be NULL) in mode none
  * scale : out, FP32 [N] (M1, M2) or [N, G] (none)

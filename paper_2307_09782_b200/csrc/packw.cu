@@ -60,8 +60,9 @@ pack_weight_kernel(const float* __restrict__ W, int N, int K, int mode, uint8_t*
       uint8_t* blk = tile_row + static_cast<int64_t>(k / kTileK) * kTB;
       const int within = k % kTileK;
       if (MX) {
-        *reinterpret_cast<uint32_t*>(blk + r * 64 + within / 2) = 0u;
-        if (within % 32 == 0) blk[kTileCodeBytes + 16 * (r % 32) + 4 * (r / 32) + within / 32] = 127;
+        const int kb = k / kTileK;
+        *reinterpret_cast<uint32_t*>(tile_row + mx_code_offset(kb) + r * 64 + within / 2) = 0u;
+        if (within % 32 == 0) tile_row[mx_scale_offset(kblocks, kb) + 16 * (r % 32) + 4 * (r / 32) + within / 32] = 127;
       } else {
         *reinterpret_cast<uint32_t*>(blk + ((within / 32) * kTileRows + r) * 16 + ((within % 32) / 8) * 4) = 0u;
         if (within % 64 == 0) blk[kTileCodeBytes + 2 * r + within / 64] = 0;
@@ -160,9 +161,10 @@ pack_weight_kernel(const float* __restrict__ W, int N, int K, int mode, uint8_t*
     uint8_t* blk = tile_row + static_cast<int64_t>(k / kTileK) * kTB;
     const int within = k % kTileK;
     if (MX) {
-      *reinterpret_cast<uint32_t*>(blk + r * 64 + within / 2) = w;
+      const int kb = k / kTileK;
+      *reinterpret_cast<uint32_t*>(tile_row + mx_code_offset(kb) + r * 64 + within / 2) = w;
       if (within % 32 == 0)
-        blk[kTileCodeBytes + 16 * (r % 32) + 4 * (r / 32) + within / 32] = static_cast<uint8_t>(127 - d);
+        tile_row[mx_scale_offset(kblocks, kb) + 16 * (r % 32) + 4 * (r / 32) + within / 32] = static_cast<uint8_t>(127 - d);
     } else {
       *reinterpret_cast<uint32_t*>(blk + ((within / 32) * kTileRows + r) * 16 + ((within % 32) / 8) * 4) = w;
       if (within % 64 == 0) blk[kTileCodeBytes + 2 * r + within / 64] = static_cast<uint8_t>(d);

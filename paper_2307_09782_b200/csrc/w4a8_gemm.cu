@@ -646,7 +646,9 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   const int kblocks = static_cast<int>(K / kBlockK);
   if (tiles <= 0 || kblocks <= 0) return pl;  // nothing to do: an empty plan (ctas == 0)
   // CTAs per SM the kernel family is sized for at this tile
-  const int ctas_per_sm = mx ? (bm <= 64 ? 2 : 1) : ((mode == ZQ_SCALE_NONE || bm > 128) ? 1 : (bm <= 16 ? 3 : 2));
+  // (the block-scaled kernel: always one; its launches with shared tiles are cooperative, and a cooperative
+  // launch of a kernel that allocates tensor memory is given one CTA per SM)
+  const int ctas_per_sm = mx ? 1 : ((mode == ZQ_SCALE_NONE || bm > 128) ? 1 : (bm <= 16 ? 3 : 2));
   const int64_t resident = static_cast<int64_t>(ctas_per_sm) * sm_count();
   const int64_t units = tiles * kblocks;
   // as many token tiles per group of the launch order as keep the group's tokens around 32 MB (they must
@@ -656,13 +658,11 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
     pl.m_group = static_cast<int>(fit < 1 ? 1 : (fit > 8 ? 8 : fit));
   }
   if (mx && ((pl.m_tiles > 1 && (tiles >= 4 * resident || tiles > kWsMaxTiles)) ||
-             (pl.m_tiles == 1 && bm >= 128 && tiles >= resident) ||
-             (pl.m_tiles == 1 && bm < 128 && 4 * tiles >= 3 * resident))) {
+             (pl.m_tiles == 1 && bm >= 128 && tiles >= resident))) {
     // many tokens: one resident wave of CTAs walks whole tiles (with fewer than four tiles per CTA the
     // uneven last round would cost too much: those shapes take the contiguous unit ranges below).  Also one
-    // row of tiles that fills at least three quarters of a resident wave (a full one for wide tiles): a CTA
-    // that shares tiles runs two epilogues and a hand-over, which measured dearer than the idle slots
-    // (7168 -> 28672: 31.6 -> 26.7 us at 8 tokens, 41 -> 29 us at 32, 60 -> 47 us at 128).
+    // row of wide tiles that fills a resident wave.  (One row of narrow tiles always takes the unit ranges:
+    // with one CTA per SM whole tiles would leave a second, half-empty round.)
     pl.persist = 1;
     const int64_t g = tiles < resident ? tiles : resident;
     pl.ctas = static_cast<int>(g);

@@ -8,11 +8,14 @@
 // power-of-two (E8M0) scale per row and 32 elements of K, which is exactly the constrained group
 // scale 2^-shift.  The kernel therefore moves bytes and issues MMAs; no CUDA core touches a weight.
 //
-//   weights  one TMA load per K block brings a 128 x 128 tile of packed nibbles (8 KB, contiguous in
-//            HBM) into shared memory, expanded by the copy engine to the tensor core's 16-byte-aligned
-//            FP4 form (8 bytes of nibbles, 8 bytes of padding);
-//   scales   the tile's 512 E8M0 bytes follow it in HBM, arrive by a bulk copy and go to tensor memory
-//            with tcgen05.cp, issued by the MMA thread right before the tile's four MMAs;
+//   weights  one TMA load per pipeline stage brings one (wide token tiles) or two (up to 64 tokens) 128 x 128
+//            tiles of packed nibbles (8 KB each, contiguous in HBM) into shared memory, expanded by the copy
+//            engine to the tensor core's 16-byte-aligned FP4 form (8 bytes of nibbles, 8 bytes of padding).
+//            With few tokens a CTA's rate is bound by the number of copies it issues, not by their bytes
+//            (a CTA got through one 8.7 KB copy per 0.3 us whatever the ring depth), hence two K blocks per
+//            copy there;
+//   scales   the tiles' 512 E8M0 bytes each (contiguous for consecutive K blocks) arrive by one bulk copy
+//            and go to tensor memory with tcgen05.cp, issued by the MMA thread right before a tile's four MMAs;
 //   tokens   E4M3 tiles by TMA, the shared-memory B operand, with a block scale of one;
 //   D        FP32 in tensor memory, two buffers where they fit, so that the epilogue of one output tile
 //            overlaps the main loop of the next.
@@ -42,33 +45,43 @@ constexpr int kSfbCols = 16;  // token-side block scales (all one): room for 256
 
 template <int BM>
 struct MxCfg {
-  static constexpr int kMinBlocks = BM <= 64 ? 2 : 1;  // CTAs per SM this configuration is sized for
+  // One CTA per SM: launches whose CTAs share output tiles are cooperative, and a cooperative launch of a
+  // kernel that allocates tensor memory is given one CTA per SM (the occupancy query answers 1 whatever the
+  // registers and shared memory; with two CTAs per SM planned, grids beyond the SM count were refused).
+  static constexpr int kMinBlocks = 1;
+  static constexpr int kKps = BM <= 64 ? 2 : 1;  // K blocks per pipeline stage
   static constexpr int kProducerWarp = 4;
   static constexpr int kMmaWarp = 5;
   static constexpr int kThreads = 192;
   static constexpr int kEpiThreads = 128;
-  static constexpr int kABytes = kTileRows * kTileK;  // shared-memory footprint of a code tile (padded FP4)
-  static constexpr int kTokBytes = BM * kBlockK;
-  static constexpr int kStageTx = kTileCodeBytes + kMxTileScaleBytes + kTokBytes;  // bytes a stage's barrier counts
+  static constexpr int kABytes1 = kTileRows * kTileK;  // shared-memory footprint of one code tile (padded FP4)
+  static constexpr int kTokBytes1 = BM * kBlockK;
+  static constexpr int kABytes = kKps * kABytes1;      // per stage
+  static constexpr int kTokBytes = kKps * kTokBytes1;
+  static constexpr int kSfBytes = kKps * kMxTileScaleBytes;
+  // bytes a stage's barrier counts besides the scales (whole boxes: what lies beyond the tensor is filled
+  // with zeros and counted too)
+  static constexpr int kStageTxBoxes = kKps * kTileCodeBytes + kTokBytes;
   static constexpr int kBudget = (kMinBlocks == 1 ? 220 : 110) * 1024 - BM * 36 - 512;
-  static constexpr int NS = cmin(12, kBudget / (kABytes + kMxTileScaleBytes + kTokBytes));
+  static constexpr int NS = cmin(12, kBudget / (kABytes + kSfBytes + kTokBytes));
   static constexpr int NB = BM <= 224 ? 2 : 1;  // accumulator buffers
   static constexpr int kDColsPad = BM < 32 ? 32 : BM;
   static constexpr int kSfaCol0 = NB * kDColsPad;
-  static constexpr int kSfbCol0 = kSfaCol0 + 4 * NS;
+  static constexpr int kSfbCol0 = kSfaCol0 + 4 * kKps * NS;
   static constexpr int kColsUsed = kSfbCol0 + kSfbCols;
   static constexpr int kTmemCols = kColsUsed <= 128 ? 128 : (kColsUsed <= 256 ? 256 : 512);
   // shared memory map (offsets from a 1024-byte aligned base)
   static constexpr int offA = 0;
   static constexpr int offTok = offA + NS * kABytes;
   static constexpr int offSf = offTok + NS * kTokBytes;
-  static constexpr int offSx = offSf + NS * kMxTileScaleBytes;  // [BM] token scales
+  static constexpr int offSx = offSf + NS * kSfBytes;  // [BM] token scales
   static constexpr int offT = offSx + BM * 4;                   // [8][BM] LoRC down-projection (rank 8)
   static constexpr int offBars = offT + BM * 32;
   static constexpr int kNumBars = 2 * NS + 2 * NB + 1;
   static constexpr int offMisc = offBars + kNumBars * 8;
   static constexpr int kSmemBytes = offMisc + 32;
   static_assert(NS >= 3, "pipeline depth");
+  static_assert(kTokBytes1 % 1024 == 0 || kKps == 1, "the second token tile of a stage must start on a swizzle atom");
   static_assert(kTmemCols * kMinBlocks <= 512, "tensor memory");
   static_assert(kSmemBytes * kMinBlocks <= 226 * 1024, "shared memory");
 };
@@ -193,20 +206,24 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       bool ok = true;
       while (ok && sg.next(p, pos, tile, kb0, nkb)) {
         const int m0 = (tile / p.n_tiles) * BM;
-        const int wt0 = (tile % p.n_tiles) * p.kblocks;  // index of the output channels' first weight tile
-        for (int kb = kb0; kb < kb0 + nkb; ++kb) {
+        const int nt = tile % p.n_tiles;
+        const uint8_t* sf_row = p.codes + static_cast<int64_t>(nt) * p.kblocks * kMxTileBytes + mx_scale_offset(p.kblocks, 0);
+        for (int kb = kb0; kb < kb0 + nkb; kb += C::kKps) {
           if (!mbar_wait(&empty[s], ph ^ 1, s_abort)) {
             if (issuer) raise_error(p, s_abort, kErrProducer);
             ok = false;
             break;
           }
           if (issuer) {
-            mbar_arrive_expect_tx(&full[s], C::kStageTx);
-            tma_load_3d(s_a + s * C::kABytes, &tm_w, 0, 0, wt0 + kb, &full[s]);
-            bulk_load(s_sf + s * kMxTileScaleBytes,
-                      p.codes + static_cast<int64_t>(wt0 + kb) * kMxTileBytes + kTileCodeBytes, kMxTileScaleBytes,
-                      &full[s]);
-            tma_load_2d(s_tok + s * C::kTokBytes, &tm_q, kb * kBlockK, m0, &full[s]);
+            // The boxes always span kKps K blocks (beyond the row's last K block the copy engine fills in
+            // zeros; a K block past the end of this CTA's range is read but not used); the scales are copied
+            // for the K blocks that exist only, never past the row's end.
+            const int nsf = min(C::kKps, p.kblocks - kb);
+            mbar_arrive_expect_tx(&full[s], C::kStageTxBoxes + nsf * kMxTileScaleBytes);
+            tma_load_4d(s_a + s * C::kABytes, &tm_w, 0, 0, kb, nt, &full[s]);
+            bulk_load(s_sf + s * C::kSfBytes, sf_row + static_cast<int64_t>(kb) * kMxTileScaleBytes,
+                      nsf * kMxTileScaleBytes, &full[s]);
+            tma_load_3d(s_tok + s * C::kTokBytes, &tm_q, 0, m0, kb, &full[s]);
           }
           __syncwarp();
           ++issued;
@@ -242,25 +259,31 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
           break;
         }
         const uint32_t d_tmem = tmem_base + buf * C::kDColsPad;
-        for (int i = 0; i < nkb; ++i) {
+        for (int i = 0; i < nkb; i += C::kKps) {
+          const int nk = min(C::kKps, nkb - i);  // K blocks of this stage that belong to the segment
           if (!mbar_wait(&full[s], ph, s_abort)) {
             failed = true;
             break;
           }
           tc_fence_after_sync();
-          const uint32_t sfa = tmem_sfa + 4 * s;
-          const uint64_t adesc = adesc0 + static_cast<uint64_t>((s * C::kABytes) >> 4);
-          const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((s * C::kTokBytes) >> 4);
           if (issuer) {
-            tmem_cp_32x128b_x4(sfa, sfdesc0 + static_cast<uint64_t>((s * kMxTileScaleBytes) >> 4));
 #pragma unroll
-            for (int k = 0; k < kBlockK / 32; ++k) {
-              // scale byte k of the stage's four columns belongs to elements 32k .. 32k+31
-              umma_mxf8f6f4(d_tmem, adesc + 2 * k, bdesc + 2 * k, umma_idesc_mx_e2m1_e4m3(BM, k, 0),
-                            sfa + (static_cast<uint32_t>(k) << 30), tmem_sfb, (i > 0 || k > 0) ? 1u : 0u);
+            for (int j = 0; j < C::kKps; ++j) {
+              if (j < nk) {
+                const uint32_t sfa = tmem_sfa + 4 * (s * C::kKps + j);
+                const uint64_t adesc = adesc0 + static_cast<uint64_t>((s * C::kABytes + j * C::kABytes1) >> 4);
+                const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((s * C::kTokBytes + j * C::kTokBytes1) >> 4);
+                tmem_cp_32x128b_x4(sfa, sfdesc0 + static_cast<uint64_t>((s * C::kSfBytes + j * kMxTileScaleBytes) >> 4));
+#pragma unroll
+                for (int k = 0; k < kBlockK / 32; ++k) {
+                  // scale byte k of the K block's four columns belongs to elements 32k .. 32k+31
+                  umma_mxf8f6f4(d_tmem, adesc + 2 * k, bdesc + 2 * k, umma_idesc_mx_e2m1_e4m3(BM, k, 0),
+                                sfa + (static_cast<uint32_t>(k) << 30), tmem_sfb, (i > 0 || j > 0 || k > 0) ? 1u : 0u);
+                }
+              }
             }
             umma_commit(&empty[s]);
-            if (i + 1 == nkb) umma_commit(&acc_full[buf]);
+            if (i + C::kKps >= nkb) umma_commit(&acc_full[buf]);
           }
           __syncwarp();
           if (++s == C::NS) {
@@ -461,16 +484,31 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
 }
 
 // ---- host ------------------------------------------------------------------------------------------
-// The packed weight as a 3-D tensor of 4-bit elements [tiles][128 rows][128 elements]; the copy engine
-// expands a 128 x 128 box to the 16-byte-aligned FP4 form in shared memory, 128-byte swizzled.
-bool make_weight_map(CUtensorMap* m, const void* base, uint64_t tiles) {
+// The packed weight as a 4-D tensor of 4-bit elements [row blocks][K blocks][128 rows][128 elements]; the copy
+// engine expands a box of `kps` 128 x 128 tiles to the 16-byte-aligned FP4 form in shared memory, 128-byte
+// swizzled, one tile after the other.
+bool make_weight_map(CUtensorMap* m, const void* base, uint64_t n_tiles, uint64_t kblocks, uint32_t kps) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
-  const cuuint64_t dims[3] = {kTileK, kTileRows, tiles};
-  const cuuint64_t strides[2] = {kTileK / 2, kMxTileBytes};
-  const cuuint32_t box[3] = {kTileK, kTileRows, 1};
+  const cuuint64_t dims[4] = {kTileK, kTileRows, kblocks, n_tiles};
+  const cuuint64_t strides[3] = {kTileK / 2, kTileCodeBytes, kblocks * kMxTileBytes};
+  const cuuint32_t box[4] = {kTileK, kTileRows, kps, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The E4M3 activations q [M, K] as a 3-D tensor [K blocks][M rows][128 bytes]: a box of `kps` K blocks x bm
+// rows lands in shared memory as `kps` token tiles of bm x 128 bytes, one after the other, 128-byte swizzled.
+bool make_token_map(CUtensorMap* m, const void* base, uint64_t K, uint64_t M, uint32_t bm, uint32_t kps) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {kBlockK, M, K / kBlockK};
+  const cuuint64_t strides[2] = {K, kBlockK};
+  const cuuint32_t box[3] = {kBlockK, bm, kps};
   const cuuint32_t estr[3] = {1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 3, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -479,9 +517,8 @@ template <int BM>
 int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStream_t st) {
   using C = MxCfg<BM>;
   CUtensorMap tm_w, tm_q;
-  if (!make_weight_map(&tm_w, a.codes, static_cast<uint64_t>(plan.n_tiles) * static_cast<uint64_t>(p.kblocks)) ||
-      !make_map(&tm_q, a.q, static_cast<uint64_t>(a.K), static_cast<uint64_t>(a.M), kBlockK, BM,
-                CU_TENSOR_MAP_SWIZZLE_128B))
+  if (!make_weight_map(&tm_w, a.codes, static_cast<uint64_t>(plan.n_tiles), static_cast<uint64_t>(p.kblocks), C::kKps) ||
+      !make_token_map(&tm_q, a.q, static_cast<uint64_t>(a.K), static_cast<uint64_t>(a.M), BM, C::kKps))
     return ZQ_ERR_CUDA;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;

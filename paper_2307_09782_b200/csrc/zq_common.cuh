@@ -37,14 +37,22 @@ constexpr int kTileCodeBytes = kTileRows * kTileK / 2;
 constexpr int kTileShiftBytes = 2 * kTileRows;
 constexpr int kTileBytes = kTileCodeBytes + kTileShiftBytes;
 
-// Tiles for the tensor core's own FP4 operand (layout ZQ_WEIGHTS_MX, modes M1 / M2).  Same tiling and tile
-// order; a tile holds
-//   [0, 8192)    codes, row-major: row r at r * 64, element k of the K block in byte k / 2 (even k in the low
-//                nibble), a nibble being the plain E2M1 code (sign in bit 3)
-//   [8192, 8704) block scales, one E8M0 byte 127 - shift per row and 32 elements, in the order the tensor
-//                memory copy wants: byte 16 * (r % 32) + 4 * (r / 32) + s for row r, elements 32s .. 32s+31
+// Layout ZQ_WEIGHTS_MX (modes M1 / M2), for the tensor core's own FP4 operand.  The same 128 x 128 tiles, 8704
+// bytes each, but a block of 128 output rows keeps the codes of all its K blocks first and their scales after:
+// block nt starts at nt * (K / 128) * 8704 and holds
+//   [kb * 8192, +8192)                codes of K block kb, row-major: row r at r * 64, element k of the K block
+//                                     in byte k / 2 (even k in the low nibble), a nibble being the plain E2M1
+//                                     code (sign in bit 3)
+//   [(K / 128) * 8192 + kb * 512, +512)  its block scales, one E8M0 byte 127 - shift per row and 32 elements, in
+//                                     the order the tensor-memory copy wants: byte 16 * (r % 32) + 4 * (r / 32) + s
+//                                     for row r, elements 32s .. 32s+31
+// so that the codes (and the scales) of consecutive K blocks are contiguous and one copy brings several.
 constexpr int kMxTileScaleBytes = 4 * kTileRows;
 constexpr int kMxTileBytes = kTileCodeBytes + kMxTileScaleBytes;
+__host__ __device__ inline int64_t mx_code_offset(int kb) { return static_cast<int64_t>(kb) * kTileCodeBytes; }
+__host__ __device__ inline int64_t mx_scale_offset(int kblocks, int kb) {
+  return static_cast<int64_t>(kblocks) * kTileCodeBytes + static_cast<int64_t>(kb) * kMxTileScaleBytes;
+}
 
 inline size_t tile_bytes(int layout) { return layout == ZQ_WEIGHTS_MX ? kMxTileBytes : kTileBytes; }
 
@@ -207,6 +215,16 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
+// The same for a 4-D tensor map.
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* m, int c0, int c1, int c2, int c3,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2),
+        "r"(c3)
       : "memory");
 }
 

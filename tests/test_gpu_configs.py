@@ -28,7 +28,7 @@ def _sample_rows(M, bms, seed, full=True):
     rows = {0, M - 1}
     for bm in bms:
         n_tiles = (M + bm - 1) // bm
-        tiles = range(n_tiles) if full else sorted({0, 1, n_tiles - 1})
+        tiles = range(n_tiles) if full else sorted({0, min(1, n_tiles - 1), n_tiles - 1})
         for ti in tiles:
             lo, hi = ti * bm, min((ti + 1) * bm, M)
             rows.update((lo, hi - 1))
@@ -37,6 +37,7 @@ def _sample_rows(M, bms, seed, full=True):
             if full:
                 rows.add(int(rng.integers(lo, hi)))
     rows.update(int(v) for v in rng.integers(0, M, size=32 if full else 8))
+    assert all(0 <= v < M for v in rows)
     return sorted(rows)
 
 
