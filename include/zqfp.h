@@ -203,6 +203,16 @@ int zq_w4a8_linear_host(const void* x_bf16_host, int64_t M, int64_t N, int64_t K
 int zq_device_status(void* workspace, int* detail, void* stream);
 
 /*
+ * (No operation of the paper: a check of the library's own failure reporting.)  Launches one CTA that waits,
+ * with the wait routine the GEMM kernels use and a limit of `limit_us` microseconds (1 .. 1000000), on a
+ * barrier that nothing ever completes.  The wait gives up, the kernel writes ZQ_ERR_DEVICE_TIMEOUT and the
+ * detail code 100 into the workspace status words and returns by itself: no trap, no fault, nothing left
+ * spinning.  zq_device_status(workspace) then returns ZQ_ERR_DEVICE_TIMEOUT and clears the words; the same
+ * workspace is usable again after zq_workspace_init.
+ */
+int zq_selftest_bounded_wait(void* workspace, size_t workspace_bytes, uint32_t limit_us, void* stream);
+
+/*
  * (The paper has no counterpart for this entry point; it exists for deployment reasons only.)
  *
  * zq_w4a8_linear for callers that cannot allocate device memory and therefore have no workspace to

@@ -26,7 +26,7 @@ EXPORTS = [
     "zq_status_string", "zq_quantize_act_fp8", "zq_packed_weight_sizes", "zq_pack_weight_fp4",
     "zq_w4a8_linear_workspace_bytes", "zq_workspace_init", "zq_w4a8_linear",
     "zq_w4a8_linear_host_workspace_bytes", "zq_w4a8_linear_host", "zq_device_status", "zq_launch_count",
-    "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc", "zq_w4a8_linear_noalloc_status", "zq_w4a8_linear_plan",
+    "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc", "zq_w4a8_linear_noalloc_status", "zq_w4a8_linear_plan", "zq_selftest_bounded_wait",
 ]
 PLAN_FIELDS = ("bm", "m_tiles", "n_tiles", "ctas", "stream", "persist", "splits", "kb_per_split", "base", "rem",
                "tail_pos0", "m_group", "partial_floats", "sms")
@@ -80,6 +80,8 @@ def lib() -> C.CDLL:
         L.zq_w4a8_linear_noalloc.argtypes = [vp, vp, i64, i64, i64, ci, ci, vp, vp, vp, vp, vp, ci, vp, ci, i64, vp]
         L.zq_w4a8_linear_noalloc_status.restype = ci
         L.zq_w4a8_linear_noalloc_status.argtypes = [C.POINTER(ci), vp]
+        L.zq_selftest_bounded_wait.restype = ci
+        L.zq_selftest_bounded_wait.argtypes = [vp, sz, C.c_uint32, vp]
         _lib = L
     return _lib
 
@@ -230,6 +232,12 @@ def w4a8_linear_noalloc(w: PackedWeight, *, q, sx, t=None, U=None, y=None, out_d
                                         _ptr(scale), _ptr(U), _ptr(t), r, _ptr(y), ydt, ldy, _stream()),
            "zq_w4a8_linear_noalloc")
     return y
+
+
+def selftest_bounded_wait(workspace: torch.Tensor, limit_us: int = 1000):
+    """Launches the kernel whose bounded wait is meant to run out; read the outcome with device_status()."""
+    _check(lib().zq_selftest_bounded_wait(_ptr(workspace), workspace.numel(), int(limit_us), _stream()),
+           "zq_selftest_bounded_wait")
 
 
 def noalloc_status():

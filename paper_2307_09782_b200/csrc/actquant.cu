@@ -76,6 +76,8 @@ template <bool CACHED>
 __global__ void __launch_bounds__(kMaxThreads)
 act_quant_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, uint8_t* __restrict__ q,
                  float* __restrict__ sx, const uint4* __restrict__ V, int r, float* __restrict__ t) {
+  pdl_launch_dependents();
+  pdl_wait();  // x may be the output of the kernel before this one
   const int64_t m = blockIdx.x;
   const int nunits = K / kUnit;
   const uint4* row = x + m * ldx_vec;  // 8 bf16 per uint4
@@ -208,6 +210,8 @@ act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec
   __shared__ float s_amax[kRowsWarps][kRows];
   __shared__ float s_acc[kRowsWarps][kRows * 8];
   __shared__ float s_inv[kRows];
+  pdl_launch_dependents();
+  pdl_wait();  // x may be the output of the kernel before this one
   const int m0 = blockIdx.x * kRows;
   const int nrows = min(kRows, M - m0);
   const int nvec = K / 8;  // 16-byte vectors per row
@@ -297,6 +301,8 @@ act_quant_cluster_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, ui
                          float* __restrict__ sx, const uint4* __restrict__ V, int r, float* __restrict__ t) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
+  pdl_launch_dependents();
+  pdl_wait();  // x may be the output of the kernel before this one
   const int rank = static_cast<int>(cluster.block_rank());
   const int64_t m = blockIdx.y;
   const int nunits = K / kUnit;
@@ -399,28 +405,31 @@ act_quant_cluster_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, ui
 int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
                      const void* V, int r, float* t, cudaStream_t st) {
   if (M == 0) return ZQ_OK;
+  cudaError_t err = cudaSuccess;
   // enough rows for the eight-row CTAs to beat one row per CTA (measured: from about 50 CTAs on), and the
   // rank the row kernel is written for
   if (M >= kRowsMinTokens && (V == nullptr || r == 8)) {
     dim3 grid(static_cast<unsigned>((M + kRows - 1) / kRows));
     if (V)
-      act_quant_rows_kernel<true><<<grid, kRowsThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(M),
-                                                                static_cast<int>(K), ldx / 8, q, sx,
-                                                                static_cast<const uint4*>(V), t);
+      err = launch_chained(act_quant_rows_kernel<true>, grid, dim3(kRowsThreads), 0, st, false,
+                           static_cast<const uint4*>(x), static_cast<int>(M), static_cast<int>(K), ldx / 8, q, sx,
+                           static_cast<const uint4*>(V), t);
     else
-      act_quant_rows_kernel<false><<<grid, kRowsThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(M),
-                                                                 static_cast<int>(K), ldx / 8, q, sx, nullptr, t);
+      err = launch_chained(act_quant_rows_kernel<false>, grid, dim3(kRowsThreads), 0, st, false,
+                           static_cast<const uint4*>(x), static_cast<int>(M), static_cast<int>(K), ldx / 8, q, sx,
+                           static_cast<const uint4*>(nullptr), t);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+    return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
   }
   // fewer tokens than the eight-row kernel needs, rows long enough to be worth sharing: a cluster of eight CTAs per row
   if (M < kRowsMinTokens && (M <= 256 || K >= 16384) && K >= 2048 &&
       K / kUnit <= kClusterSize * kClusterThreads * kClusterVpt) {
     dim3 grid(kClusterSize, static_cast<unsigned>(M));
-    act_quant_cluster_kernel<<<grid, kClusterThreads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(K),
-                                                              ldx / 8, q, sx, static_cast<const uint4*>(V), r, t);
+    err = launch_chained(act_quant_cluster_kernel, grid, dim3(kClusterThreads), 0, st, false,
+                         static_cast<const uint4*>(x), static_cast<int>(K), ldx / 8, q, sx,
+                         static_cast<const uint4*>(V), r, t);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+    return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
   }
   const int nunits = static_cast<int>(K / kUnit);
   int threads = ((nunits + 31) / 32) * 32;
@@ -428,13 +437,13 @@ int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* 
   const bool cached = nunits <= threads * kVpt;
   dim3 grid(static_cast<unsigned>(M));
   if (cached)
-    act_quant_kernel<true><<<grid, threads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(K), ldx / 8, q,
-                                                     sx, static_cast<const uint4*>(V), r, t);
+    err = launch_chained(act_quant_kernel<true>, grid, dim3(threads), 0, st, false, static_cast<const uint4*>(x),
+                         static_cast<int>(K), ldx / 8, q, sx, static_cast<const uint4*>(V), r, t);
   else
-    act_quant_kernel<false><<<grid, threads, 0, st>>>(static_cast<const uint4*>(x), static_cast<int>(K), ldx / 8, q,
-                                                      sx, static_cast<const uint4*>(V), r, t);
+    err = launch_chained(act_quant_kernel<false>, grid, dim3(threads), 0, st, false, static_cast<const uint4*>(x),
+                         static_cast<int>(K), ldx / 8, q, sx, static_cast<const uint4*>(V), r, t);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
 }
 
 }  // namespace zq

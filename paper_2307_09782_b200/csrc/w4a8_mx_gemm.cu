@@ -132,6 +132,29 @@ struct Segments {
   }
 };
 
+// One pipeline stage at a time through a CTA's segments, in the order the MMAs take them: the stage holds
+// the K blocks kb .. kb + nk - 1 (nk <= KPS) of the output tile `tile`.
+template <int KPS>
+struct StageWalker {
+  Segments sg;
+  int tile = 0, kb = 0, left = 0;
+  __device__ __forceinline__ explicit StageWalker(const Segments& s) : sg(s) {}
+  __device__ __forceinline__ bool next(const Params& p, int& o_tile, int& o_kb) {
+    if (left == 0) {
+      int pos, kb0, nkb;
+      if (!sg.next(p, pos, tile, kb0, nkb)) return false;
+      kb = kb0;
+      left = nkb;
+    }
+    o_tile = tile;
+    o_kb = kb;
+    const int nk = min(KPS, left);
+    kb += nk;
+    left -= nk;
+    return true;
+  }
+};
+
 template <int BM>
 __global__ void __launch_bounds__(MxCfg<BM>::kThreads, MxCfg<BM>::kMinBlocks)
 w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
@@ -196,41 +219,62 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
 
   Segments sg(p);
   int pos, tile, kb0, nkb;
+  if (threadIdx.x == 0) pdl_launch_dependents();  // the next kernel of the stream may begin its own setup
 
   if (warp == C::kProducerWarp) {
     // ------------------------------------------------------------------ producer
     if (ok_start) {  // warp-uniform loops, one elected lane issues the copies
       const bool issuer = elect_one();
+      // The copies of one stage.  The boxes always span kKps K blocks (beyond the row's last K block the copy
+      // engine fills in zeros; a K block past the end of this CTA's range is read but not used); the scales
+      // are copied for the K blocks that exist only, never past the row's end.
+      auto issue_weights = [&](int s, int tile_, int kb) {
+        if (issuer) {
+          const int nt = tile_ % p.n_tiles;
+          const uint8_t* sf_row =
+              p.codes + static_cast<int64_t>(nt) * p.kblocks * kMxTileBytes + mx_scale_offset(p.kblocks, 0);
+          const int nsf = min(C::kKps, p.kblocks - kb);
+          mbar_arrive_expect_tx(&full[s], C::kStageTxBoxes + nsf * kMxTileScaleBytes);  // the tokens' bytes too
+          tma_load_4d(s_a + s * C::kABytes, &tm_w, 0, 0, kb, nt, &full[s]);
+          bulk_load(s_sf + s * C::kSfBytes, sf_row + static_cast<int64_t>(kb) * kMxTileScaleBytes,
+                    nsf * kMxTileScaleBytes, &full[s]);
+        }
+      };
+      auto issue_tokens = [&](int s, int tile_, int kb) {
+        if (issuer) tma_load_3d(s_tok + s * C::kTokBytes, &tm_q, 0, (tile_ / p.n_tiles) * BM, kb, &full[s]);
+      };
       int s = 0, issued = 0;
       uint32_t ph = 0;
       bool ok = true;
-      while (ok && sg.next(p, pos, tile, kb0, nkb)) {
-        const int m0 = (tile / p.n_tiles) * BM;
-        const int nt = tile % p.n_tiles;
-        const uint8_t* sf_row = p.codes + static_cast<int64_t>(nt) * p.kblocks * kMxTileBytes + mx_scale_offset(p.kblocks, 0);
-        for (int kb = kb0; kb < kb0 + nkb; kb += C::kKps) {
-          if (!mbar_wait(&empty[s], ph ^ 1, s_abort)) {
-            if (issuer) raise_error(p, s_abort, kErrProducer);
-            ok = false;
-            break;
-          }
-          if (issuer) {
-            // The boxes always span kKps K blocks (beyond the row's last K block the copy engine fills in
-            // zeros; a K block past the end of this CTA's range is read but not used); the scales are copied
-            // for the K blocks that exist only, never past the row's end.
-            const int nsf = min(C::kKps, p.kblocks - kb);
-            mbar_arrive_expect_tx(&full[s], C::kStageTxBoxes + nsf * kMxTileScaleBytes);
-            tma_load_4d(s_a + s * C::kABytes, &tm_w, 0, 0, kb, nt, &full[s]);
-            bulk_load(s_sf + s * C::kSfBytes, sf_row + static_cast<int64_t>(kb) * kMxTileScaleBytes,
-                      nsf * kMxTileScaleBytes, &full[s]);
-            tma_load_3d(s_tok + s * C::kTokBytes, &tm_q, 0, m0, kb, &full[s]);
-          }
-          __syncwarp();
-          ++issued;
-          if (++s == C::NS) {
-            s = 0;
-            ph ^= 1;
-          }
+      StageWalker<C::kKps> w(sg), w_tok(sg);
+      int w_tile, w_kb;
+      // The weights are the layer's own read-only data: the copies of the first NS stages (all free at the
+      // start) go out before the wait for the kernel ahead in the stream, whose output the tokens may be.
+      while (issued < C::NS && w.next(p, w_tile, w_kb)) {
+        issue_weights(issued, w_tile, w_kb);
+        ++issued;
+      }
+      __syncwarp();
+      pdl_wait();
+      for (int i = 0; i < issued; ++i) {
+        w_tok.next(p, w_tile, w_kb);
+        issue_tokens(i, w_tile, w_kb);
+      }
+      __syncwarp();
+      if (issued == C::NS) ph = 1;  // the ring has wrapped once
+      while (ok && w.next(p, w_tile, w_kb)) {
+        if (!mbar_wait(&empty[s], ph ^ 1, s_abort)) {
+          if (issuer) raise_error(p, s_abort, kErrProducer);
+          ok = false;
+          break;
+        }
+        issue_weights(s, w_tile, w_kb);
+        issue_tokens(s, w_tile, w_kb);
+        __syncwarp();
+        ++issued;
+        if (++s == C::NS) {
+          s = 0;
+          ph ^= 1;
         }
       }
       // never leave with copies still in flight: wait (bounded) for the last phase issued per stage
@@ -311,6 +355,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
     constexpr int EC = BM <= 32 ? 4 : (BM <= 128 ? 8 : 16);  // columns per step
     bool failed = !ok_start;
     int m0_loaded = -1;
+    pdl_wait();  // sx, t, the hand-over flags and y may still be in use by the kernel ahead in the stream
 
     // Every thread walks every segment and executes the same named-barrier sequence whether or not it
     // has failed, so a bounded wait that ran out can never leave others stuck at a hardware barrier.
@@ -539,6 +584,13 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
     pc.atomic_y = 1;
     pc.handover = 1;
     void* args[3] = {&tm_w, &tm_q, &pc};
+    // chained to the kernel ahead (see pdl_wait); if the two launch attributes are refused together, cooperative alone
+    if (launch_chained(w4a8_mx_gemm_kernel<BM>, grid, dim3(C::kThreads), C::kSmemBytes, st, true, tm_w, tm_q, pc) ==
+        cudaSuccess) {
+      count_launch();
+      return ZQ_OK;
+    }
+    (void)cudaGetLastError();
     if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM>), grid, dim3(C::kThreads),
                                     args, C::kSmemBytes, st) == cudaSuccess) {
       count_launch();
@@ -549,9 +601,10 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
                                         static_cast<size_t>(a.M), st) != cudaSuccess)
       return ZQ_ERR_CUDA;
   }
-  w4a8_mx_gemm_kernel<BM><<<grid, C::kThreads, C::kSmemBytes, st>>>(tm_w, tm_q, p);
+  const cudaError_t err = launch_chained(w4a8_mx_gemm_kernel<BM>, grid, dim3(C::kThreads), C::kSmemBytes, st, false,
+                                         tm_w, tm_q, p);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? ZQ_OK : ZQ_ERR_CUDA;
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
 }
 
 }  // namespace

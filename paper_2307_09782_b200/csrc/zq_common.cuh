@@ -101,8 +101,42 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout);
 int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st);           // ZQ_WEIGHTS_CAST
 int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st);        // ZQ_WEIGHTS_MX
 int sm_count();
+constexpr int kErrDetailSelfTest = 100;  // status detail written by zq_selftest_bounded_wait
 
 #ifdef __CUDACC__
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// The kernels of one layer (quantizer, then GEMM) and of consecutive layers are chained with programmatic
+// stream serialization: a kernel lets its successor start early (launch_dependents), and every kernel waits
+// for its predecessor's completion (pdl_wait) before it touches anything the predecessor may have written.
+// What runs before that wait is setup, and in the GEMM the first weight copies (weights are read-only data
+// of the layer).  A kernel launched without such a predecessor passes the wait at once.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Launch with the programmatic-serialization attribute (and, if asked, as a cooperative launch).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  bool cooperative, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  unsigned n = 0;
+  at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cooperative) {
+    at[n].id = cudaLaunchAttributeCooperative;
+    at[n].val.cooperative = 1;
+    ++n;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = n;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- device: bounded waits -----------------------------------------------------------------------
 // Every wait in this library is bounded (a poll count and, for the parked waits, two seconds of
 // wall time); when one runs out the kernel records an error in the workspace status word and
@@ -158,13 +192,14 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // Bounded wait.  Returns false when kWaitLimitNs passed or another thread of the CTA already raised
 // `abort_flag`; the caller then records the error and unwinds.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
     if (mbar_try_wait_parked(bar, parity, 50000u)) return true;
     if (*abort_flag) return false;
-    if ((spin & 7u) == 7u && global_timer_ns() - t0 > kWaitLimitNs) return false;
+    if (((spin & 7u) == 7u || limit_ns < kWaitLimitNs) && global_timer_ns() - t0 > limit_ns) return false;
   }
   return false;
 }

@@ -187,3 +187,21 @@ def test_host_buffer_entry_point():
     c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, 128, "M1")
     y_o = oracle.w4a8_linear(q_o, sx_o, c_o, sh_o, sc_o, 128, "M1", U, t_o)
     assert np.abs(yh.numpy() - y_o).max() <= TOL_REL * np.abs(y_o).max()
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    # the failure path of every in-kernel wait: record ZQ_ERR_DEVICE_TIMEOUT, return, nothing hangs or faults
+    x_bits, W, U, V = _layer(7, 16, 256, 512, 8)
+    ws = binding.make_workspace(binding.linear_workspace_bytes(16, 256, 512, 8))
+    binding.selftest_bounded_wait(ws, limit_us=1000)
+    assert binding.device_status(ws) == (-8, 100)
+    assert binding.device_status(ws)[0] == 0          # reading the status cleared it
+    binding.lib().zq_workspace_init(ws.data_ptr(), ws.numel(), None)
+    for layout in (binding.WEIGHTS_CAST, binding.WEIGHTS_MX):   # a normal call on the re-initialized workspace
+        pw = binding.pack_weight_fp4(up(W), 128, "M2", layout)
+        y = binding.w4a8_linear(pw, x=to_bf16(x_bits), U=up(U), V=up(V), workspace=ws)
+        assert binding.device_status(ws) == (0, 0)
+        q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
+        c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, 128, "M2")
+        y_o = oracle.w4a8_linear(q_o, sx_o, c_o, sh_o, sc_o, 128, "M2", U, t_o)
+        assert np.abs(host(y).astype(np.float64) - y_o).max() <= TOL_REL * np.abs(y_o).max()
