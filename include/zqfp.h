@@ -45,8 +45,15 @@ typedef enum { ZQ_OUT_F32 = 0, ZQ_OUT_BF16 = 1 } zq_out_dtype;
  * ("Casting the FP4 to FP8") during the GEMM.  Codes, shifts and scales are the same either way. */
 typedef enum {
   ZQ_WEIGHTS_CAST = 0, /* the kernel casts each code to E4M3 itself, as an exponent-field subtraction */
-  ZQ_WEIGHTS_MX = 1    /* modes M1 / M2 only: the tensor core reads the E2M1 codes directly and applies the
+  ZQ_WEIGHTS_MX = 1,   /* modes M1 / M2 only: the tensor core reads the E2M1 codes directly and applies the
                           power-of-two shift of each group as an E8M0 block scale (exact, being a power of two) */
+  ZQ_WEIGHTS_MX_FP8 = 2,    /* modes M1 / M2 only: FP8-E4M3 weight codes instead of FP4 (the W8A8 FP - FP rows of
+                               Table 2; group scale absmax / 448), in the block-scaled arrangement: the same GEMM
+                               without the cast */
+  ZQ_WEIGHTS_CAST_E5M2 = 3  /* modes M1 / M2 only: as ZQ_WEIGHTS_CAST, but the kernel casts each code to E5M2 (Section
+                               3, footnote to "Casting the FP4 to FP8"), whose five exponent bits keep the cast a
+                               subtraction in the exponent field down to a shift of 13; shifts are stored clamped
+                               to [0, 13] */
 } zq_weight_layout;
 
 const char* zq_status_string(int status);
@@ -71,7 +78,8 @@ int zq_quantize_act_fp8(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, u
 
 /*
  * Sizes in bytes of the three buffers zq_pack_weight_fp4 writes:
- *   codes: ceil(N/128) * (K/128) * 8448 (ZQ_WEIGHTS_CAST) or * 8704 (ZQ_WEIGHTS_MX), tiled, see below ;
+ *   codes: ceil(N/128) * (K/128) * 8448 (ZQ_WEIGHTS_CAST, ZQ_WEIGHTS_CAST_E5M2), * 8704 (ZQ_WEIGHTS_MX) or
+ *          * 16896 (ZQ_WEIGHTS_MX_FP8), tiled, see below ;
  *   shift: N*G (M1, M2) or 0 (none) ;
  *   scale: 4*N (M1, M2) or 4*N*G (none).
  */
@@ -111,9 +119,14 @@ int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, 
  *             32s .. 32s+31 of K block kb (the E8M0 encoding of 2^-shift), the order in which the tensor
  *             core's scale copy reads them.
  *         Rows beyond N have zero codes and scale bytes 127.
+ *         With ZQ_WEIGHTS_MX_FP8 the codes are E4M3 bytes, code = RNE_E4M3(fl32(W / S^)) saturating at +-448
+ *         with S_j = max|W| / 448, one byte per element: a block of 128 output rows takes (K/128) * 16896
+ *         bytes, [kb*16384, +16384) holding K block kb with row r at r*128, then the scale bytes as above
+ *         from (K/128)*16384 on; shifts are stored clamped to [0, 127].
  * shift : out, u8 [N, G] (M1, M2), the same shifts in plain form; ignored (may be NULL) in mode none
  * scale : out, FP32 [N] (M1, M2) or [N, G] (none)
- * group in {64, 128, 256}; K % group == 0 and K % 128 == 0; N >= 0.
+ * group in {64, 128, 256, 320} (320, the paper's choice for a hidden size of 3200, with M1 / M2 only);
+ * K % group == 0 and K % 128 == 0; N >= 0.
  */
 int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale_mode mode,
                        zq_weight_layout layout, uint8_t* codes, uint8_t* shift, float* scale, void* stream);
@@ -146,7 +159,7 @@ int zq_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  *                 (the tiles carry the shifts) and may be NULL
  * U : fp16 [N, r] dense or NULL (r = 0);  V : fp16 [r, K], only read when x_bf16 is given and r > 0
  * y : out, [M, ldy] FP32 or bf16 (ydt), ldy >= N in elements
- * K % 128 == 0; group in {64, 128, 256}; r in {0, 8, 16, ..., 64}; q, codes 16-byte aligned (codes 32-byte
+ * K % 128 == 0; group in {64, 128, 256, 320}; r in {0, 8, 16, ..., 64}; q, codes 16-byte aligned (codes 32-byte
  * aligned with ZQ_WEIGHTS_MX).
  * M == 0 or N == 0 is a no-op.  Summation order over K depends on the launch shape, so FP32 results are
  * not bit-identical across token counts.  Where the K range of an output tile is shared by several CTAs

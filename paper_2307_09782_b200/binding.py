@@ -19,8 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libzqfp.so")
 SCALE_NONE, SCALE_M1, SCALE_M2 = 0, 1, 2
 MODES = {"none": SCALE_NONE, "M1": SCALE_M1, "M2": SCALE_M2}
 OUT_F32, OUT_BF16 = 0, 1
-WEIGHTS_CAST, WEIGHTS_MX = 0, 1
-LAYOUTS = {"cast": WEIGHTS_CAST, "mx": WEIGHTS_MX}
+WEIGHTS_CAST, WEIGHTS_MX, WEIGHTS_MX_FP8, WEIGHTS_CAST_E5M2 = 0, 1, 2, 3
+LAYOUTS = {"cast": WEIGHTS_CAST, "mx": WEIGHTS_MX, "mx_fp8": WEIGHTS_MX_FP8, "cast_e5m2": WEIGHTS_CAST_E5M2}
 
 EXPORTS = [
     "zq_status_string", "zq_quantize_act_fp8", "zq_packed_weight_sizes", "zq_pack_weight_fp4",

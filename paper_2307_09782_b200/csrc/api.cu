@@ -23,10 +23,14 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 bool valid_mode(int mode) { return mode == ZQ_SCALE_NONE || mode == ZQ_SCALE_M1 || mode == ZQ_SCALE_M2; }
-bool valid_group(int g) { return g == 64 || g == 128 || g == 256; }
-// the tensor core's block scales are powers of two: only the constrained modes can use that layout
+// 320 does not divide the 128-element K block: the per-group promotion of mode none is not written for it
+bool valid_group(int g, int mode) { return g == 64 || g == 128 || g == 256 || (g == 320 && mode != ZQ_SCALE_NONE); }
+// the tensor core's block scales are powers of two, and E5M2 as the cast target is about the shifts: only
+// the constrained modes can use those layouts
 bool valid_layout(int layout, int mode) {
-  return layout == ZQ_WEIGHTS_CAST || (layout == ZQ_WEIGHTS_MX && mode != ZQ_SCALE_NONE);
+  return layout == ZQ_WEIGHTS_CAST ||
+         ((layout == ZQ_WEIGHTS_MX || layout == ZQ_WEIGHTS_MX_FP8 || layout == ZQ_WEIGHTS_CAST_E5M2) &&
+          mode != ZQ_SCALE_NONE);
 }
 inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 // the sizes every linear entry point and size query accepts (the group size is checked where it is known)
@@ -131,7 +135,7 @@ int zq_quantize_act_fp8(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_
 int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout,
                            size_t* codes_bytes, size_t* shift_bytes, size_t* scale_bytes) {
   if (!valid_mode(mode) || !valid_layout(layout, mode)) return ZQ_ERR_MODE;
-  if (N < 0 || K <= 0 || !valid_group(group) || K % group || K % kTileK) return ZQ_ERR_SHAPE;
+  if (N < 0 || K <= 0 || !valid_group(group, mode) || K % group || K % kTileK) return ZQ_ERR_SHAPE;
   const size_t G = static_cast<size_t>(K / group);
   if (codes_bytes)
     *codes_bytes = static_cast<size_t>((N + kTileRows - 1) / kTileRows) * static_cast<size_t>(K / kTileK) * tile_bytes(layout);
@@ -143,7 +147,7 @@ int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, 
 int zq_pack_weight_fp4(const float* W, int64_t N, int64_t K, int group, zq_scale_mode mode,
                        zq_weight_layout layout, uint8_t* codes, uint8_t* shift, float* scale, void* stream) {
   if (!valid_mode(mode) || !valid_layout(layout, mode)) return ZQ_ERR_MODE;
-  if (N < 0 || K <= 0 || !valid_group(group) || K % group || K % kTileK || N > 0x7FFFFFFF - kTileRows ||
+  if (N < 0 || K <= 0 || !valid_group(group, mode) || K % group || K % kTileK || N > 0x7FFFFFFF - kTileRows ||
       K > (int64_t(1) << 30))
     return ZQ_ERR_SHAPE;
   if (N == 0) return ZQ_OK;
@@ -177,7 +181,7 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
                    void* y, zq_out_dtype ydt, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
   if (!valid_mode(mode) || !valid_layout(layout, mode) || (ydt != ZQ_OUT_F32 && ydt != ZQ_OUT_BF16))
     return ZQ_ERR_MODE;
-  if (!valid_linear_shape(M, N, K, r) || !valid_group(group) || K % group || ldy < N) return ZQ_ERR_SHAPE;
+  if (!valid_linear_shape(M, N, K, r) || !valid_group(group, mode) || K % group || ldy < N) return ZQ_ERR_SHAPE;
   if (M == 0 || N == 0) return ZQ_OK;
   if (!codes || !scale || !y || (r > 0 && !U)) return ZQ_ERR_NULL;
   if (x_bf16) {
@@ -188,7 +192,7 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
   }
   if (!aligned16(codes) || (q && !aligned16(q)) || (U && !aligned16(U)) || (t && !aligned16(t)) ||
       (x_bf16 && (!aligned16(x_bf16) || ldx % 8 || (V && !aligned16(V)))) ||
-      (layout == ZQ_WEIGHTS_MX && !aligned32(codes)))
+      (layout_is_mx(layout) && !aligned32(codes)))
     return ZQ_ERR_ALIGN;
   if (!workspace) return ZQ_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) & 255u) return ZQ_ERR_ALIGN;
@@ -233,7 +237,7 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
   a.counters = reinterpret_cast<int*>(ws + kWsStatusBytes);
   a.partials = reinterpret_cast<float*>(ws + w.off_partials);
   a.partial_floats = w.partial_floats;
-  return layout == ZQ_WEIGHTS_MX ? launch_w4a8_mx_gemm(a, st) : launch_w4a8_gemm(a, st);
+  return layout_is_mx(layout) ? launch_w4a8_mx_gemm(a, st) : launch_w4a8_gemm(a, st);
 }
 
 int zq_w4a8_linear_plan(int64_t M, int64_t N, int64_t K, zq_scale_mode mode, zq_weight_layout layout,
@@ -287,7 +291,7 @@ int zq_w4a8_linear_host(const void* x_host, int64_t M, int64_t N, int64_t K, int
                         const void* U, const void* V, int r, float* y_host, void* workspace, size_t workspace_bytes,
                         void* stream) {
   if (!valid_mode(mode) || !valid_layout(layout, mode)) return ZQ_ERR_MODE;
-  if (!valid_linear_shape(M, N, K, r) || !valid_group(group) || K % group) return ZQ_ERR_SHAPE;
+  if (!valid_linear_shape(M, N, K, r) || !valid_group(group, mode) || K % group) return ZQ_ERR_SHAPE;
   if (M == 0 || N == 0) return ZQ_OK;
   if (!x_host || !y_host) return ZQ_ERR_NULL;
   if (!workspace) return ZQ_ERR_WORKSPACE;

@@ -246,7 +246,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
     // The whole warp runs the loop (uniform control flow and addresses); one elected lane issues.
     if (ok_start) {
       const bool issuer = elect_one();
-      const uint32_t idesc = umma_idesc_e4m3(BM);
+      const uint32_t idesc = umma_idesc_e4m3(BM) | (p.cast_e5m2 ? (1u << 7) : 0u);  // A operand E4M3 or E5M2
       const uint64_t bdesc0 = umma_desc_k128(smem_u32(s_tok));
       const int mpg = p.group / 32;  // MMAs per weight group (mode none)
       int mma_count = 0;
@@ -381,8 +381,10 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             const uint32_t d = (d2 >> (8 * h)) & 0xFFu;
-            const uint32_t lut_lo = 0x3C383000u - d * 0x08080800u;
-            const uint32_t lut_hi = 0x4C484440u - d * 0x08080808u;
+            // the magnitudes 0, 0.5, 1, 1.5 | 2, 3, 4, 6 as E4M3 bytes (exponent field from bit 3) or as E5M2
+            // bytes (from bit 2), the shift subtracted from the exponent field of every non-zero entry
+            const uint32_t lut_lo = p.cast_e5m2 ? 0x3E3C3800u - d * 0x04040400u : 0x3C383000u - d * 0x08080800u;
+            const uint32_t lut_hi = p.cast_e5m2 ? 0x46444240u - d * 0x04040404u : 0x4C484440u - d * 0x08080808u;
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
               const uint4 v = pk[2 * h + c];
@@ -622,7 +624,7 @@ int sm_count() {
 
 GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   GemmPlan pl{};
-  const bool mx = layout == ZQ_WEIGHTS_MX;
+  const bool mx = layout_is_mx(layout);
   const int bm_max = (mode == ZQ_SCALE_NONE) ? 64 : 256;
   int bm = 16;
   while (bm < bm_max && bm < M) bm *= 2;
@@ -722,7 +724,8 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
 int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st) {
   const GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode, ZQ_WEIGHTS_CAST);
   if (plan.partial_floats > a.partial_floats) return ZQ_ERR_WORKSPACE;
-  const Params p = make_params(a, plan);
+  Params p = make_params(a, plan);
+  p.cast_e5m2 = a.layout == ZQ_WEIGHTS_CAST_E5M2 ? 1 : 0;
   const bool none = a.mode == ZQ_SCALE_NONE;
   switch (plan.bm) {
     case 16: return none ? launch_cfg<16, true>(a, plan, p, st) : launch_cfg<16, false>(a, plan, p, st);

@@ -54,6 +54,7 @@ struct Params {
   int* status;
   int* counters;
   float* partials;
+  int cast_e5m2;  // the kernel that casts: E5M2 instead of E4M3 as the cast target
 };
 
 constexpr int cmin(int a, int b) { return a < b ? a : b; }

@@ -43,13 +43,17 @@ using namespace gemm;
 
 constexpr int kSfbCols = 16;  // token-side block scales (all one): room for 256 tokens, written once
 
-template <int BM>
+// W8: the weight codes are FP8-E4M3 bytes (layout ZQ_WEIGHTS_MX_FP8) instead of packed E2M1 nibbles: 16 KB per
+// tile in HBM, copied as they are (they fill the same 16 KB of shared memory as the padded FP4 form).
+template <int BM, bool W8>
 struct MxCfg {
   // One CTA per SM: launches whose CTAs share output tiles are cooperative, and a cooperative launch of a
   // kernel that allocates tensor memory is given one CTA per SM (the occupancy query answers 1 whatever the
   // registers and shared memory; with two CTAs per SM planned, grids beyond the SM count were refused).
   static constexpr int kMinBlocks = 1;
   static constexpr int kKps = BM <= 64 ? 2 : 1;  // K blocks per pipeline stage
+  static constexpr int kCodeBytes = W8 ? 2 * kTileCodeBytes : kTileCodeBytes;  // a tile's codes in HBM
+  static constexpr int kTileBytesHbm = kCodeBytes + kMxTileScaleBytes;
   static constexpr int kProducerWarp = 4;
   static constexpr int kMmaWarp = 5;
   static constexpr int kThreads = 192;
@@ -61,7 +65,7 @@ struct MxCfg {
   static constexpr int kSfBytes = kKps * kMxTileScaleBytes;
   // bytes a stage's barrier counts besides the scales (whole boxes: what lies beyond the tensor is filled
   // with zeros and counted too)
-  static constexpr int kStageTxBoxes = kKps * kTileCodeBytes + kTokBytes;
+  static constexpr int kStageTxBoxes = kKps * kCodeBytes + kTokBytes;
   static constexpr int kBudget = (kMinBlocks == 1 ? 220 : 110) * 1024 - BM * 36 - 512;
   static constexpr int NS = cmin(12, kBudget / (kABytes + kSfBytes + kTokBytes));
   static constexpr int NB = BM <= 224 ? 2 : 1;  // accumulator buffers
@@ -155,11 +159,11 @@ struct StageWalker {
   }
 };
 
-template <int BM>
-__global__ void __launch_bounds__(MxCfg<BM>::kThreads, MxCfg<BM>::kMinBlocks)
+template <int BM, bool W8>
+__global__ void __launch_bounds__(MxCfg<BM, W8>::kThreads, MxCfg<BM, W8>::kMinBlocks)
 w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
                     const Params p) {
-  using C = MxCfg<BM>;
+  using C = MxCfg<BM, W8>;
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* s_a = smem + C::offA;
   uint8_t* s_tok = smem + C::offTok;
@@ -231,8 +235,8 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       auto issue_weights = [&](int s, int tile_, int kb) {
         if (issuer) {
           const int nt = tile_ % p.n_tiles;
-          const uint8_t* sf_row =
-              p.codes + static_cast<int64_t>(nt) * p.kblocks * kMxTileBytes + mx_scale_offset(p.kblocks, 0);
+          const uint8_t* sf_row = p.codes + static_cast<int64_t>(nt) * p.kblocks * C::kTileBytesHbm +
+                                  static_cast<int64_t>(p.kblocks) * C::kCodeBytes;  // the row block's scales
           const int nsf = min(C::kKps, p.kblocks - kb);
           mbar_arrive_expect_tx(&full[s], C::kStageTxBoxes + nsf * kMxTileScaleBytes);  // the tokens' bytes too
           tma_load_4d(s_a + s * C::kABytes, &tm_w, 0, 0, kb, nt, &full[s]);
@@ -321,7 +325,8 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
 #pragma unroll
                 for (int k = 0; k < kBlockK / 32; ++k) {
                   // scale byte k of the K block's four columns belongs to elements 32k .. 32k+31
-                  umma_mxf8f6f4(d_tmem, adesc + 2 * k, bdesc + 2 * k, umma_idesc_mx_e2m1_e4m3(BM, k, 0),
+                  umma_mxf8f6f4(d_tmem, adesc + 2 * k, bdesc + 2 * k,
+                                W8 ? umma_idesc_mx_e4m3_e4m3(BM, k, 0) : umma_idesc_mx_e2m1_e4m3(BM, k, 0),
                                 sfa + (static_cast<uint32_t>(k) << 30), tmem_sfb, (i > 0 || j > 0 || k > 0) ? 1u : 0u);
                 }
               }
@@ -532,14 +537,16 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
 // The packed weight as a 4-D tensor of 4-bit elements [row blocks][K blocks][128 rows][128 elements]; the copy
 // engine expands a box of `kps` 128 x 128 tiles to the 16-byte-aligned FP4 form in shared memory, 128-byte
 // swizzled, one tile after the other.
-bool make_weight_map(CUtensorMap* m, const void* base, uint64_t n_tiles, uint64_t kblocks, uint32_t kps) {
+// (FP8 weights: the same tensor of bytes, copied as it is.)
+bool make_weight_map(CUtensorMap* m, const void* base, uint64_t n_tiles, uint64_t kblocks, uint32_t kps, bool w8) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
+  const uint64_t code_bytes = w8 ? 2 * kTileCodeBytes : kTileCodeBytes;
   const cuuint64_t dims[4] = {kTileK, kTileRows, kblocks, n_tiles};
-  const cuuint64_t strides[3] = {kTileK / 2, kTileCodeBytes, kblocks * kMxTileBytes};
+  const cuuint64_t strides[3] = {code_bytes / kTileRows, code_bytes, kblocks * (code_bytes + kMxTileScaleBytes)};
   const cuuint32_t box[4] = {kTileK, kTileRows, kps, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 4, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(m, w8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 4, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -558,17 +565,17 @@ bool make_token_map(CUtensorMap* m, const void* base, uint64_t K, uint64_t M, ui
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BM>
+template <int BM, bool W8>
 int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStream_t st) {
-  using C = MxCfg<BM>;
+  using C = MxCfg<BM, W8>;
   CUtensorMap tm_w, tm_q;
-  if (!make_weight_map(&tm_w, a.codes, static_cast<uint64_t>(plan.n_tiles), static_cast<uint64_t>(p.kblocks), C::kKps) ||
+  if (!make_weight_map(&tm_w, a.codes, static_cast<uint64_t>(plan.n_tiles), static_cast<uint64_t>(p.kblocks), C::kKps, W8) ||
       !make_token_map(&tm_q, a.q, static_cast<uint64_t>(a.K), static_cast<uint64_t>(a.M), BM, C::kKps))
     return ZQ_ERR_CUDA;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(w4a8_mx_gemm_kernel<BM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    attr_err = cudaFuncSetAttribute(w4a8_mx_gemm_kernel<BM, W8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     C::kSmemBytes);
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
@@ -585,13 +592,13 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
     pc.handover = 1;
     void* args[3] = {&tm_w, &tm_q, &pc};
     // chained to the kernel ahead (see pdl_wait); if the two launch attributes are refused together, cooperative alone
-    if (launch_chained(w4a8_mx_gemm_kernel<BM>, grid, dim3(C::kThreads), C::kSmemBytes, st, true, tm_w, tm_q, pc) ==
+    if (launch_chained(w4a8_mx_gemm_kernel<BM, W8>, grid, dim3(C::kThreads), C::kSmemBytes, st, true, tm_w, tm_q, pc) ==
         cudaSuccess) {
       count_launch();
       return ZQ_OK;
     }
     (void)cudaGetLastError();
-    if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM>), grid, dim3(C::kThreads),
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM, W8>), grid, dim3(C::kThreads),
                                     args, C::kSmemBytes, st) == cudaSuccess) {
       count_launch();
       return ZQ_OK;
@@ -601,7 +608,7 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
                                         static_cast<size_t>(a.M), st) != cudaSuccess)
       return ZQ_ERR_CUDA;
   }
-  const cudaError_t err = launch_chained(w4a8_mx_gemm_kernel<BM>, grid, dim3(C::kThreads), C::kSmemBytes, st, false,
+  const cudaError_t err = launch_chained(w4a8_mx_gemm_kernel<BM, W8>, grid, dim3(C::kThreads), C::kSmemBytes, st, false,
                                          tm_w, tm_q, p);
   count_launch();
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
@@ -614,15 +621,19 @@ int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
   const GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode, ZQ_WEIGHTS_MX);
   if (plan.partial_floats > a.partial_floats) return ZQ_ERR_WORKSPACE;
   const Params p = make_params(a, plan);
+  const bool w8 = a.layout == ZQ_WEIGHTS_MX_FP8;
+#define ZQ_MX_CASE(BM_) \
+  case BM_: return w8 ? launch_mx_cfg<BM_, true>(a, plan, p, st) : launch_mx_cfg<BM_, false>(a, plan, p, st)
   switch (plan.bm) {
-    case 16: return launch_mx_cfg<16>(a, plan, p, st);
-    case 32: return launch_mx_cfg<32>(a, plan, p, st);
-    case 64: return launch_mx_cfg<64>(a, plan, p, st);
-    case 128: return launch_mx_cfg<128>(a, plan, p, st);
-    case 192: return launch_mx_cfg<192>(a, plan, p, st);
-    case 224: return launch_mx_cfg<224>(a, plan, p, st);
-    case 256: return launch_mx_cfg<256>(a, plan, p, st);
+    ZQ_MX_CASE(16);
+    ZQ_MX_CASE(32);
+    ZQ_MX_CASE(64);
+    ZQ_MX_CASE(128);
+    ZQ_MX_CASE(192);
+    ZQ_MX_CASE(224);
+    ZQ_MX_CASE(256);
   }
+#undef ZQ_MX_CASE
   return ZQ_ERR_SHAPE;
 }
 

@@ -54,7 +54,14 @@ __host__ __device__ inline int64_t mx_scale_offset(int kblocks, int kb) {
   return static_cast<int64_t>(kblocks) * kTileCodeBytes + static_cast<int64_t>(kb) * kMxTileScaleBytes;
 }
 
-inline size_t tile_bytes(int layout) { return layout == ZQ_WEIGHTS_MX ? kMxTileBytes : kTileBytes; }
+// Layout ZQ_WEIGHTS_MX_FP8: the same arrangement with one E4M3 byte per element (a tile's codes are 16384 bytes,
+// row r at r * 128), for FP8 weights.
+constexpr int kMx8TileBytes = 2 * kTileCodeBytes + kMxTileScaleBytes;
+
+inline size_t tile_bytes(int layout) {
+  return layout == ZQ_WEIGHTS_MX ? kMxTileBytes : (layout == ZQ_WEIGHTS_MX_FP8 ? kMx8TileBytes : kTileBytes);
+}
+inline bool layout_is_mx(int layout) { return layout == ZQ_WEIGHTS_MX || layout == ZQ_WEIGHTS_MX_FP8; }
 
 // ---- launchers implemented in the .cu files ------------------------------------------------------
 int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
@@ -429,6 +436,11 @@ __device__ __forceinline__ uint64_t umma_desc_rows16(uint32_t smem_addr, uint32_
 // D is 128 x n; sf_id selects which of the four scale bytes of a tensor-memory column this MMA uses.
 __device__ __forceinline__ uint32_t umma_idesc_mx_e2m1_e4m3(uint32_t n, uint32_t a_sf_id, uint32_t b_sf_id) {
   return (b_sf_id << 4) | (5u << 7) | (0u << 10) | ((n >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) |
+         (a_sf_id << 29);
+}
+// The same with an E4M3 A operand (FP8 weights).
+__device__ __forceinline__ uint32_t umma_idesc_mx_e4m3_e4m3(uint32_t n, uint32_t a_sf_id, uint32_t b_sf_id) {
+  return (b_sf_id << 4) | (0u << 7) | (0u << 10) | ((n >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24) |
          (a_sf_id << 29);
 }
 // Instruction descriptor: E4M3 x E4M3 -> FP32, both operands K-major, D is 128 x n.

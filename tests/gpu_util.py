@@ -28,13 +28,20 @@ def untile_codes(tiles: np.ndarray, N: int, K: int, layout=binding.WEIGHTS_CAST)
     """Decodes either tiled weight format (include/zqfp.h) back to plain form:
     returns (codes uint8 [N, K/2] with element 2b in the low nibble of byte b, shifts uint8 [N, K/32])."""
     nt, kb = (N + 127) // 128, K // 128
+    if layout == binding.WEIGHTS_MX_FP8:
+        # a block of 128 output rows: E4M3 bytes of all K blocks (row r of a K block at r * 128), then the scales
+        t = np.ascontiguousarray(tiles, dtype=np.uint8).reshape(nt, kb * 16896)
+        codes = t[:, :kb * 16384].reshape(nt, kb, 128, 128).transpose(0, 2, 1, 3).reshape(nt * 128, K)
+        sf = t[:, kb * 16384:].reshape(nt, kb, 32, 4, 4).transpose(0, 3, 2, 1, 4).reshape(nt * 128, kb * 4)
+        assert not codes[N:].any() and np.all(sf[N:] == 127), "padding rows: zero codes, unit scales"
+        return codes[:N], (127 - sf[:N].astype(np.int32)).astype(np.uint8)
     if layout == binding.WEIGHTS_MX:
         t = np.ascontiguousarray(tiles, dtype=np.uint8).reshape(nt, kb * 8704)   # a block of 128 output rows:
         codes = t[:, :kb * 8192].reshape(nt, kb, 128, 64).transpose(0, 2, 1, 3).reshape(nt * 128, K // 2)
         sf = t[:, kb * 8192:].reshape(nt, kb, 32, 4, 4)  # codes of all K blocks, then scales [kb, r % 32, r / 32, s]
         sf = sf.transpose(0, 3, 2, 1, 4).reshape(nt * 128, kb * 4)      # [n, K / 32]
         assert not codes[N:].any() and np.all(sf[N:] == 127), "padding rows: zero codes, unit scales"
-        assert np.all(sf <= 127) and np.all(sf >= 122)
+        assert np.all(sf <= 127) and np.all(sf >= 122)   # shifts 0 .. 5
         return codes[:N], (127 - sf[:N]).astype(np.uint8)
     t = np.ascontiguousarray(tiles, dtype=np.uint8).reshape(nt, kb, 8448)
     words = t[:, :, :8192].copy().view(np.uint32).reshape(nt, kb, 4, 128, 4)     # [nt, kb, chunk, row, word]

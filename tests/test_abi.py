@@ -37,6 +37,10 @@ def test_size_queries(L):
     assert binding.packed_weight_sizes(768, 768, 128, "none") == (6 * 6 * 8448, 0, 768 * 6 * 4)
     assert binding.packed_weight_sizes(768, 768, 128, "M2") == (6 * 6 * 8448, 768 * 6, 768 * 4)
     assert binding.packed_weight_sizes(129, 256, 64, "M1") == (2 * 2 * 8448, 129 * 4, 129 * 4)
+    assert binding.packed_weight_sizes(129, 256, 64, "M1", "mx") == (2 * 2 * 8704, 129 * 4, 129 * 4)
+    assert binding.packed_weight_sizes(129, 256, 64, "M1", "mx_fp8") == (2 * 2 * 16896, 129 * 4, 129 * 4)
+    assert binding.packed_weight_sizes(129, 256, 64, "M2", "cast_e5m2") == (2 * 2 * 8448, 129 * 4, 129 * 4)
+    assert binding.packed_weight_sizes(8, 640, 320, "M2") == (5 * 8448, 8 * 2, 8 * 4)
     with pytest.raises(binding.ZqError) as e:
         binding.packed_weight_sizes(8, 100, 128, "M1")
     assert e.value.status == -2
@@ -83,7 +87,10 @@ def test_validation_before_launch(L):
     # packer
     assert L.zq_pack_weight_fp4(fake, 4, 256, 100, 1, 0, fake, fake, fake, null) == -2
     assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 3, 0, fake, fake, fake, null) == -4
-    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 1, 2, fake, fake, fake, null) == -4   # unknown layout
+    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 1, 4, fake, fake, fake, null) == -4   # unknown layout
+    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 0, 2, fake, fake, fake, null) == -4   # FP8 codes need M1 / M2
+    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 0, 3, fake, fake, fake, null) == -4   # so does the E5M2 target
+    assert L.zq_pack_weight_fp4(fake, 4, 640, 320, 0, 0, fake, fake, fake, null) == -2   # groups of 320: M1 / M2 only
     assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 0, 1, fake, fake, fake, null) == -4   # block scales need M1 / M2
     assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 1, 0, fake, null, fake, null) == -1
     assert L.zq_pack_weight_fp4(fake, 0, 256, 128, 1, 1, fake, fake, fake, null) == 0
@@ -109,7 +116,7 @@ def test_validation_before_launch(L):
     assert call(codes=C.c_void_p(0x1008)) == -3
     assert call(layout=1, codes=C.c_void_p(0x1010)) == -3   # the 4-bit tensor map wants 32-byte alignment
     assert call(layout=1, mode=0) == -4
-    assert call(layout=3) == -4
+    assert call(layout=4) == -4
     assert call(ws=null) == -5
     assert call(wsb=1024) == -5
     assert call(M=0) == 0
