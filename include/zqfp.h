@@ -216,6 +216,30 @@ int zq_w4a8_linear_host(const void* x_bf16_host, int64_t M, int64_t N, int64_t K
 int zq_device_status(void* workspace, int* detail, void* stream);
 
 /*
+ * Construction of the LoRC factors (Section 3, first paragraph; Appendix A: ranks 8 .. 56): the rank-r part of
+ * the singular value decomposition of the error matrix E = W - W^ between the original weight and its
+ * quantized form (FP4-E2M1 codes with the scales of zq_pack_weight_fp4), the singular values split evenly:
+ *   U^ = P_r diag(sigma_r)^(1/2) [N, r],  V^ = diag(sigma_r)^(1/2) Q_r^T [r, K],  E ~ U^ V^.
+ * The paper takes a full SVD on the host; here the leading subspace is found by randomized subspace
+ * iteration, which needs only products with E and its transpose: `omega` is the caller's draw of a Gaussian
+ * test matrix and `iters` the number of power iterations (2 is plenty when E has a spectral gap; the error
+ * of a plain quantized weight has a nearly flat spectrum, where more iterations buy little).  Any orthogonal
+ * re-mixing of the factors is an equally valid answer: compare U^ V^ or the spanned subspace, not elements.
+ *
+ * W      : FP32 [N, K] dense, the original weight
+ * shift / scale : as written by zq_pack_weight_fp4 for (N, K, group, mode) with ZQ_WEIGHTS_CAST or ZQ_WEIGHTS_MX
+ * omega  : FP32 [K, r + 8] dense, independent standard normal draws
+ * U_f16  : out, fp16 [N, r];  V_f16 : out, fp16 [r, K];  sigma2 : out, optional, FP32 [r], squares of the r
+ *          leading singular values of E
+ * workspace : zq_lorc_workspace_bytes(N, K, r) bytes, 256-byte aligned (holds E in FP32 and the iterates)
+ * r in {8, 16, ..., 64}; r + 8 <= min(N, K); 0 <= iters <= 8; K % group == 0.
+ */
+size_t zq_lorc_workspace_bytes(int64_t N, int64_t K, int r);
+int zq_lorc_factors(const float* W, int64_t N, int64_t K, int group, zq_scale_mode mode, const uint8_t* shift,
+                    const float* scale, int r, const float* omega, int iters, void* U_f16, void* V_f16,
+                    float* sigma2, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * (No operation of the paper: a check of the library's own failure reporting.)  Launches one CTA that waits,
  * with the wait routine the GEMM kernels use and a limit of `limit_us` microseconds (1 .. 1000000), on a
  * barrier that nothing ever completes.  The wait gives up, the kernel writes ZQ_ERR_DEVICE_TIMEOUT and the

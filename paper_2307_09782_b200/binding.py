@@ -26,7 +26,7 @@ EXPORTS = [
     "zq_status_string", "zq_quantize_act_fp8", "zq_packed_weight_sizes", "zq_pack_weight_fp4",
     "zq_w4a8_linear_workspace_bytes", "zq_workspace_init", "zq_w4a8_linear",
     "zq_w4a8_linear_host_workspace_bytes", "zq_w4a8_linear_host", "zq_device_status", "zq_launch_count",
-    "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc", "zq_w4a8_linear_noalloc_status", "zq_w4a8_linear_plan", "zq_selftest_bounded_wait",
+    "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc", "zq_w4a8_linear_noalloc_status", "zq_w4a8_linear_plan", "zq_selftest_bounded_wait", "zq_lorc_workspace_bytes", "zq_lorc_factors",
 ]
 PLAN_FIELDS = ("bm", "m_tiles", "n_tiles", "ctas", "stream", "persist", "splits", "kb_per_split", "base", "rem",
                "tail_pos0", "m_group", "partial_floats", "sms")
@@ -82,6 +82,10 @@ def lib() -> C.CDLL:
         L.zq_w4a8_linear_noalloc_status.argtypes = [C.POINTER(ci), vp]
         L.zq_selftest_bounded_wait.restype = ci
         L.zq_selftest_bounded_wait.argtypes = [vp, sz, C.c_uint32, vp]
+        L.zq_lorc_workspace_bytes.restype = sz
+        L.zq_lorc_workspace_bytes.argtypes = [i64, i64, ci]
+        L.zq_lorc_factors.restype = ci
+        L.zq_lorc_factors.argtypes = [vp, i64, i64, ci, ci, vp, vp, ci, vp, ci, vp, vp, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -232,6 +236,20 @@ def w4a8_linear_noalloc(w: PackedWeight, *, q, sx, t=None, U=None, y=None, out_d
                                         _ptr(scale), _ptr(U), _ptr(t), r, _ptr(y), ydt, ldy, _stream()),
            "zq_w4a8_linear_noalloc")
     return y
+
+
+def lorc_factors(W: torch.Tensor, w: "PackedWeight", r: int, omega: torch.Tensor, iters: int = 2):
+    """LoRC factors of W - dequant(w): returns (U^ fp16 [N,r], V^ fp16 [r,K], sigma2 float32 [r])."""
+    assert W.dtype == torch.float32 and W.is_contiguous() and omega.dtype == torch.float32 and omega.is_contiguous()
+    N, K = W.shape
+    assert omega.shape == (K, r + 8)
+    U = torch.empty((N, r), dtype=torch.float16, device=W.device)
+    V = torch.empty((r, K), dtype=torch.float16, device=W.device)
+    s2 = torch.empty((r,), dtype=torch.float32, device=W.device)
+    ws = torch.empty((max(int(lib().zq_lorc_workspace_bytes(N, K, r)), 1),), dtype=torch.uint8, device=W.device)
+    _check(lib().zq_lorc_factors(_ptr(W), N, K, w.group, _mode(w.mode), _ptr(w.shift), _ptr(w.scale), r, _ptr(omega),
+                                 iters, _ptr(U), _ptr(V), _ptr(s2), _ptr(ws), ws.numel(), _stream()), "zq_lorc_factors")
+    return U, V, s2
 
 
 def selftest_bounded_wait(workspace: torch.Tensor, limit_us: int = 1000):
