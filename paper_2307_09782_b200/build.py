@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libzqfp.so")
 SOURCES = ["api.cu", "actquant.cu", "packw.cu", "w4a8_gemm.cu", "w4a8_mx_gemm.cu", "noalloc.cu", "selftest.cu", "lorc.cu"]
-HEADERS = [os.path.join(CSRC, "zq_common.cuh"), os.path.join(CSRC, "w4a8_gemm_shared.cuh"), os.path.join(HERE, "..", "include", "zqfp.h")]
+HEADERS = [os.path.join(CSRC, "zq_common.cuh"), os.path.join(CSRC, "w4a8_gemm_shared.cuh"), os.path.join(CSRC, "act_cast.cuh"), os.path.join(HERE, "..", "include", "zqfp.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-fmad=true"]
 

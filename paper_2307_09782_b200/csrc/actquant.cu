@@ -7,6 +7,7 @@
 #include <cooperative_groups.h>
 #include <cuda_fp16.h>
 
+#include "act_cast.cuh"
 #include "zq_common.cuh"
 
 namespace zq {
@@ -17,16 +18,6 @@ constexpr int kVpt = 8;     // units a thread keeps in registers
 constexpr int kMaxThreads = 256;
 constexpr int kRChunk = 8;  // LoRC rows of V handled per pass over the registers
 
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
-
-// Two FP32 values -> two E4M3 bytes (round to nearest even, saturate to +-448); `lo` lands in bits 0..7.
-__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
-  uint16_t r;
-  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
@@ -36,40 +27,6 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
   return v;
-}
-
-__device__ __forceinline__ float absmax8(uint4 v, float a) {
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    a = fmaxf(a, fabsf(bf16_lo(w[i])));  // fmaxf drops a NaN operand
-    a = fmaxf(a, fabsf(bf16_hi(w[i])));
-  }
-  return a;
-}
-
-__device__ __forceinline__ uint2 cast8(uint4 v, float inv) {
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-  uint32_t p[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i)
-    p[i] = cvt_e4m3x2(__fmul_rn(bf16_lo(w[i]), inv), __fmul_rn(bf16_hi(w[i]), inv));
-  return make_uint2(p[0] | (p[1] << 16), p[2] | (p[3] << 16));
-}
-
-// acc + sum over 8 elements of x (bf16 pairs in xv) times V (fp16 pairs in vv)
-__device__ __forceinline__ float dot8(uint4 xv, uint4 vv, float acc) {
-  const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
-  const uint32_t vw[4] = {vv.x, vv.y, vv.z, vv.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    __half2 h;
-    *reinterpret_cast<uint32_t*>(&h) = vw[i];
-    const float2 vf = __half22float2(h);
-    acc = fmaf(bf16_lo(xw[i]), vf.x, acc);
-    acc = fmaf(bf16_hi(xw[i]), vf.y, acc);
-  }
-  return acc;
 }
 
 template <bool CACHED>

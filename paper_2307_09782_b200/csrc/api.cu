@@ -205,6 +205,36 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if (x_bf16 && layout_is_mx(layout) && M <= kFusedMaxTokens) {
+    // Few tokens (decode): the block-scaled kernel quantizes the activations itself, so the layer is one
+    // launch.  If that launch is refused, the two-kernel path below runs instead.
+    GemmArgs f{};
+    f.q = ws + w.off_q;  // where the kernel leaves the codes
+    f.M = M;
+    f.N = N;
+    f.K = K;
+    f.group = group;
+    f.mode = mode;
+    f.layout = layout;
+    f.codes = codes;
+    f.shift = shift;
+    f.scale = scale;
+    f.U = r > 0 ? U : nullptr;
+    f.r = r;
+    f.y = y;
+    f.ydt = ydt;
+    f.ldy = ldy;
+    f.status = reinterpret_cast<int*>(ws);
+    f.counters = reinterpret_cast<int*>(ws + kWsStatusBytes);
+    f.partials = reinterpret_cast<float*>(ws + w.off_partials);
+    f.partial_floats = w.partial_floats;
+    f.x = x_bf16;
+    f.ldx = ldx;
+    f.V = r > 0 ? V : nullptr;
+    f.fused_scratch = ws + kWsStatusBytes + kWsCounterBytes;
+    const int e = launch_w4a8_mx_gemm(f, st);
+    if (e != kFusedLaunchRefused) return e;
+  }
   if (x_bf16) {
     uint8_t* q_ws = ws + w.off_q;
     float* sx_ws = reinterpret_cast<float*>(ws + w.off_sx);

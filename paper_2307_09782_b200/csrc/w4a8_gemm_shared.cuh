@@ -19,7 +19,25 @@ constexpr int kBlockK = 128;  // K elements per pipeline step
 constexpr int kAStageCols = kBlockK / 4;  // TMEM columns of one widened 128 x 128 tile (4 bytes per column)
 
 // error detail codes written to status[1]
-enum { kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6, kErrHandover = 7 };
+enum {
+  kErrProducer = 1, kErrWiden = 2, kErrMma = 3, kErrEpilogue = 4, kErrPromote = 5, kErrAlign = 6, kErrHandover = 7,
+  kErrGridWait = 8  // the quantizer inside the block-scaled kernel gave up waiting for the other CTAs' shares
+};
+
+// Scratch of the quantizer that runs inside the block-scaled kernel, part of the workspace head.  Every launch
+// finds it zero and leaves it zero.
+struct FusedScratch {
+  unsigned int arrived_absmax;  // CTAs whose share of the tokens' absmax / LoRC sums is in
+  unsigned int arrived_codes;   // CTAs whose share of the E4M3 codes is written
+  unsigned int departed;        // CTAs that have finished; the last one clears the scratch
+  unsigned int pad;
+  // Atomics of many CTAs on one address are served one after the other (224 K blocks on one word took about
+  // 10 us), so K block kb adds into copy kb % kFusedSlots and the readers combine the copies.
+  unsigned int amax_bits[kFusedSlots][kFusedMaxTokens];   // per token: max |x| as FP32 bits (non-negative floats order like integers)
+  float t[kFusedSlots][kFusedMaxTokens * kFusedMaxRank];  // per token: t = V x, [m][r] token-major, accumulated with atomics
+  float t_sum[kFusedMaxTokens * kFusedMaxRank];           // the copies of t added up (by CTA 0, between the two meetings)
+};
+static_assert(sizeof(FusedScratch) <= kWsFusedBytes, "the scratch must fit its part of the workspace head");
 
 struct Params {
   int M, N, K;
@@ -55,6 +73,13 @@ struct Params {
   int* counters;
   float* partials;
   int cast_e5m2;  // the kernel that casts: E5M2 instead of E4M3 as the cast target
+  // the block-scaled kernel with the quantizer inside: raw activations, LoRC down-projection matrix, where the
+  // codes go (the buffer the token tensor map reads), and the scratch the CTAs meet in
+  const __nv_bfloat16* x;
+  int64_t ldx;
+  const __half* V;
+  uint8_t* q_out;
+  FusedScratch* fq;
 };
 
 constexpr int cmin(int a, int b) { return a < b ? a : b; }
@@ -150,7 +175,8 @@ __device__ __forceinline__ void finalize(const Params& p, const float* v, int m0
       if (m < p.M) {
         const float* tr = p.t + static_cast<int64_t>(m) * p.r;
         const __half* ur = p.U + static_cast<int64_t>(n) * p.r;
-        for (int j = 0; j < p.r; ++j) out[c] = fmaf(__ldg(tr + j), __half2float(__ldg(ur + j)), out[c]);
+        // t may have been accumulated by this very launch (quantizer inside the kernel): read it through L2
+        for (int j = 0; j < p.r; ++j) out[c] = fmaf(__ldcg(tr + j), __half2float(__ldg(ur + j)), out[c]);
       }
     }
   }
@@ -251,6 +277,11 @@ inline Params make_params(const GemmArgs& a, const GemmPlan& plan) {
   p.status = a.status;
   p.counters = a.counters;
   p.partials = a.partials;
+  p.x = static_cast<const __nv_bfloat16*>(a.x);
+  p.ldx = a.ldx;
+  p.V = static_cast<const __half*>(a.V);
+  p.q_out = const_cast<uint8_t*>(a.q);
+  p.fq = static_cast<FusedScratch*>(a.fused_scratch);
   return p;
 }
 

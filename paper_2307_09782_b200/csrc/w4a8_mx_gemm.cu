@@ -34,6 +34,7 @@
 //
 // Warp roles: 0..3 epilogue (one TMEM lane quarter each), 4 producer (one lane issues all copies of a
 // stage onto one barrier), 5 TMEM allocation and MMA issue.
+#include "act_cast.cuh"
 #include "w4a8_gemm_shared.cuh"
 
 namespace zq {
@@ -159,7 +160,34 @@ struct StageWalker {
   }
 };
 
-template <int BM, bool W8>
+// Thread 0 of a CTA: count this CTA in (if it had a share of the work) and wait, bounded, until `expected`
+// CTAs have.  The launch is cooperative, so all of them are running.
+__device__ __forceinline__ bool grid_meet(unsigned int* counter, unsigned int expected, bool counts,
+                                          volatile int* abort_flag) {
+  __threadfence();
+  if (counts) atomicAdd(counter, 1u);
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+    if (*reinterpret_cast<volatile unsigned int*>(counter) >= expected) {
+      __threadfence();
+      return true;
+    }
+    if (*abort_flag) return false;
+    if ((spin & 63u) == 63u && global_timer_ns() - t0 > kWaitLimitNs) return false;
+  }
+  return false;
+}
+
+// FUSEQ: the kernel quantizes the activations itself (one tile of at most 16 tokens), so that the layer is one
+// launch.  While the producer's first weight copies are on their way, the epilogue warps (idle until the first
+// accumulator is due) (1) add their CTA's share of every token's absmax and of the LoRC down-projection
+// t = V x into a scratch in which all CTAs meet, (2) once all shares are in, cast their share of x to E4M3
+// into the workspace's q buffer, and (3) once all codes are written, release the producer, which loads the
+// token tiles from q exactly as it would after a separate quantizer kernel.  The main loop is untouched.
+// (Casting the tokens straight into the pipeline stages, by extra warps or by the producer warp, was tried in
+// several forms first: each ran the main loop at 0.7 us or more per stage against the 0.39 us of the copies
+// alone.)  The two meetings cost about 3 us during which only the ring's first stages stream.
+template <int BM, bool W8, bool FUSEQ>
 __global__ void __launch_bounds__(MxCfg<BM, W8>::kThreads, MxCfg<BM, W8>::kMinBlocks)
 w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
                     const Params p) {
@@ -259,7 +287,12 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
         ++issued;
       }
       __syncwarp();
-      pdl_wait();
+      if (FUSEQ) {
+        named_bar_sync(3, C::kEpiThreads + 32);  // every CTA's codes are in q
+        asm volatile("fence.proxy.async.global;" ::: "memory");  // written by ordinary stores, read by the copy engine
+      } else {
+        pdl_wait();
+      }
       for (int i = 0; i < issued; ++i) {
         w_tok.next(p, w_tile, w_kb);
         issue_tokens(i, w_tile, w_kb);
@@ -287,6 +320,8 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
         while (!mbar_try_wait(&full[i % C::NS], (i / C::NS) & 1) && ++spin < kSpinLimit) {
         }
       }
+    } else if (FUSEQ) {
+      named_bar_sync(3, C::kEpiThreads + 32);
     }
   } else if (warp == C::kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer
@@ -360,7 +395,118 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
     constexpr int EC = BM <= 32 ? 4 : (BM <= 128 ? 8 : 16);  // columns per step
     bool failed = !ok_start;
     int m0_loaded = -1;
-    pdl_wait();  // sx, t, the hand-over flags and y may still be in use by the kernel ahead in the stream
+    pdl_wait();  // x, sx, t, the hand-over flags and y may still be in use by the kernel ahead in the stream
+    if (FUSEQ) {
+      // Section 3 / Appendix A, token-wise: a_m = max_k |x[m,k]|, q = RNE_E4M3(fl32(x * fl32(448 / a_m))), and
+      // t = V x with the raw x.  This CTA's share: K blocks blockIdx.x, + gridDim.x, ...; a thread takes 16
+      // consecutive elements of token row threadIdx.x / 8 (eight neighbouring lanes share a row).
+      FusedScratch* fq = p.fq;
+      const int chunk = threadIdx.x & 7, m = threadIdx.x >> 3;
+      const bool m_ok = m < p.M;
+      const unsigned int sharers = static_cast<unsigned int>(min(static_cast<int>(gridDim.x), p.kblocks));
+      const bool has_share = static_cast<int>(blockIdx.x) < p.kblocks;
+      // the first two K blocks of the share stay in registers between the two passes
+      constexpr int kKeep = 2;
+      uint4 xk[kKeep][2];
+#pragma unroll
+      for (int i = 0; i < kKeep; ++i) {
+        const int kb = blockIdx.x + i * gridDim.x;
+        xk[i][0] = xk[i][1] = make_uint4(0, 0, 0, 0);
+        if (ok_start && m_ok && kb < p.kblocks) {
+          const uint4* xp = reinterpret_cast<const uint4*>(p.x + static_cast<int64_t>(m) * p.ldx + kb * kBlockK) + 2 * chunk;
+          xk[i][0] = __ldg(xp);
+          xk[i][1] = __ldg(xp + 1);
+        }
+      }
+      if (ok_start) {
+        int i = 0;
+        for (int kb = blockIdx.x; kb < p.kblocks; kb += gridDim.x, ++i) {
+          uint4 x0 = make_uint4(0, 0, 0, 0), x1 = x0;
+          if (i == 0) {
+            x0 = xk[0][0];
+            x1 = xk[0][1];
+          } else if (i == 1) {
+            x0 = xk[1][0];
+            x1 = xk[1][1];
+          } else if (m_ok) {
+            const uint4* xp = reinterpret_cast<const uint4*>(p.x + static_cast<int64_t>(m) * p.ldx + kb * kBlockK) + 2 * chunk;
+            x0 = __ldg(xp);
+            x1 = __ldg(xp + 1);
+          }
+          const int slot = kb % kFusedSlots;
+          float a = absmax8(x1, absmax8(x0, 0.0f));
+          a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, 1));
+          a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, 2));
+          a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, 4));
+          if (m_ok && chunk == 0 && a != 0.0f) atomicMax(&fq->amax_bits[slot][m], __float_as_uint(a));
+          for (int j0 = 0; j0 < p.r; j0 += 8) {  // p.r is a multiple of 8 (0 without LoRC)
+            float acc[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              const uint4* vp = reinterpret_cast<const uint4*>(p.V + static_cast<int64_t>(j0 + j) * p.K + kb * kBlockK) + 2 * chunk;
+              acc[j] = dot8(x1, __ldg(vp + 1), dot8(x0, __ldg(vp), 0.0f));
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              acc[j] += __shfl_xor_sync(0xFFFFFFFFu, acc[j], 1);
+              acc[j] += __shfl_xor_sync(0xFFFFFFFFu, acc[j], 2);
+              acc[j] += __shfl_xor_sync(0xFFFFFFFFu, acc[j], 4);
+            }
+            if (m_ok && chunk == 0) {
+#pragma unroll
+              for (int j = 0; j < 8; ++j) atomicAdd(&fq->t[slot][m * p.r + j0 + j], acc[j]);
+            }
+          }
+        }
+      }
+      __threadfence();
+      named_bar_sync(2, C::kEpiThreads);
+      if (threadIdx.x == 0 && !grid_meet(&fq->arrived_absmax, sharers, has_share && ok_start, s_abort))
+        raise_error(p, s_abort, kErrGridWait);
+      named_bar_sync(2, C::kEpiThreads);
+      if (ok_start && *s_abort == 0) {
+        if (blockIdx.x == 0)  // one CTA adds the copies of t up for everybody's epilogue
+          for (int e = threadIdx.x; e < p.M * p.r; e += C::kEpiThreads) {
+            float v = 0.0f;
+#pragma unroll
+            for (int sl = 0; sl < kFusedSlots; ++sl) v += __ldcg(&fq->t[sl][e]);
+            fq->t_sum[e] = v;
+          }
+        float a = 0.0f;
+        if (m_ok) {
+#pragma unroll
+          for (int sl = 0; sl < kFusedSlots; ++sl) a = fmaxf(a, __uint_as_float(__ldcg(&fq->amax_bits[sl][m])));
+        }
+        const float inv = a != 0.0f ? __fdiv_rn(448.0f, a) : 1.0f;
+        int i = 0;
+        for (int kb = blockIdx.x; kb < p.kblocks; kb += gridDim.x, ++i) {
+          if (m_ok) {
+            uint4 x0, x1;
+            if (i == 0) {
+              x0 = xk[0][0];
+              x1 = xk[0][1];
+            } else if (i == 1) {
+              x0 = xk[1][0];
+              x1 = xk[1][1];
+            } else {
+              const uint4* xp = reinterpret_cast<const uint4*>(p.x + static_cast<int64_t>(m) * p.ldx + kb * kBlockK) + 2 * chunk;
+              x0 = __ldg(xp);
+              x1 = __ldg(xp + 1);
+            }
+            const uint2 lo = cast8(x0, inv), hi = cast8(x1, inv);
+            *reinterpret_cast<uint4*>(p.q_out + static_cast<int64_t>(m) * p.K + kb * kBlockK + 16 * chunk) =
+                make_uint4(lo.x, lo.y, hi.x, hi.y);
+          }
+        }
+        asm volatile("fence.proxy.async.global;" ::: "memory");  // the copy engine will read these stores
+      }
+      __threadfence();
+      named_bar_sync(2, C::kEpiThreads);
+      if (threadIdx.x == 0 && !grid_meet(&fq->arrived_codes, sharers, has_share && ok_start, s_abort))
+        raise_error(p, s_abort, kErrGridWait);
+      named_bar_sync(3, C::kEpiThreads + 32);  // releases the producer's token loads
+      if (*s_abort) failed = true;
+    }
 
     // Every thread walks every segment and executes the same named-barrier sequence whether or not it
     // has failed, so a bounded wait that ran out can never leave others stuck at a hardware barrier.
@@ -374,11 +520,24 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       if (m0 != m0_loaded) {
         // token scales and (rank 8) LoRC rows of this tile's tokens
         named_bar_sync(2, C::kEpiThreads);  // the previous tile's reads are done
-        for (int c = threadIdx.x; c < BM; c += C::kEpiThreads) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
-        if (p.r == 8)
-          for (int c = threadIdx.x; c < BM * 8; c += C::kEpiThreads)  // transposed: [j][BM]
-            s_t[(c & 7) * BM + (c >> 3)] =
-                (m0 + (c >> 3) < p.M) ? __ldg(p.t + static_cast<int64_t>(m0) * 8 + c) : 0.0f;
+        if (FUSEQ) {
+          // token scales from the absmax the CTAs agreed on: sx = fl32(a / 448), 1 for an all-zero token
+          for (int c = threadIdx.x; c < BM; c += C::kEpiThreads) {
+            float a = 0.0f;
+            if (c < p.M)
+              for (int sl = 0; sl < kFusedSlots; ++sl) a = fmaxf(a, __uint_as_float(__ldcg(&p.fq->amax_bits[sl][c])));
+            s_sx[c] = c < p.M ? (a != 0.0f ? __fdiv_rn(a, 448.0f) : 1.0f) : 0.0f;
+          }
+          if (p.r == 8)
+            for (int c = threadIdx.x; c < BM * 8; c += C::kEpiThreads)
+              s_t[(c & 7) * BM + (c >> 3)] = ((c >> 3) < p.M) ? __ldcg(&p.fq->t_sum[c]) : 0.0f;
+        } else {
+          for (int c = threadIdx.x; c < BM; c += C::kEpiThreads) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
+          if (p.r == 8)
+            for (int c = threadIdx.x; c < BM * 8; c += C::kEpiThreads)  // transposed: [j][BM]
+              s_t[(c & 7) * BM + (c >> 3)] =
+                  (m0 + (c >> 3) < p.M) ? __ldg(p.t + static_cast<int64_t>(m0) * 8 + c) : 0.0f;
+        }
         named_bar_sync(2, C::kEpiThreads);
         m0_loaded = m0;
       }
@@ -531,6 +690,24 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, C::kTmemCols);
   }
+  if (FUSEQ) {
+    // The CTA that leaves last clears the scratch for the next launch (every other CTA has read what it
+    // needs before it counts itself out).  After a wait that ran out the scratch is left as it is: the
+    // workspace has to be re-initialized anyway.
+    if (threadIdx.x == 0)
+      *s_last = (*s_abort == 0 && atomicAdd(&p.fq->departed, 1u) == gridDim.x - 1) ? 1 : 0;
+    __syncthreads();
+    if (*s_last) {
+      for (int i = threadIdx.x; i < kFusedSlots * kFusedMaxTokens; i += C::kThreads) (&p.fq->amax_bits[0][0])[i] = 0u;
+      for (int sl = 0; sl < kFusedSlots; ++sl)
+        for (int i = threadIdx.x; i < kFusedMaxTokens * p.r; i += C::kThreads) p.fq->t[sl][i] = 0.0f;
+      if (threadIdx.x == 0) {
+        p.fq->arrived_absmax = 0u;
+        p.fq->arrived_codes = 0u;
+        p.fq->departed = 0u;
+      }
+    }
+  }
 }
 
 // ---- host ------------------------------------------------------------------------------------------
@@ -565,7 +742,7 @@ bool make_token_map(CUtensorMap* m, const void* base, uint64_t K, uint64_t M, ui
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BM, bool W8>
+template <int BM, bool W8, bool FUSEQ>
 int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStream_t st) {
   using C = MxCfg<BM, W8>;
   CUtensorMap tm_w, tm_q;
@@ -575,40 +752,45 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(w4a8_mx_gemm_kernel<BM, W8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    attr_err = cudaFuncSetAttribute(w4a8_mx_gemm_kernel<BM, W8, FUSEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     C::kSmemBytes);
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
   dim3 grid(static_cast<unsigned>(plan.ctas));
   const bool shared_f32 =
       a.ydt == ZQ_OUT_F32 && (p.atomic_y || (plan.persist && plan.tail_pos0 < p.tiles));
-  if (shared_f32) {
+  if (shared_f32 || FUSEQ) {
     // Output tiles are shared by CTAs that accumulate into FP32 y.  In a cooperative launch (all CTAs
     // resident, which the plan's grid is sized for) they hand over through per-tile flags: one stores,
     // the others wait for it and add.  If the device cannot hold the grid at once: unit ranges -> clear
     // y with a memset and let every CTA add; persistent launch -> partial sums through the workspace.
+    // (The kernel with the quantizer inside has its CTAs meet in a scratch as well, so its launch is always
+    // cooperative; if that is refused nothing has run and the caller takes the two-kernel path.)
     Params pc = p;
-    pc.atomic_y = 1;
-    pc.handover = 1;
+    if (shared_f32) {
+      pc.atomic_y = 1;
+      pc.handover = 1;
+    }
     void* args[3] = {&tm_w, &tm_q, &pc};
     // chained to the kernel ahead (see pdl_wait); if the two launch attributes are refused together, cooperative alone
-    if (launch_chained(w4a8_mx_gemm_kernel<BM, W8>, grid, dim3(C::kThreads), C::kSmemBytes, st, true, tm_w, tm_q, pc) ==
+    if (launch_chained(w4a8_mx_gemm_kernel<BM, W8, FUSEQ>, grid, dim3(C::kThreads), C::kSmemBytes, st, true, tm_w, tm_q, pc) ==
         cudaSuccess) {
       count_launch();
       return ZQ_OK;
     }
     (void)cudaGetLastError();
-    if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM, W8>), grid, dim3(C::kThreads),
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM, W8, FUSEQ>), grid, dim3(C::kThreads),
                                     args, C::kSmemBytes, st) == cudaSuccess) {
       count_launch();
       return ZQ_OK;
     }
     (void)cudaGetLastError();  // not launched; fall back
+    if (FUSEQ) return kFusedLaunchRefused;
     if (p.atomic_y && cudaMemset2DAsync(a.y, static_cast<size_t>(a.ldy) * 4, 0, static_cast<size_t>(a.N) * 4,
                                         static_cast<size_t>(a.M), st) != cudaSuccess)
       return ZQ_ERR_CUDA;
   }
-  const cudaError_t err = launch_chained(w4a8_mx_gemm_kernel<BM, W8>, grid, dim3(C::kThreads), C::kSmemBytes, st, false,
+  const cudaError_t err = launch_chained(w4a8_mx_gemm_kernel<BM, W8, FUSEQ>, grid, dim3(C::kThreads), C::kSmemBytes, st, false,
                                          tm_w, tm_q, p);
   count_launch();
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
@@ -620,10 +802,18 @@ int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.mode == ZQ_SCALE_NONE) return ZQ_ERR_MODE;
   const GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode, ZQ_WEIGHTS_MX);
   if (plan.partial_floats > a.partial_floats) return ZQ_ERR_WORKSPACE;
-  const Params p = make_params(a, plan);
+  Params p = make_params(a, plan);
   const bool w8 = a.layout == ZQ_WEIGHTS_MX_FP8;
+  if (a.x) {
+    // the kernel quantizes the activations itself: one tile of at most kFusedMaxTokens tokens
+    if (a.M > kFusedMaxTokens || plan.bm != 16 || plan.m_tiles != 1 || a.r > kFusedMaxRank || !a.fused_scratch || !a.q)
+      return ZQ_ERR_SHAPE;
+    p.sx = nullptr;
+    p.t = p.fq->t_sum;  // token-major [M, r], as the separate quantizer writes it
+    return w8 ? launch_mx_cfg<16, true, true>(a, plan, p, st) : launch_mx_cfg<16, false, true>(a, plan, p, st);
+  }
 #define ZQ_MX_CASE(BM_) \
-  case BM_: return w8 ? launch_mx_cfg<BM_, true>(a, plan, p, st) : launch_mx_cfg<BM_, false>(a, plan, p, st)
+  case BM_: return w8 ? launch_mx_cfg<BM_, true, false>(a, plan, p, st) : launch_mx_cfg<BM_, false, false>(a, plan, p, st)
   switch (plan.bm) {
     ZQ_MX_CASE(16);
     ZQ_MX_CASE(32);

@@ -19,7 +19,12 @@ constexpr size_t kWsStatusBytes = 256;
 // status[0] error code, status[1] detail
 constexpr int kWsMaxTiles = 16384;  // counters: one int per output tile
 constexpr size_t kWsCounterBytes = size_t(kWsMaxTiles) * 4;
-constexpr size_t kWsHeadBytes = kWsStatusBytes + kWsCounterBytes;
+// ... then the scratch in which the CTAs of the block-scaled kernel meet when it quantizes the activations itself
+constexpr int kFusedMaxTokens = 16;
+constexpr int kFusedMaxRank = 64;
+constexpr int kFusedSlots = 8;           // copies of the absmax / LoRC sums the atomics are spread over
+constexpr size_t kWsFusedBytes = 37632;  // 16 bytes of counters + 8 x (16 absmax words + 16 x 64 LoRC sums) + the sums' total, rounded up
+constexpr size_t kWsHeadBytes = kWsStatusBytes + kWsCounterBytes + kWsFusedBytes;
 
 // ---- packed weight format (written by the packer, streamed by the GEMM) --------------------------
 // The weight is stored as tiles of 128 output rows x 128 input features, tile (nt, kb) at byte offset
@@ -88,7 +93,16 @@ struct GemmArgs {
   int* counters;         // split-K tile counters
   float* partials;       // split-K partial sums
   size_t partial_floats; // capacity of `partials`
+  // set only when the block-scaled kernel is to quantize the activations itself (at most kFusedMaxTokens tokens;
+  // q then names the buffer the kernel writes the codes to, sx and t are unused):
+  const void* x;         // bf16 [M, ldx]
+  int64_t ldx;
+  const void* V;         // fp16 [r, K] or NULL
+  void* fused_scratch;   // kWsFusedBytes of the workspace head
 };
+// Returned by launch_w4a8_mx_gemm when that launch was refused (the grid cannot be resident at once): nothing
+// ran; the caller quantizes with the separate kernel and launches the plain GEMM.
+constexpr int kFusedLaunchRefused = 1;
 // Tile shape chosen for a problem (shared by the workspace-size query and the launcher).
 struct GemmPlan {
   int bm;      // tokens per tile (the MMA's N extent)
