@@ -4,7 +4,8 @@ A step is SWEEPS passes of the whole hot path (token-wise FP8 quantization with 
 then the W4A8 GEMM with its scale + LoRC epilogue) over the OPT-30B-shaped sweep: the two MLP layers
 (7168 -> 28672 and 28672 -> 7168), each at M in {8192, 2048, 512, 128, 32, 8, 1} tokens, constraint M2,
 group 128, LoRC rank 8.  Weights are packed once before the timed region.  A layer call is
-zq_w4a8_linear on raw bf16 activations (the library runs its quantizer and then the GEMM); the calls at the
+zq_w4a8_linear on raw bf16 activations (the library quantizes: inside the GEMM kernel up to 16 tokens, with its
+quantizer kernel chained to the GEMM beyond); the calls at the
 largest token count are issued as quantizer call + GEMM call so that CUDA events can bracket the dominant
 GEMM kernel inside the timed region.  The sweep runs from many tokens to few: a decode-size call right
 after the 8192-token GEMM would be timed while that kernel's 235 MB of output is still being written back
@@ -480,7 +481,8 @@ def run_ours(args):
     roofline_decode = None
     if dec:
         roofline_decode = {"bound": "hbm", "kernel": f"{kfam}<16>",
-                           "what": "the GEMM alone on pre-quantized activations at M <= 16: algorithmic bytes / gemm_us",
+                           "what": "the GEMM alone on pre-quantized activations at M <= 16: algorithmic bytes / gemm_us; "
+                                   "frac_whole_layer: one zq_w4a8_linear call on raw x (quantizer inside the kernel)",
                            "achieved": round(statistics.mean(s["gemm_frac_hbm"] for s in dec) * peaks["hbm_gbs"], 1),
                            "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": round(statistics.mean(s["gemm_frac_hbm"] for s in dec), 4),
@@ -496,6 +498,7 @@ def run_ours(args):
 
     # ---- further rows the configurations ask for (not part of the timed step)
     extra_rows = []
+    lorc_ms = None
     if not args.case and not args.no_extra:
         def extra(wl_, shape, M, md, lay, r_):
             ly = B.make_layer(wl_, shape, M, md, lay, rank_lorc=r_)
@@ -510,6 +513,22 @@ def run_ours(args):
                 extra(wl, shape, M, mode, args.layout, 0)
             for M in (1, 8, Mmax):  # the other kernel family (cast: kind::f8f6f4, E4M3 x E4M3, the kernel casts)
                 extra(wl, shape, M, mode, other, RANK)
+        for shape in shapes:  # FP8-E4M3 weights (W8A8 FP - FP) through the block-scaled kernel
+            for M in (8, Mmax):
+                extra(wl, shape, M, mode, "mx_fp8", RANK)
+        extra(wl, shapes[0], Mmax, mode, "cast_e5m2", RANK)  # E5M2 as the cast target
+        # LoRC factor construction on the device (offline step), rank 8, two power iterations
+        shape = shapes[0]
+        Wd = torch.from_numpy(B.w_cache[(wl.seed, shape.N, shape.K, wl.sigma_w)]).to(dev)
+        pw = binding.pack_weight_fp4(Wd, GROUP, mode, "mx")
+        om = torch.randn((shape.K, RANK + 8), dtype=torch.float32, device=dev)
+        binding.lorc_factors(Wd, pw, RANK, om, iters=2)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        binding.lorc_factors(Wd, pw, RANK, om, iters=2)
+        torch.cuda.synchronize()
+        lorc_ms = (time.perf_counter() - t0) * 1e3
+        del Wd, pw, om
         wl7 = synth.WORKLOADS["llama7b"]  # unconstrained scales (per-group FP32 promotion) at 2048 tokens
         for shape in wl7.shapes:
             for md, lay in EXTRA_LLAMA7B:
@@ -580,7 +599,7 @@ def run_ours(args):
                           "around n = 6-20 back-to-back launches (rotated weight copies), divided by n, median of 3 "
                           "batches; layer_us = one zq_w4a8_linear call on raw x; quant_us / gemm_us = the quantizer "
                           "kernel alone and the GEMM alone on pre-quantized activations",
-            "sweep": table, "extra_rows": extra_rows}
+            "sweep": table, "extra_rows": extra_rows, "lorc_factors_ms": lorc_ms}
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(wl)
     print(json.dumps(line))

@@ -28,9 +28,8 @@ bool valid_group(int g, int mode) { return g == 64 || g == 128 || g == 256 || (g
 // the tensor core's block scales are powers of two, and E5M2 as the cast target is about the shifts: only
 // the constrained modes can use those layouts
 bool valid_layout(int layout, int mode) {
-  return layout == ZQ_WEIGHTS_CAST ||
-         ((layout == ZQ_WEIGHTS_MX || layout == ZQ_WEIGHTS_MX_FP8 || layout == ZQ_WEIGHTS_CAST_E5M2) &&
-          mode != ZQ_SCALE_NONE);
+  return layout == ZQ_WEIGHTS_CAST || layout == ZQ_WEIGHTS_MX ||
+         ((layout == ZQ_WEIGHTS_MX_FP8 || layout == ZQ_WEIGHTS_CAST_E5M2) && mode != ZQ_SCALE_NONE);
 }
 inline bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 // the sizes every linear entry point and size query accepts (the group size is checked where it is known)
@@ -49,9 +48,9 @@ size_t max_partial_floats(int64_t M, int64_t N, int64_t K) {
   if (M <= 0 || N <= 0) return 0;
   auto probe = [&](int64_t m) {
     if (m <= 0 || m > M) return;
-    for (int variant = 0; variant < 3; ++variant) {
-      const GemmPlan pl = plan_gemm(m, N, K, variant == 0 ? ZQ_SCALE_NONE : ZQ_SCALE_M1,
-                                    variant == 2 ? ZQ_WEIGHTS_MX : ZQ_WEIGHTS_CAST);
+    for (int variant = 0; variant < 4; ++variant) {  // (none, cast), (M1, cast), (M1, block-scaled), (none, block-scaled)
+      const GemmPlan pl = plan_gemm(m, N, K, (variant == 0 || variant == 3) ? ZQ_SCALE_NONE : ZQ_SCALE_M1,
+                                    variant >= 2 ? ZQ_WEIGHTS_MX : ZQ_WEIGHTS_CAST);
       if (pl.partial_floats > best) best = pl.partial_floats;
     }
   };
@@ -205,7 +204,7 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  if (x_bf16 && layout_is_mx(layout) && M <= kFusedMaxTokens) {
+  if (x_bf16 && layout_is_mx(layout) && mode != ZQ_SCALE_NONE && M <= kFusedMaxTokens) {
     // Few tokens (decode): the block-scaled kernel quantizes the activations itself, so the layer is one
     // launch.  If that launch is refused, the two-kernel path below runs instead.
     GemmArgs f{};

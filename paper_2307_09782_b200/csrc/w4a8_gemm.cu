@@ -625,20 +625,22 @@ int sm_count() {
 GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   GemmPlan pl{};
   const bool mx = layout_is_mx(layout);
-  const int bm_max = (mode == ZQ_SCALE_NONE) ? 64 : 256;
+  // mode none keeps a tile's running sums in registers: 64 tokens in the kernel that casts, 128 in the block-scaled one
+  const int bm_max = (mode == ZQ_SCALE_NONE) ? (mx ? 128 : 64) : 256;
   int bm = 16;
   while (bm < bm_max && bm < M) bm *= 2;
   // the block-scaled kernel also has a 192-token tile, the widest that leaves room for two accumulators:
   // it serves every token count beyond one 256-token tile
-  if (mx && (M > 256 || (M > 128 && M <= 192))) bm = 192;
+  const bool wide = mx && mode != ZQ_SCALE_NONE;  // token tiles beyond 128
+  if (wide && (M > 256 || (M > 128 && M <= 192))) bm = 192;
   // 224 tokens still leave room for two accumulators and move fewer shared-memory bytes per flop (the
   // bound of this kernel); taken when the padding of the last tile does not eat the gain
-  if (mx && M > 256 && ((M + 223) / 224) * 224 * 20 < ((M + 191) / 192) * 192 * 21 &&
+  if (wide && M > 256 && ((M + 223) / 224) * 224 * 20 < ((M + 191) / 192) * 192 * 21 &&
       ((M + 223) / 224) * ((N + kTileN - 1) / kTileN) >= 4 * static_cast<int64_t>(sm_count()))
     bm = 224;
   // long rows: the epilogue is a small share of a tile, and a 256-token tile (one accumulator, no overlap)
   // moves fewer shared-memory bytes per flop
-  if (mx && M > 256 && K >= 16384 &&
+  if (wide && M > 256 && K >= 16384 &&
       ((M + 255) / 256) * ((N + kTileN - 1) / kTileN) >= 4 * static_cast<int64_t>(sm_count()))
     bm = 256;
   pl.bm = bm;
@@ -681,7 +683,7 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
     pl.partial_floats = tail_tiles > 0 ? 2 * static_cast<size_t>(g) * bm * kTileN : 0;
     return pl;
   }
-  if (mode != ZQ_SCALE_NONE && (mx || (bm == 16 && pl.m_tiles == 1)) && tiles <= kWsMaxTiles && units >= 8 &&
+  if ((mx || (mode != ZQ_SCALE_NONE && bm == 16 && pl.m_tiles == 1)) && tiles <= kWsMaxTiles && units >= 8 &&
       units < (int64_t(1) << 30)) {
     // At most 16 tokens (decode): the weight streams exactly once and the per-tile epilogue is tiny, so deal
     // the (tile, K block) units out evenly to one resident wave of CTAs, at least 4 units each.  (In the casting

@@ -46,8 +46,13 @@ constexpr int kSfbCols = 16;  // token-side block scales (all one): room for 256
 
 // W8: the weight codes are FP8-E4M3 bytes (layout ZQ_WEIGHTS_MX_FP8) instead of packed E2M1 nibbles: 16 KB per
 // tile in HBM, copied as they are (they fill the same 16 KB of shared memory as the padded FP4 form).
-template <int BM, bool W8>
+// NONE (unconstrained FP32 group scales, Section 3: what M1 / M2 remove): the block scales are all 2^0, the two
+// accumulator buffers hold one weight group's partial sum each, the epilogue warps multiply it by the group's
+// FP32 scale and add it up in registers while the MMAs of the next group run, and the finished tile goes back to a
+// third tensor-memory region, from which the usual epilogue takes it.
+template <int BM, bool W8, bool NONE = false>
 struct MxCfg {
+  static_assert(!NONE || (BM <= 128 && !W8), "mode none: the running sums are BM registers per thread");
   // One CTA per SM: launches whose CTAs share output tiles are cooperative, and a cooperative launch of a
   // kernel that allocates tensor memory is given one CTA per SM (the occupancy query answers 1 whatever the
   // registers and shared memory; with two CTAs per SM planned, grids beyond the SM count were refused).
@@ -71,7 +76,8 @@ struct MxCfg {
   static constexpr int NS = cmin(12, kBudget / (kABytes + kSfBytes + kTokBytes));
   static constexpr int NB = BM <= 224 ? 2 : 1;  // accumulator buffers
   static constexpr int kDColsPad = BM < 32 ? 32 : BM;
-  static constexpr int kSfaCol0 = NB * kDColsPad;
+  static constexpr int kResultCol0 = NB * kDColsPad;  // NONE: the finished tile
+  static constexpr int kSfaCol0 = (NONE ? NB + 1 : NB) * kDColsPad;
   static constexpr int kSfbCol0 = kSfaCol0 + 4 * kKps * NS;
   static constexpr int kColsUsed = kSfbCol0 + kSfbCols;
   static constexpr int kTmemCols = kColsUsed <= 128 ? 128 : (kColsUsed <= 256 ? 256 : 512);
@@ -187,11 +193,12 @@ __device__ __forceinline__ bool grid_meet(unsigned int* counter, unsigned int ex
 // (Casting the tokens straight into the pipeline stages, by extra warps or by the producer warp, was tried in
 // several forms first: each ran the main loop at 0.7 us or more per stage against the 0.39 us of the copies
 // alone.)  The two meetings cost about 3 us during which only the ring's first stages stream.
-template <int BM, bool W8, bool FUSEQ>
-__global__ void __launch_bounds__(MxCfg<BM, W8>::kThreads, MxCfg<BM, W8>::kMinBlocks)
+template <int BM, bool W8, bool FUSEQ, bool NONE>
+__global__ void __launch_bounds__(MxCfg<BM, W8, NONE>::kThreads, MxCfg<BM, W8, NONE>::kMinBlocks)
 w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
                     const Params p) {
-  using C = MxCfg<BM, W8>;
+  using C = MxCfg<BM, W8, NONE>;
+  static_assert(!NONE || C::NB == 2, "mode none alternates two group accumulators");
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* s_a = smem + C::offA;
   uint8_t* s_tok = smem + C::offTok;
@@ -334,40 +341,61 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       int s = 0, seg = 0;
       uint32_t ph = 0;
       bool failed = false;
+      int gcount = 0;  // NONE: weight groups started so far (group g accumulates in buffer g % 2)
+      const int mpg = NONE ? p.group / 32 : 1;  // NONE: MMAs (32 elements of K each) per weight group
       while (!failed && sg.next(p, pos, tile, kb0, nkb)) {
         const int buf = seg % C::NB;
         // the epilogue of the segment that used this accumulator buffer last must have read it
-        if (seg >= C::NB && !mbar_wait(&acc_empty[buf], ((seg / C::NB) - 1) & 1, s_abort)) {
+        if (!NONE && seg >= C::NB && !mbar_wait(&acc_empty[buf], ((seg / C::NB) - 1) & 1, s_abort)) {
           failed = true;
           break;
         }
-        const uint32_t d_tmem = tmem_base + buf * C::kDColsPad;
-        for (int i = 0; i < nkb; i += C::kKps) {
+        uint32_t d_tmem = tmem_base + buf * C::kDColsPad;
+        int gid_prev = -1, gbuf = 0;
+        for (int i = 0; i < nkb && !failed; i += C::kKps) {
           const int nk = min(C::kKps, nkb - i);  // K blocks of this stage that belong to the segment
           if (!mbar_wait(&full[s], ph, s_abort)) {
             failed = true;
             break;
           }
           tc_fence_after_sync();
-          if (issuer) {
 #pragma unroll
-            for (int j = 0; j < C::kKps; ++j) {
-              if (j < nk) {
-                const uint32_t sfa = tmem_sfa + 4 * (s * C::kKps + j);
-                const uint64_t adesc = adesc0 + static_cast<uint64_t>((s * C::kABytes + j * C::kABytes1) >> 4);
-                const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((s * C::kTokBytes + j * C::kTokBytes1) >> 4);
+          for (int j = 0; j < C::kKps; ++j) {
+            if (j < nk && !failed) {
+              const uint32_t sfa = tmem_sfa + 4 * (s * C::kKps + j);
+              const uint64_t adesc = adesc0 + static_cast<uint64_t>((s * C::kABytes + j * C::kABytes1) >> 4);
+              const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((s * C::kTokBytes + j * C::kTokBytes1) >> 4);
+              if (issuer)
                 tmem_cp_32x128b_x4(sfa, sfdesc0 + static_cast<uint64_t>((s * C::kSfBytes + j * kMxTileScaleBytes) >> 4));
 #pragma unroll
-                for (int k = 0; k < kBlockK / 32; ++k) {
-                  // scale byte k of the K block's four columns belongs to elements 32k .. 32k+31
+              for (int k = 0; k < kBlockK / 32; ++k) {
+                uint32_t accumulate = (i > 0 || j > 0 || k > 0) ? 1u : 0u;
+                if (NONE) {
+                  // a new weight group (by its absolute position in the row) starts a fresh partial sum in the
+                  // other buffer, once the epilogue warps have read what that buffer held
+                  const int gid = ((kb0 + i + j) * (kBlockK / 32) + k) / mpg;
+                  if (gid != gid_prev) {
+                    if (gid_prev >= 0 && issuer) umma_commit(&acc_full[gbuf]);
+                    gbuf = gcount & 1;
+                    if (gcount >= 2 && !mbar_wait(&acc_empty[gbuf], ((gcount >> 1) - 1) & 1, s_abort)) failed = true;
+                    tc_fence_after_sync();
+                    ++gcount;
+                    gid_prev = gid;
+                    accumulate = 0u;
+                    d_tmem = tmem_base + gbuf * C::kDColsPad;
+                  }
+                }
+                // scale byte k of the K block's four columns belongs to elements 32k .. 32k+31
+                if (issuer && !failed)
                   umma_mxf8f6f4(d_tmem, adesc + 2 * k, bdesc + 2 * k,
                                 W8 ? umma_idesc_mx_e4m3_e4m3(BM, k, 0) : umma_idesc_mx_e2m1_e4m3(BM, k, 0),
-                                sfa + (static_cast<uint32_t>(k) << 30), tmem_sfb, (i > 0 || j > 0 || k > 0) ? 1u : 0u);
-                }
+                                sfa + (static_cast<uint32_t>(k) << 30), tmem_sfb, accumulate);
               }
             }
+          }
+          if (issuer) {
             umma_commit(&empty[s]);
-            if (i + C::kKps >= nkb) umma_commit(&acc_full[buf]);
+            if (i + C::kKps >= nkb) umma_commit(&acc_full[NONE ? gbuf : buf]);
           }
           __syncwarp();
           if (++s == C::NS) {
@@ -395,6 +423,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
     constexpr int EC = BM <= 32 ? 4 : (BM <= 128 ? 8 : 16);  // columns per step
     bool failed = !ok_start;
     int m0_loaded = -1;
+    int gcount = 0;  // NONE: weight groups promoted so far
     pdl_wait();  // x, sx, t, the hand-over flags and y may still be in use by the kernel ahead in the stream
     if (FUSEQ) {
       // Section 3 / Appendix A, token-wise: a_m = max_k |x[m,k]|, q = RNE_E4M3(fl32(x * fl32(448 / a_m))), and
@@ -515,7 +544,8 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       const int n = (tile % p.n_tiles) * kTileN + row;
       const bool n_ok = n < p.N;
       const int buf = seg % C::NB;
-      const uint32_t t_lane = tmem_base + buf * C::kDColsPad + lane_base;
+      // where the finished tile is read from: the segment's accumulator, or (NONE) the region the promoted sums go to
+      const uint32_t t_lane = tmem_base + (NONE ? C::kResultCol0 : buf * C::kDColsPad) + lane_base;
 
       if (m0 != m0_loaded) {
         // token scales and (rank 8) LoRC rows of this tile's tokens
@@ -546,7 +576,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       uint64_t u[8];  // the channel's U row, each value in both halves of a packed pair
 #pragma unroll
       for (int e = 0; e < 8; ++e) u[e] = 0ull;
-      if (n_ok) cs = __ldg(p.scale + n);
+      if (n_ok && !NONE) cs = __ldg(p.scale + n);
       if (p.r == 8 && n_ok) {
         const uint4 h = __ldg(reinterpret_cast<const uint4*>(p.U + static_cast<int64_t>(n) * 8));
         const uint32_t hw[4] = {h.x, h.y, h.z, h.w};
@@ -559,7 +589,46 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
           u[2 * e + 1] = pack2(f.y, f.y);
         }
       }
-      if (!failed) {
+      if (NONE) {
+        // Per-group promotion (Section 3, the unconstrained scales that M1 / M2 do away with): every weight
+        // group's FP32 partial sum is multiplied by the group's scale S[n, g] and added to the running sums in
+        // registers, while the MMAs of the next group fill the other buffer.
+        const int mpg = p.group / 32;
+        const int g_first = (kb0 * (kBlockK / 32)) / mpg, g_last = ((kb0 + nkb) * (kBlockK / 32) - 1) / mpg;
+        const float* srow = p.scale + static_cast<int64_t>(n_ok ? n : 0) * p.G;
+        float run[BM];
+#pragma unroll
+        for (int c = 0; c < BM; ++c) run[c] = 0.0f;
+        float S_next = n_ok ? __ldg(srow + g_first) : 0.0f;
+        for (int g = g_first; g <= g_last; ++g) {
+          const float S = S_next;
+          if (n_ok && g < g_last) S_next = __ldg(srow + g + 1);
+          const int gb = gcount & 1;
+          if (!failed && !mbar_wait_warp(&acc_full[gb], (gcount >> 1) & 1, s_abort)) {
+            raise_error(p, s_abort, kErrEpilogue);
+            failed = true;
+          }
+          tc_fence_after_sync();
+          if (!failed) {
+            const uint32_t g_lane = tmem_base + gb * C::kDColsPad + lane_base;
+#pragma unroll
+            for (int c = 0; c < BM; c += 16) {
+              float v[16];
+              tmem_ld_cols<16>(g_lane + c, v);
+#pragma unroll
+              for (int e = 0; e < 16; ++e) run[c + e] = fmaf(S, v[e], run[c + e]);
+            }
+          }
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&acc_empty[gb]);  // the MMA warp may start a new group in this buffer
+          ++gcount;
+        }
+        // the finished tile goes to the result region, where the common code below finds it
+#pragma unroll
+        for (int c = 0; c < BM; c += 16) tmem_st16(t_lane + c, reinterpret_cast<const uint32_t*>(run + c));
+        tmem_st_wait();
+      } else if (!failed) {
         if (!mbar_wait_warp(&acc_full[buf], (seg / C::NB) & 1, s_abort)) {
           raise_error(p, s_abort, kErrEpilogue);
           failed = true;
@@ -680,7 +749,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
       // the accumulator buffer has been read: the MMA warp may reuse it
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&acc_empty[buf]);
+      if (!NONE && lane == 0) mbar_arrive(&acc_empty[buf]);
     }
   }
 
@@ -742,9 +811,9 @@ bool make_token_map(CUtensorMap* m, const void* base, uint64_t K, uint64_t M, ui
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BM, bool W8, bool FUSEQ>
+template <int BM, bool W8, bool FUSEQ, bool NONE>
 int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cudaStream_t st) {
-  using C = MxCfg<BM, W8>;
+  using C = MxCfg<BM, W8, NONE>;
   CUtensorMap tm_w, tm_q;
   if (!make_weight_map(&tm_w, a.codes, static_cast<uint64_t>(plan.n_tiles), static_cast<uint64_t>(p.kblocks), C::kKps, W8) ||
       !make_token_map(&tm_q, a.q, static_cast<uint64_t>(a.K), static_cast<uint64_t>(a.M), BM, C::kKps))
@@ -752,7 +821,7 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(w4a8_mx_gemm_kernel<BM, W8, FUSEQ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    attr_err = cudaFuncSetAttribute(w4a8_mx_gemm_kernel<BM, W8, FUSEQ, NONE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     C::kSmemBytes);
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
@@ -773,13 +842,13 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
     }
     void* args[3] = {&tm_w, &tm_q, &pc};
     // chained to the kernel ahead (see pdl_wait); if the two launch attributes are refused together, cooperative alone
-    if (launch_chained(w4a8_mx_gemm_kernel<BM, W8, FUSEQ>, grid, dim3(C::kThreads), C::kSmemBytes, st, true, tm_w, tm_q, pc) ==
+    if (launch_chained(w4a8_mx_gemm_kernel<BM, W8, FUSEQ, NONE>, grid, dim3(C::kThreads), C::kSmemBytes, st, true, tm_w, tm_q, pc) ==
         cudaSuccess) {
       count_launch();
       return ZQ_OK;
     }
     (void)cudaGetLastError();
-    if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM, W8, FUSEQ>), grid, dim3(C::kThreads),
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(w4a8_mx_gemm_kernel<BM, W8, FUSEQ, NONE>), grid, dim3(C::kThreads),
                                     args, C::kSmemBytes, st) == cudaSuccess) {
       count_launch();
       return ZQ_OK;
@@ -790,7 +859,7 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
                                         static_cast<size_t>(a.M), st) != cudaSuccess)
       return ZQ_ERR_CUDA;
   }
-  const cudaError_t err = launch_chained(w4a8_mx_gemm_kernel<BM, W8, FUSEQ>, grid, dim3(C::kThreads), C::kSmemBytes, st, false,
+  const cudaError_t err = launch_chained(w4a8_mx_gemm_kernel<BM, W8, FUSEQ, NONE>, grid, dim3(C::kThreads), C::kSmemBytes, st, false,
                                          tm_w, tm_q, p);
   count_launch();
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
@@ -799,7 +868,6 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
 }  // namespace
 
 int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
-  if (a.mode == ZQ_SCALE_NONE) return ZQ_ERR_MODE;
   const GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode, ZQ_WEIGHTS_MX);
   if (plan.partial_floats > a.partial_floats) return ZQ_ERR_WORKSPACE;
   Params p = make_params(a, plan);
@@ -810,10 +878,21 @@ int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
       return ZQ_ERR_SHAPE;
     p.sx = nullptr;
     p.t = p.fq->t_sum;  // token-major [M, r], as the separate quantizer writes it
-    return w8 ? launch_mx_cfg<16, true, true>(a, plan, p, st) : launch_mx_cfg<16, false, true>(a, plan, p, st);
+    if (a.mode == ZQ_SCALE_NONE) return ZQ_ERR_MODE;
+    return w8 ? launch_mx_cfg<16, true, true, false>(a, plan, p, st) : launch_mx_cfg<16, false, true, false>(a, plan, p, st);
+  }
+  if (a.mode == ZQ_SCALE_NONE) {  // unconstrained FP32 group scales: per-group promotion, token tiles up to 128
+    if (w8) return ZQ_ERR_MODE;
+    switch (plan.bm) {
+      case 16: return launch_mx_cfg<16, false, false, true>(a, plan, p, st);
+      case 32: return launch_mx_cfg<32, false, false, true>(a, plan, p, st);
+      case 64: return launch_mx_cfg<64, false, false, true>(a, plan, p, st);
+      case 128: return launch_mx_cfg<128, false, false, true>(a, plan, p, st);
+    }
+    return ZQ_ERR_SHAPE;
   }
 #define ZQ_MX_CASE(BM_) \
-  case BM_: return w8 ? launch_mx_cfg<BM_, true, false>(a, plan, p, st) : launch_mx_cfg<BM_, false, false>(a, plan, p, st)
+  case BM_: return w8 ? launch_mx_cfg<BM_, true, false, false>(a, plan, p, st) : launch_mx_cfg<BM_, false, false, false>(a, plan, p, st)
   switch (plan.bm) {
     ZQ_MX_CASE(16);
     ZQ_MX_CASE(32);

@@ -91,7 +91,6 @@ def test_validation_before_launch(L):
     assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 0, 2, fake, fake, fake, null) == -4   # FP8 codes need M1 / M2
     assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 0, 3, fake, fake, fake, null) == -4   # so does the E5M2 target
     assert L.zq_pack_weight_fp4(fake, 4, 640, 320, 0, 0, fake, fake, fake, null) == -2   # groups of 320: M1 / M2 only
-    assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 0, 1, fake, fake, fake, null) == -4   # block scales need M1 / M2
     assert L.zq_pack_weight_fp4(fake, 4, 256, 128, 1, 0, fake, null, fake, null) == -1
     assert L.zq_pack_weight_fp4(fake, 0, 256, 128, 1, 1, fake, fake, fake, null) == 0
     # linear
@@ -115,7 +114,7 @@ def test_validation_before_launch(L):
     assert call(ldy=64) == -2
     assert call(codes=C.c_void_p(0x1008)) == -3
     assert call(layout=1, codes=C.c_void_p(0x1010)) == -3   # the 4-bit tensor map wants 32-byte alignment
-    assert call(layout=1, mode=0) == -4
+    assert call(layout=2, mode=0) == -4
     assert call(layout=4) == -4
     assert call(ws=null) == -5
     assert call(wsb=1024) == -5

@@ -63,8 +63,8 @@ def _run_layer(wl, shape, modes, Ms, lorc_variants=(True,)):
     ws = binding.make_workspace(binding.linear_workspace_bytes(Mmax, N, K, r))
     for mode in modes:
         c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, wl.group, mode)
-        # both weight layouts for the constrained modes: the kernel that casts and the block-scaled one
-        layouts = [binding.WEIGHTS_CAST] + ([binding.WEIGHTS_MX] if mode != "none" else [])
+        # both weight layouts: the kernel that casts and the block-scaled one
+        layouts = [binding.WEIGHTS_CAST, binding.WEIGHTS_MX]
         pws = []
         for layout in layouts:
             pw = binding.pack_weight_fp4(W_d, wl.group, mode, layout)

@@ -23,11 +23,37 @@ def test_pack_weight_mx_bit_exact(mode, group):
     check_packed(binding.pack_weight_fp4(up(W), group, mode, MX), c_o, sh_o, sc_o, group)
 
 
-def test_mx_layout_rejects_unconstrained_scales():
-    W = up(synth.make_w(1, 128, 256))
-    with pytest.raises(binding.ZqError) as e:
-        binding.pack_weight_fp4(W, 128, "none", MX)
-    assert e.value.status == -4
+@pytest.mark.parametrize("group", [64, 128, 256])
+def test_pack_weight_mx_unconstrained_scales(group):
+    # mode none in the block-scaled arrangement: the same codes, unit block scales, FP32 scales beside them
+    W = _special_weights(9, 512, 31)
+    c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, group, "none")
+    check_packed(binding.pack_weight_fp4(up(W), group, "none", MX), c_o, sh_o, sc_o, group)
+
+
+@pytest.mark.parametrize("group", [64, 128, 256])
+@pytest.mark.parametrize("M,N,K,r", [(1, 384, 1024, 8), (16, 256, 8192, 8), (40, 200, 2048, 0), (100, 640, 512, 8),
+                                     (128, 128 * 9, 768, 16), (300, 1000, 1024, 8), (700, 128 * 150, 512, 8)])
+def test_linear_unconstrained_scales(M, N, K, r, group):
+    # per-group promotion with the FP32 group scale (Section 3: what M1 / M2 remove) in the block-scaled kernel:
+    # unit ranges with shared tiles, whole tiles, several token tiles of 128, groups of half / one / two K blocks
+    x_bits, W, U, V = _layer(900 + M, M, N, K, r)
+    rows = None if M <= 300 else [0, 127, 128, 255, 256, 511, 512, M - 1]
+    check_linear(x_bits, W, U, V, group, "none", layout=MX, rows=rows)
+
+
+def test_linear_unconstrained_scales_bf16_and_exact():
+    x_bits, W, U, V = _layer(950, 48, 512, 1024, 8)
+    check_linear(x_bits, W, U, V, 128, "none", out_dtype=torch.bfloat16, layout=MX)
+    M, N, K = 16, 256, 512
+    rng = np.random.default_rng(5)
+    x = rng.choice([0.0, 0.25, 0.5, 1.0, -1.0, 2.0], (M, K)).astype(np.float32)
+    x[:, 0] = 7.0
+    W = rng.choice([0.0, 0.5, -1.0, 1.5, 3.0, -4.0], (N, K)).astype(np.float32)
+    W[:, ::128] = 6.0
+    W[3, 128:256] *= 0.125
+    y, y_o = check_linear(synth.f32_to_bf16_bits(x), W, None, None, 128, "none", layout=MX)
+    assert np.array_equal(y, y_o)
 
 
 @pytest.mark.parametrize("mode", ["M1", "M2"])

@@ -95,5 +95,7 @@ def test_plan_tile_choices_of_the_block_scaled_kernel():
     assert binding.linear_plan(8192, 7168, 28672, "M2", "mx")["bm"] == 256
     p = binding.linear_plan(8192, 7168, 28672, "M2", "mx")
     assert p["persist"] == 1 and p["tail_pos0"] == (32 * 56) // p["ctas"] * p["ctas"]   # 12 whole rounds
+    # unconstrained scales: the running sums of a tile live in registers, so its token tiles stop at 128
+    assert [binding.linear_plan(M, 4096, 4096, "none", "mx")["bm"] for M in (16, 100, 300, 2048)] == [16, 128, 128, 128]
     with pytest.raises(binding.ZqError):
-        binding.linear_plan(16, 128, 256, "none", "mx")
+        binding.linear_plan(16, 128, 256, "none", "mx_fp8")
