@@ -42,7 +42,7 @@ NOMINAL_FP8_TFLOPS = 4500.0  # public dense FP8 figure of the part, for context
 DOMINANT_TRAFFIC = None
 DECODE_TRAFFIC = None
 # LLaMA-7B-shaped rows outside the timed step: (scale mode, weight layout)
-EXTRA_LLAMA7B = (("none", "cast"), ("M2", "mx"))
+EXTRA_LLAMA7B = (("none", "cast"), ("none", "mx"), ("M2", "mx"))
 METRIC = "w4a8_linear_tflops"
 UNIT = "TFLOP/s"
 N_WEIGHT_COPIES = 2  # per layer; rotated so that > 2x the L2 size streams between two reads of one buffer
@@ -473,6 +473,7 @@ def run_ours(args):
     # ---- per (layer, M): steady-state times of each shape by itself, after the timed region
     table = []
     if not args.no_sweep_table:
+        time.sleep(1.5)  # the timed region ends power-capped; the per-shape rows are kernels timed by themselves
         for li, M in calls:
             ly = layers[li]
             tl, tq, tg = B.time_shape(ly, M, n=20 if M <= 2048 else 6)
@@ -595,7 +596,7 @@ def run_ours(args):
             "timed_region_s": round(ms_max * 1e-3, 3),
             "roofline": roofline, "roofline_decode": roofline_decode, "roofline_quant": roofline_quant,
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-            "sweep_note": "per-shape rows: each (layer, M) timed by itself after the timed region: one event pair "
+            "sweep_note": "per-shape rows: each (layer, M) timed by itself after the timed region and a 1.5 s pause: one event pair "
                           "around n = 6-20 back-to-back launches (rotated weight copies), divided by n, median of 3 "
                           "batches; layer_us = one zq_w4a8_linear call on raw x; quant_us / gemm_us = the quantizer "
                           "kernel alone and the GEMM alone on pre-quantized activations",

@@ -611,10 +611,16 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
           tc_fence_after_sync();
           if (!failed) {
             const uint32_t g_lane = tmem_base + gb * C::kDColsPad + lane_base;
+            // the next 16 columns are in flight while these are added up
+            float nxt[16];
+            tmem_ld_issue<16>(g_lane, nxt);
 #pragma unroll
             for (int c = 0; c < BM; c += 16) {
               float v[16];
-              tmem_ld_cols<16>(g_lane + c, v);
+              tmem_ld_wait_regs<16>(nxt);
+#pragma unroll
+              for (int e = 0; e < 16; ++e) v[e] = nxt[e];
+              if (c + 16 < BM) tmem_ld_issue<16>(g_lane + c + 16, nxt);
 #pragma unroll
               for (int e = 0; e < 16; ++e) run[c + e] = fmaf(S, v[e], run[c + e]);
             }
