@@ -186,9 +186,14 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
  *                tiles from tail_pos0 on are dealt out as ranges like stream),
  *   [6] splits, [7] kb_per_split (neither stream nor persist: CTA z * tiles + pos takes K blocks
  *                [z * kb_per_split, ...) of the tile at position pos),
- *   [8] base, [9] rem, [10] tail_pos0, [11] m_group, [12] floats of partial-sum scratch, [13] SMs assumed.
+ *   [8] base, [9] rem, [10] tail_pos0, [11] m_group, [12] floats of partial-sum scratch, [13] SMs assumed,
+ *   [14] pair   (1, with persist: the CTAs work in pairs, CTAs 2c and 2c + 1 on one token tile and two
+ *                neighbouring channel tiles; pair c walks the pair positions c, c + ctas / 2, ... of
+ *                m_tiles x n_tiles / 2, whole tiles only; a pair position maps to (token tile, channel-tile
+ *                pair) through the same groups of m_group token tiles, and CTA 2c + h takes channel tile
+ *                2 * pair + h).
  */
-#define ZQ_PLAN_WORDS 14
+#define ZQ_PLAN_WORDS 15
 int zq_w4a8_linear_plan(int64_t M, int64_t N, int64_t K, zq_scale_mode mode, zq_weight_layout layout,
                         int64_t* plan);
 

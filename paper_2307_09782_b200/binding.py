@@ -29,7 +29,7 @@ EXPORTS = [
     "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc", "zq_w4a8_linear_noalloc_status", "zq_w4a8_linear_plan", "zq_selftest_bounded_wait", "zq_lorc_workspace_bytes", "zq_lorc_factors",
 ]
 PLAN_FIELDS = ("bm", "m_tiles", "n_tiles", "ctas", "stream", "persist", "splits", "kb_per_split", "base", "rem",
-               "tail_pos0", "m_group", "partial_floats", "sms")
+               "tail_pos0", "m_group", "partial_floats", "sms", "pair")
 
 
 class ZqError(RuntimeError):

@@ -278,7 +278,7 @@ int zq_w4a8_linear_plan(int64_t M, int64_t N, int64_t K, zq_scale_mode mode, zq_
   const GemmPlan pl = plan_gemm(M, N, K, mode, layout);
   const int64_t v[ZQ_PLAN_WORDS] = {pl.bm,   pl.m_tiles,     pl.n_tiles, pl.ctas, pl.stream,    pl.persist,
                                     pl.splits, pl.kb_per_split, pl.base,  pl.rem,  pl.tail_pos0, pl.m_group,
-                                    static_cast<int64_t>(pl.partial_floats), sm_count()};
+                                    static_cast<int64_t>(pl.partial_floats), sm_count(), pl.pair};
   for (int i = 0; i < ZQ_PLAN_WORDS; ++i) plan[i] = v[i];
   return ZQ_OK;
 }

@@ -681,6 +681,36 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
     pl.base = static_cast<int>(tail_tiles * kblocks / g);
     pl.rem = static_cast<int>(tail_tiles * kblocks % g);
     pl.partial_floats = tail_tiles > 0 ? 2 * static_cast<size_t>(g) * bm * kTileN : 0;
+    if (wide && bm >= 192 && pl.n_tiles % 2 == 0 && sm_count() >= 2) {
+      // CTA pairs (two CTAs share each token tile and take two neighbouring channel tiles): whole tiles only,
+      // pair c walks the pair positions c, c + pairs, ...  The token tile (224 or 192 tokens: two accumulators)
+      // is the one with the fewest rounds x width; taken unless its last, incomplete round would cost more
+      // than the pairs save.
+      const int64_t pairs = sm_count() / 2, np = pl.n_tiles / 2;
+      int best_bm = 0;
+      int64_t best_cost = 0;
+      for (const int cand : {224, 192}) {
+        const int64_t mt = (M + cand - 1) / cand;
+        const int64_t cost = ((mt * np + pairs - 1) / pairs) * cand;
+        if (best_bm == 0 || cost < best_cost) {
+          best_bm = cand;
+          best_cost = cost;
+        }
+      }
+      const double single_cost = static_cast<double>(tiles) * bm / sm_count();
+      if (static_cast<double>(best_cost) <= 1.10 * single_cost) {
+        pl.pair = 1;
+        pl.bm = best_bm;
+        pl.m_tiles = static_cast<int>((M + best_bm - 1) / best_bm);
+        const int64_t positions = pl.m_tiles * np;
+        pl.ctas = static_cast<int>(2 * (positions < pairs ? positions : pairs));
+        pl.tail_pos0 = pl.m_tiles * pl.n_tiles;
+        pl.base = pl.rem = 0;
+        pl.partial_floats = 0;
+        const int64_t fit = (int64_t(32) << 20) / (static_cast<int64_t>(best_bm) * K);
+        pl.m_group = pl.m_tiles > 1 ? static_cast<int>(fit < 1 ? 1 : (fit > 8 ? 8 : fit)) : 0;
+      }
+    }
     return pl;
   }
   if ((mx || (mode != ZQ_SCALE_NONE && bm == 16 && pl.m_tiles == 1)) && tiles <= kWsMaxTiles && units >= 8 &&

@@ -785,6 +785,303 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
   }
 }
 
+// ---- many tokens: CTA pairs ---------------------------------------------------------------------------
+// With wide token tiles the kernel above is bound by the bytes that reach shared memory: per K block 16 KB of
+// codes and 128 bytes per token.  Here the two CTAs of a cluster share one token tile: one MMA of 256 channels x
+// BM tokens (cta_group::2) reads channels 0..127 and tokens 0..BM/2-1 from the leader's shared memory, channels
+// 128..255 and the other half of the tokens from its peer's, and accumulates each CTA's 128 channels in that
+// CTA's own tensor memory.  Each CTA loads its own weight tile, scales and half of the tokens (all counted on
+// the leader's barrier), the leader's MMA thread issues for both, its commits release the stages and publish
+// the accumulators in both CTAs, and each CTA's epilogue warps finish their own 128 channels.  The token bytes
+// per CTA and K block are halved.
+// Whole output tiles only: pair `c` of the grid walks pair positions c, c + pairs, ... below p.pair_end.
+template <int BM, bool W8>
+struct PairCfg {
+  static constexpr int kThreads = 192;
+  static constexpr int kEpiThreads = 128;
+  static constexpr int kProducerWarp = 4;
+  static constexpr int kMmaWarp = 5;
+  static constexpr int kHalf = BM / 2;  // token rows in each CTA's shared memory
+  static constexpr int kCodeBytes = W8 ? 2 * kTileCodeBytes : kTileCodeBytes;  // a tile's codes in HBM
+  static constexpr int kABytes = kTileRows * kTileK;  // in shared memory (padded FP4, or FP8)
+  static constexpr int kTokBytes = kHalf * kBlockK;
+  static constexpr int kSfBytes = kMxTileScaleBytes;
+  static constexpr int kStageTx = kCodeBytes + kTokBytes + kSfBytes;  // bytes one CTA's copies of a stage count
+  static constexpr int kStageBytes = kABytes + kTokBytes + kSfBytes;
+  static constexpr int NS = cmin(8, (218 * 1024 - BM * 36 - 512) / kStageBytes);
+  static constexpr int NB = 2;  // accumulator buffers
+  static constexpr int kSfaCol0 = NB * BM;
+  static constexpr int kSfbCol0 = kSfaCol0 + 4 * NS;
+  static constexpr int kColsUsed = kSfbCol0 + kSfbCols;
+  static constexpr int kTmemCols = 512;
+  static constexpr int offA = 0;
+  static constexpr int offTok = offA + NS * kABytes;
+  static constexpr int offSf = offTok + NS * kTokBytes;
+  static constexpr int offSx = offSf + NS * kSfBytes;
+  static constexpr int offT = offSx + BM * 4;
+  static constexpr int offBars = offT + BM * 32;
+  static constexpr int kNumBars = 2 * NS + 2 * NB + 1;
+  static constexpr int offMisc = offBars + kNumBars * 8;
+  static constexpr int kSmemBytes = offMisc + 32;
+  static_assert(BM % 32 == 0 && BM >= 64 && BM <= 224, "token tile of the pair: two accumulators");
+  static_assert(kTokBytes % 1024 == 0, "token stages must start on a swizzle atom");
+  static_assert(NS >= 4, "pipeline depth");
+  static_assert(kColsUsed <= kTmemCols, "tensor memory");
+  static_assert(kSmemBytes <= 226 * 1024, "shared memory");
+};
+
+// Pair position -> (token tile, pair of channel tiles).  Like raster_tile: through groups of m_group token
+// tiles, the group's token tiles inner, so that the pairs running at one time share operands in L2.
+__device__ __forceinline__ void pair_tile(const Params& p, int pos, int& m_tile, int& n_pair) {
+  const int np = p.n_tiles / 2, m_tiles = p.tiles / p.n_tiles;
+  const int mg = p.m_group < 1 ? 1 : p.m_group;
+  const int per_group = mg * np;
+  const int g = pos / per_group, within = pos - g * per_group;
+  const int gm = min(mg, m_tiles - g * mg);
+  m_tile = g * mg + within % gm;
+  n_pair = within / gm;
+}
+
+template <int BM, bool W8>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairCfg<BM, W8>::kThreads, 1)
+w4a8_mx_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_q,
+                         const __grid_constant__ CUtensorMap tm_sf, const Params p) {
+  using C = PairCfg<BM, W8>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint8_t* s_a = smem + C::offA;
+  uint8_t* s_tok = smem + C::offTok;
+  uint8_t* s_sf = smem + C::offSf;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::offBars);
+  uint64_t* full = bars;                  // [NS] leader's: both CTAs' copies of the stage landed   (MMA waits)
+  uint64_t* empty = full + C::NS;         // [NS] each CTA's: the MMAs that read the stage are done  (producers wait)
+  uint64_t* acc_full = empty + C::NS;     // [NB] each CTA's: a tile's accumulation is complete      (epilogues wait)
+  uint64_t* acc_empty = acc_full + C::NB; // [NB] leader's: both CTAs' epilogues have read the buffer (MMA waits)
+  uint64_t* drain_bar = acc_empty + C::NB;
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + C::offMisc);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + C::offMisc + 4);
+  float* s_sx = reinterpret_cast<float*>(smem + C::offSx);
+  float* s_t = reinterpret_cast<float*>(smem + C::offT);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const int pairs = static_cast<int>(gridDim.x) / 2, pair = static_cast<int>(blockIdx.x) / 2;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < C::NS; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
+    }
+    for (int i = 0; i < C::NB; ++i) {
+      mbar_init(&acc_full[i], 1);
+      mbar_init(&acc_empty[i], 8);  // one arrival per epilogue warp of either CTA
+    }
+    mbar_init(drain_bar, 1);
+    *s_abort = 0;
+    fence_mbar_init();
+    if ((smem_u32(smem) & 1023u) != 0) raise_error(p, s_abort, kErrAlign);
+  }
+  if (warp == C::kProducerWarp && lane == 0) {
+    prefetch_tensormap(&tm_w);
+    prefetch_tensormap(&tm_q);
+    prefetch_tensormap(&tm_sf);
+  }
+  if (warp == C::kMmaWarp) tmem_alloc_pair(s_tmem, C::kTmemCols);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *s_tmem;
+  const uint32_t tmem_sfa = tmem_base + C::kSfaCol0;
+  const uint32_t tmem_sfb = tmem_base + C::kSfbCol0;
+  if (warp < 4) {
+    // the tokens' block scales are all 2^0: each CTA fills its copy once
+    uint32_t ones[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) ones[i] = 0x7F7F7F7Fu;
+    tmem_st16(tmem_sfb + (static_cast<uint32_t>(warp * 32) << 16), ones);
+    tmem_st_wait();
+  }
+  tc_fence_before_sync();
+  cluster_sync_all();  // both CTAs' barriers are initialized, their tensor memory allocated and the scales of one written
+  tc_fence_after_sync();
+  const bool ok_start = (*s_abort == 0);
+  if (threadIdx.x == 0) pdl_launch_dependents();
+
+  if (warp == C::kProducerWarp) {
+    // ------------------------------------------------------------------ producer (both CTAs)
+    if (ok_start) {
+      const bool issuer = elect_one();
+      pdl_wait();  // the tokens may be the output of the kernel ahead in the stream
+      int s = 0, issued = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int pos = pair; ok && pos < p.pair_end; pos += pairs) {
+        int m_tile, n_pair;
+        pair_tile(p, pos, m_tile, n_pair);
+        const int nt = 2 * n_pair + static_cast<int>(rank);
+        const int row0 = m_tile * BM + static_cast<int>(rank) * C::kHalf;
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (issued >= C::NS && !mbar_wait(&empty[s], ph ^ 1, s_abort)) {
+            if (issuer) raise_error(p, s_abort, kErrProducer);
+            ok = false;
+            break;
+          }
+          if (issuer) {
+            const uint32_t bar = map_to_rank(smem_u32(&full[s]), 0);
+            if (leader) mbar_arrive_expect_tx(&full[s], 2 * C::kStageTx);
+            tma_load_4d_pair(s_a + s * C::kABytes, &tm_w, 0, 0, kb, nt, bar);
+            tma_load_3d_pair(s_sf + s * C::kSfBytes, &tm_sf, 0, 4 * kb, nt, bar);
+            tma_load_3d_pair(s_tok + s * C::kTokBytes, &tm_q, 0, row0, kb, bar);
+          }
+          __syncwarp();
+          ++issued;
+          if (++s == C::NS) {
+            s = 0;
+            ph ^= 1;
+          }
+        }
+      }
+      // never leave with copies still in flight: the stages this CTA filled last are released by the MMAs that
+      // read them, which run only after the copies landed
+      for (int i = max(0, issued - C::NS); i < issued; ++i) {
+        uint32_t spin = 0;
+        while (!mbar_try_wait(&empty[i % C::NS], (i / C::NS) & 1) && ++spin < kSpinLimit && !*s_abort) {
+        }
+      }
+    }
+  } else if (warp == C::kMmaWarp) {
+    // ------------------------------------------------------------------ MMA issuer (leader only)
+    if (ok_start && leader) {
+      const bool issuer = elect_one();
+      const uint64_t adesc0 = umma_desc_k128(smem_u32(s_a));
+      const uint64_t bdesc0 = umma_desc_k128(smem_u32(s_tok));
+      const uint64_t sfdesc0 = umma_desc_rows16(smem_u32(s_sf), 128);
+      int s = 0, seg = 0;
+      uint32_t ph = 0;
+      bool failed = false;
+      for (int pos = pair; !failed && pos < p.pair_end; pos += pairs, ++seg) {
+        const int buf = seg % C::NB;
+        if (seg >= C::NB && !mbar_wait(&acc_empty[buf], ((seg / C::NB) - 1) & 1, s_abort)) {
+          failed = true;
+          break;
+        }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + buf * BM;
+        for (int kb = 0; kb < p.kblocks && !failed; ++kb) {
+          if (!mbar_wait(&full[s], ph, s_abort)) {
+            failed = true;
+            break;
+          }
+          tc_fence_after_sync();
+          if (issuer) {
+            const uint32_t sfa = tmem_sfa + 4 * s;
+            const uint64_t adesc = adesc0 + static_cast<uint64_t>((s * C::kABytes) >> 4);
+            const uint64_t bdesc = bdesc0 + static_cast<uint64_t>((s * C::kTokBytes) >> 4);
+            tmem_cp_32x128b_x4_pair(sfa, sfdesc0 + static_cast<uint64_t>((s * C::kSfBytes) >> 4));
+#pragma unroll
+            for (int k = 0; k < kBlockK / 32; ++k) {
+              const uint32_t idesc = (W8 ? umma_idesc_mx_e4m3_e4m3(BM, k, 0) : umma_idesc_mx_e2m1_e4m3(BM, k, 0)) +
+                                     ((128u >> 4) << 24);  // 256 rows: 128 in each CTA
+              umma_mxf8f6f4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, sfa + (static_cast<uint32_t>(k) << 30),
+                                 tmem_sfb, (kb > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit_pair(&empty[s]);
+            if (kb + 1 == p.kblocks) umma_commit_pair(&acc_full[buf]);
+          }
+          __syncwarp();
+          if (++s == C::NS) {
+            s = 0;
+            ph ^= 1;
+          }
+        }
+      }
+      if (failed) {
+        if (issuer) {
+          raise_error(p, s_abort, kErrMma);
+          umma_commit_pair(drain_bar);  // let the MMAs already issued finish before tensor memory is released
+        }
+        uint32_t spin = 0;
+        while (!mbar_try_wait(drain_bar, 0) && ++spin < kSpinLimit) {
+        }
+      }
+      __syncwarp();
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (both CTAs, own 128 channels)
+    const int row = warp * 32 + lane;
+    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    constexpr int EC = 16;
+    bool failed = !ok_start;
+    int m0_loaded = -1;
+    pdl_wait();  // sx, t and y may still be in use by the kernel ahead in the stream
+    int seg = 0;
+    for (int pos = pair; pos < p.pair_end; pos += pairs, ++seg) {
+      int m_tile, n_pair;
+      pair_tile(p, pos, m_tile, n_pair);
+      const int m0 = m_tile * BM;
+      const int n = (2 * n_pair + static_cast<int>(rank)) * kTileN + row;
+      const bool n_ok = n < p.N;
+      const int buf = seg % C::NB;
+      const uint32_t t_lane = tmem_base + buf * BM + lane_base;
+      if (m0 != m0_loaded) {
+        named_bar_sync(2, C::kEpiThreads);  // the previous tile's reads are done
+        for (int c = threadIdx.x; c < BM; c += C::kEpiThreads) s_sx[c] = (m0 + c < p.M) ? __ldg(p.sx + m0 + c) : 0.0f;
+        if (p.r == 8)
+          for (int c = threadIdx.x; c < BM * 8; c += C::kEpiThreads)  // transposed: [j][BM]
+            s_t[(c & 7) * BM + (c >> 3)] = (m0 + (c >> 3) < p.M) ? __ldg(p.t + static_cast<int64_t>(m0) * 8 + c) : 0.0f;
+        named_bar_sync(2, C::kEpiThreads);
+        m0_loaded = m0;
+      }
+      float cs = 1.0f;
+      uint64_t u[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) u[e] = 0ull;
+      if (n_ok) cs = __ldg(p.scale + n);
+      if (p.r == 8 && n_ok) {
+        const uint4 h = __ldg(reinterpret_cast<const uint4*>(p.U + static_cast<int64_t>(n) * 8));
+        const uint32_t hw[4] = {h.x, h.y, h.z, h.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __half2 h2;
+          *reinterpret_cast<uint32_t*>(&h2) = hw[e];
+          const float2 f = __half22float2(h2);
+          u[2 * e] = pack2(f.x, f.x);
+          u[2 * e + 1] = pack2(f.y, f.y);
+        }
+      }
+      if (!failed && !mbar_wait_warp(&acc_full[buf], (seg / C::NB) & 1, s_abort)) {
+        raise_error(p, s_abort, kErrEpilogue);
+        failed = true;
+      }
+      tc_fence_after_sync();
+      if (!failed) {
+        float nxt[EC];
+        tmem_ld_issue<EC>(t_lane, nxt);
+#pragma unroll 1
+        for (int c = 0; c < BM; c += EC) {
+          float v[EC];
+          tmem_ld_wait_regs<EC>(nxt);
+#pragma unroll
+          for (int e = 0; e < EC; ++e) v[e] = nxt[e];
+          if (c + EC < BM) tmem_ld_issue<EC>(t_lane + c + EC, nxt);
+          if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t);
+        }
+      }
+      // this warp has read the buffer: tell the leader's MMA thread
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&acc_empty[buf]), 0));
+    }
+  }
+
+  tc_fence_before_sync();
+  cluster_sync_all();  // both CTAs are done with both CTAs' tensor memory and barriers
+  if (warp == C::kMmaWarp) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, C::kTmemCols);
+  }
+}
+
 // ---- host ------------------------------------------------------------------------------------------
 // The packed weight as a 4-D tensor of 4-bit elements [row blocks][K blocks][128 rows][128 elements]; the copy
 // engine expands a box of `kps` 128 x 128 tiles to the 16-byte-aligned FP4 form in shared memory, 128-byte
@@ -871,6 +1168,57 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
 }
 
+// The tiles' E8M0 scales (512 bytes per tile, behind the row block's codes) as a 3-D tensor
+// [row blocks][4 * K blocks][128 bytes]: a box of 4 rows is one tile's scales.
+bool make_scale_map(CUtensorMap* m, const void* codes, uint64_t n_tiles, uint64_t kblocks, bool w8) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const uint64_t code_bytes = w8 ? 2 * kTileCodeBytes : kTileCodeBytes;
+  const cuuint64_t dims[3] = {128, 4 * kblocks, n_tiles};
+  const cuuint64_t strides[2] = {128, kblocks * (code_bytes + kMxTileScaleBytes)};
+  const cuuint32_t box[3] = {128, 4, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const uint8_t* base = static_cast<const uint8_t*>(codes) + kblocks * code_bytes;
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<uint8_t*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Returns kPairNotTaken when the device grants no CTA pair for this kernel; nothing has run then.
+constexpr int kPairNotTaken = -1001;
+template <int BM, bool W8>
+int launch_pair_cfg(const GemmArgs& a, const GemmPlan& plan, Params p, cudaStream_t st) {
+  using C = PairCfg<BM, W8>;
+  auto kernel = w4a8_mx_pair_gemm_kernel<BM, W8>;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  static int max_pairs = 0;
+  std::call_once(once, [&] {
+    attr_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    if (attr_err == cudaSuccess) {
+      cudaLaunchConfig_t cfg{};
+      cfg.gridDim = dim3(2 * sm_count());
+      cfg.blockDim = dim3(C::kThreads);
+      cfg.dynamicSmemBytes = C::kSmemBytes;
+      if (cudaOccupancyMaxActiveClusters(&max_pairs, kernel, &cfg) != cudaSuccess) max_pairs = 0;
+      (void)cudaGetLastError();
+    }
+  });
+  if (attr_err != cudaSuccess || max_pairs < 1) return kPairNotTaken;
+  CUtensorMap tm_w, tm_q, tm_sf;
+  if (!make_weight_map(&tm_w, a.codes, static_cast<uint64_t>(plan.n_tiles), static_cast<uint64_t>(p.kblocks), 1, W8) ||
+      !make_token_map(&tm_q, a.q, static_cast<uint64_t>(a.K), static_cast<uint64_t>(a.M), C::kHalf, 1) ||
+      !make_scale_map(&tm_sf, a.codes, static_cast<uint64_t>(plan.n_tiles), static_cast<uint64_t>(p.kblocks), W8))
+    return ZQ_ERR_CUDA;
+  const int positions = plan.m_tiles * (plan.n_tiles / 2);
+  p.pair_end = positions;
+  const int pairs = positions < max_pairs ? positions : max_pairs;
+  const cudaError_t err = launch_chained(kernel, dim3(2 * pairs), dim3(C::kThreads), C::kSmemBytes, st, false, tm_w,
+                                         tm_q, tm_sf, p);
+  count_launch();
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
+}
+
 }  // namespace
 
 int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
@@ -896,6 +1244,16 @@ int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
       case 128: return launch_mx_cfg<128, false, false, true>(a, plan, p, st);
     }
     return ZQ_ERR_SHAPE;
+  }
+  if (plan.pair) {
+    // many tokens, whole tiles: CTA pairs sharing each token tile
+    int e = kPairNotTaken;
+    switch (plan.bm) {
+      case 192: e = w8 ? launch_pair_cfg<192, true>(a, plan, p, st) : launch_pair_cfg<192, false>(a, plan, p, st); break;
+      case 224: e = w8 ? launch_pair_cfg<224, true>(a, plan, p, st) : launch_pair_cfg<224, false>(a, plan, p, st); break;
+    }
+    if (e != kPairNotTaken) return e;
+    return ZQ_ERR_CUDA;  // the device grants this kernel no CTA pair
   }
 #define ZQ_MX_CASE(BM_) \
   case BM_: return w8 ? launch_mx_cfg<BM_, true, false, false>(a, plan, p, st) : launch_mx_cfg<BM_, false, false, false>(a, plan, p, st)

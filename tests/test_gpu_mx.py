@@ -107,6 +107,40 @@ def test_linear_persistent_whole_tiles(M):
     check_linear(x_bits, W, U, V, 128, "M2", layout=MX, rows=rows)
 
 
+@pytest.mark.parametrize("M,N,K,r,mode,layout,out_dtype", [
+    (1120, 128 * 120, 512, 8, "M2", MX, torch.bfloat16),           # 224-token tiles, bf16 y
+    (1000, 128 * 120 - 37, 384, 8, "M1", MX, torch.float32),       # 192-token tiles, ragged last channel tile
+    (1100, 128 * 120, 256, 0, "M2", MX, torch.float32),            # no LoRC
+    (1120, 128 * 120, 256, 16, "M2", MX, torch.float32),           # a rank the epilogue reads through the cache
+    (896, 128 * 148, 256, 8, "M2", MX, torch.float32),             # four whole rounds of 74 pairs
+])
+def test_linear_cta_pairs(M, N, K, r, mode, layout, out_dtype):
+    """Many tokens and an even number of channel tiles: two CTAs share each token tile (one MMA of 256 channels
+    over both CTAs' tensor memory), whole tiles only."""
+    pl = binding.linear_plan(M, N, K, mode, layout)
+    assert pl["pair"] == 1 and pl["bm"] in (192, 224)
+    x_bits, W, U, V = _layer(91 + r, M, N, K, r)
+    bm = pl["bm"]
+    rows = sorted({0, bm // 2 - 1, bm // 2, bm - 1, bm, bm + bm // 2, 2 * bm - 1, 3 * bm + 5, M - bm // 2 - 1, M - 2, M - 1})
+    check_linear(x_bits, W, U, V, 128, mode, layout=layout, rows=rows, out_dtype=out_dtype)
+
+
+def test_linear_cta_pairs_fp8_weights():
+    M, N, K, r = 1120, 128 * 120, 384, 8
+    assert binding.linear_plan(M, N, K, "M2", binding.WEIGHTS_MX_FP8)["pair"] == 1
+    x_bits, W, U, V = _layer(97, M, N, K, r)
+    rows = [0, 111, 112, 223, 224, 500, M - 113, M - 1]
+    q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
+    c_o, sh_o, sc_o = oracle.pack_weight(W, 128, "M2", "e4m3", 127)
+    y_o = oracle.linear_general(q_o[rows], sx_o[rows], c_o, sh_o, sc_o, 128, "M2", "e4m3", U, t_o[rows])
+    pw = binding.pack_weight_fp4(up(W), 128, "M2", binding.WEIGHTS_MX_FP8)
+    ws = binding.make_workspace(binding.linear_workspace_bytes(M, N, K, r))
+    q, sx, t = binding.quantize_act_fp8(to_bf16(x_bits), up(V))
+    y = binding.w4a8_linear(pw, q=q, sx=sx, t=t, U=up(U), workspace=ws)
+    assert binding.device_status(ws) == (0, 0)
+    assert np.abs(host(y).astype(np.float64)[rows] - y_o).max() <= TOL_REL * np.abs(y_o).max()
+
+
 @pytest.mark.parametrize("out_dtype", [torch.float32, torch.bfloat16])
 def test_linear_persistent_last_round_shared(out_dtype):
     # 600 tiles of 72 K blocks on 148 SMs: four whole rounds, then the 8 tiles of the last round are dealt

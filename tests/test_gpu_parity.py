@@ -28,9 +28,12 @@ def test_act_quant_bit_exact(M, K):
 
 @pytest.mark.parametrize("M,K,lorc", [(1187, 768, True), (1184, 2048, False), (2500, 256, True), (385, 4096, True),
                                       (384, 48, True), (300, 16384, True), (1030, 7168, True), (520, 28672, True),
-                                      (400, 3584, False), (390, 14336, True), (386, 28704, True)])
+                                      (400, 3584, False), (390, 14336, True), (386, 28704, True),
+                                      (388, 33024, True), (391, 4112, True), (8192, 1024, True)])
 def test_act_quant_many_rows_kernel(M, K, lorc):
-    """Token counts large enough for the eight-rows-per-CTA kernel, with a ragged last CTA."""
+    """Token counts large enough for the eight-rows kernels (one pass with the rows in shared memory, split over a
+    cluster of 1 / 2 / 4 / 8 CTAs by row length; two passes beyond 32768 columns), with a ragged last row group and
+    ragged last slices."""
     x_bits = synth.make_x(300 + M, M, K, max(1, K // 100), 20.0)
     x_bits[5] = 0                                 # an all-zero token
     V = synth.make_lorc(300 + M, 8, K, 8)[1] if lorc else None
@@ -40,6 +43,18 @@ def test_act_quant_many_rows_kernel(M, K, lorc):
     assert np.array_equal(host(sx).view(np.uint32), sx_o.view(np.uint32))
     if lorc:
         assert np.abs(host(t) - t_o).max() <= 1e-4 * np.abs(t_o).max()
+
+
+def test_act_quant_many_rows_strided_input():
+    M, K = 517, 7168
+    x_bits = synth.make_x(77, M, K, 70, 20.0)
+    V = synth.make_lorc(77, 8, K, 8)[1]
+    wide = torch.full((M, K + 264), 1e30, dtype=torch.bfloat16, device=dev())
+    wide[:, :K] = to_bf16(x_bits)
+    q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
+    q, sx, t = binding.quantize_act_fp8(wide[:, :K], up(V))
+    assert np.array_equal(host(q), q_o) and np.array_equal(host(sx).view(np.uint32), sx_o.view(np.uint32))
+    assert np.abs(host(t) - t_o).max() <= 1e-4 * np.abs(t_o).max()
 
 
 def test_act_quant_edge_rows_and_strided_input():

@@ -8,7 +8,7 @@ import pytest
 
 from paper_2307_09782_b200 import binding
 
-SHAPES = [(1, 768, 768), (8, 28672, 7168), (16, 7168, 28672), (17, 4096, 4096), (32, 28672, 7168), (64, 129, 1024),
+SHAPES = [(1, 768, 768), (8192, 7296, 28672), (1120, 15488, 512), (8, 28672, 7168), (16, 7168, 28672), (17, 4096, 4096), (32, 28672, 7168), (64, 129, 1024),
           (100, 384, 512), (128, 28672, 7168), (128, 7168, 28672), (130, 384, 512), (192, 256, 512), (200, 300, 512),
           (300, 384, 512), (500, 640, 2048), (512, 28672, 7168), (512, 7168, 28672), (700, 1000, 1024),
           (1000, 15360, 512), (1120, 15360, 9216), (2048, 28672, 7168), (2048, 7168, 28672), (2048, 4096, 11008),
@@ -24,6 +24,14 @@ def raster(pos, m_tiles, n_tiles, m_group):
     return (g * m_group + within % gm) * n_tiles + within // gm
 
 
+def pair_raster(pp, m_tiles, n_pairs, m_group):
+    mg = max(1, m_group)
+    per_group = mg * n_pairs
+    g, within = divmod(pp, per_group)
+    gm = min(mg, m_tiles - g * mg)
+    return g * mg + within % gm, within // gm
+
+
 def units_of_cta(pl, c, kblocks):
     """(position, K block) units of CTA c, in order."""
     tiles = pl["m_tiles"] * pl["n_tiles"]
@@ -36,6 +44,14 @@ def units_of_cta(pl, c, kblocks):
 
     if pl["stream"]:
         return dealt(0)
+    if pl["pair"]:
+        # CTAs 2c and 2c + 1 share the token tile of every pair position c, c + pairs, ...; CTA 2c + h takes the
+        # channel tile 2 * pair + h.  Units are reported by tile index here, not by launch position.
+        pairs, (pair, half) = pl["ctas"] // 2, divmod(c, 2)
+        for pp in range(pair, pl["m_tiles"] * (pl["n_tiles"] // 2), pairs):
+            m_tile, n_pair = pair_raster(pp, pl["m_tiles"], pl["n_tiles"] // 2, pl["m_group"])
+            out += [(m_tile * pl["n_tiles"] + 2 * n_pair + half, kb) for kb in range(kblocks)]
+        return out
     if pl["persist"]:
         for pos in range(c, pl["tail_pos0"], pl["ctas"]):
             out += [(pos, kb) for kb in range(kblocks)]
@@ -92,9 +108,16 @@ def test_plan_tile_choices_of_the_block_scaled_kernel():
         [16, 16, 32, 64, 128, 192, 256]
     assert binding.linear_plan(512, 28672, 7168, "M2", "mx")["bm"] == 192
     assert binding.linear_plan(8192, 28672, 7168, "M2", "mx")["bm"] == 224
-    assert binding.linear_plan(8192, 7168, 28672, "M2", "mx")["bm"] == 256
+    # many tokens, an even number of channel tiles: CTA pairs on whole tiles, the tile width with the fewest
+    # rounds x width (37 x 28 pair positions of 224 tokens are 14 whole rounds of 74 pairs)
     p = binding.linear_plan(8192, 7168, 28672, "M2", "mx")
-    assert p["persist"] == 1 and p["tail_pos0"] == (32 * 56) // p["ctas"] * p["ctas"]   # 12 whole rounds
+    if p["sms"] == 148:
+        assert p["pair"] == 1 and p["persist"] == 1 and p["bm"] == 224 and p["ctas"] == 148 and p["partial_floats"] == 0
+    # an odd number of channel tiles: single CTAs, whole rounds of whole tiles and a dealt-out last round
+    p = binding.linear_plan(8192, 7168 + 128, 28672, "M2", "mx")
+    assert p["pair"] == 0 and p["persist"] == 1 and p["bm"] == 256
+    assert p["tail_pos0"] == (32 * 57) // p["ctas"] * p["ctas"]   # 12 whole rounds
+    assert binding.linear_plan(8192, 28672, 7168, "none", "mx")["pair"] == 0
     # unconstrained scales: the running sums of a tile live in registers, so its token tiles stop at 128
     assert [binding.linear_plan(M, 4096, 4096, "none", "mx")["bm"] for M in (16, 100, 300, 2048)] == [16, 128, 128, 128]
     with pytest.raises(binding.ZqError):
