@@ -39,7 +39,7 @@ WORKLOAD = "opt30b"
 GROUP, MODE, RANK = 128, "M2", 8
 NOMINAL_FP8_TFLOPS = 4500.0  # public dense FP8 figure of the part, for context
 # DRAM bytes per launch from the ncu captures summarised under profiles/ (null when the kernel changed since)
-DOMINANT_TRAFFIC = 1575e6  # mean of the two M = 8192 launches (1502 MB and 1648 MB)
+DOMINANT_TRAFFIC = None
 DECODE_TRAFFIC = 114.8e6   # 7168 -> 28672 at 8 tokens
 # LLaMA-7B-shaped rows outside the timed step: (scale mode, weight layout)
 EXTRA_LLAMA7B = (("none", "cast"), ("none", "mx"), ("M2", "mx"))
@@ -445,9 +445,10 @@ def run_ours(args):
         per_layer_us.append(statistics.mean(events[s][b][1].elapsed_time(events[s][b][2]) for s in range(n_sw)) * 1e3)
     bound = "tensor" if Mmax >= 512 else "hbm"
     kfam = "w4a8_mx_gemm_kernel" if args.layout == "mx" else "w4a8_gemm_kernel"
-    bms = {li: binding.linear_plan(Mmax, layers[li]["N"], layers[li]["K"], mode, args.layout)["bm"] for li in big_layers}
-    kname = ", ".join(f"{kfam}<{bms[li]}> ({layers[li]['K']}->{layers[li]['N']}, {per_layer_us[b]:.1f} us)"
-                      for b, li in enumerate(big_layers))
+    plans = {li: binding.linear_plan(Mmax, layers[li]["N"], layers[li]["K"], mode, args.layout) for li in big_layers}
+    kname = ", ".join(
+        f"{'w4a8_mx_pair_gemm_kernel' if plans[li]['pair'] else kfam}<{plans[li]['bm']}> "
+        f"({layers[li]['K']}->{layers[li]['N']}, {per_layer_us[b]:.1f} us)" for b, li in enumerate(big_layers))
     big_us = statistics.mean(per_layer_us)
     if bound == "tensor":
         big_flops = statistics.mean(2.0 * Mmax * layers[li]["N"] * layers[li]["K"] for li in big_layers)

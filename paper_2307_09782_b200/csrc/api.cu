@@ -52,6 +52,10 @@ size_t max_partial_floats(int64_t M, int64_t N, int64_t K) {
       const GemmPlan pl = plan_gemm(m, N, K, (variant == 0 || variant == 3) ? ZQ_SCALE_NONE : ZQ_SCALE_M1,
                                     variant >= 2 ? ZQ_WEIGHTS_MX : ZQ_WEIGHTS_CAST);
       if (pl.partial_floats > best) best = pl.partial_floats;
+      if (pl.pair) {  // a bf16 y takes the single-CTA plan
+        const GemmPlan ps = plan_gemm(m, N, K, ZQ_SCALE_M1, ZQ_WEIGHTS_MX, false);
+        if (ps.partial_floats > best) best = ps.partial_floats;
+      }
     }
   };
   const int64_t small[10] = {16, 32, 64, 128, 129, 192, 193, 224, 256, M};

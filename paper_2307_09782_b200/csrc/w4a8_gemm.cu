@@ -622,7 +622,7 @@ int sm_count() {
   return n;
 }
 
-GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
+GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout, bool allow_pair) {
   GemmPlan pl{};
   const bool mx = layout_is_mx(layout);
   // mode none keeps a tile's running sums in registers: 64 tokens in the kernel that casts, 128 in the block-scaled one
@@ -649,6 +649,57 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
   const int64_t tiles = static_cast<int64_t>(pl.m_tiles) * pl.n_tiles;
   const int kblocks = static_cast<int>(K / kBlockK);
   if (tiles <= 0 || kblocks <= 0) return pl;  // nothing to do: an empty plan (ctas == 0)
+  if (wide && allow_pair && bm >= 192 && pl.n_tiles % 2 == 0 && sm_count() >= 2 && tiles <= kWsMaxTiles) {
+    // CTA pairs: the two CTAs of a cluster share each token tile (192 or 224 tokens, two accumulators) and
+    // take two neighbouring channel tiles.  Work is counted in units of one K block of one pair position
+    // (token tile x channel-tile pair) and partitioned among the pairs like the single CTAs' below: whole
+    // positions in whole rounds where there are at least four rounds, the rest (or everything) dealt out as
+    // contiguous unit ranges.  Taken when its padded token columns are at most 15 % more than the single
+    // CTAs' (the pairs run about 20 % faster).
+    const int64_t pairs = sm_count() / 2, np = pl.n_tiles / 2;
+    int best_bm = 0;
+    int64_t best_cols = 0;
+    for (const int cand : {224, 192}) {  // 224 tokens move fewer shared-memory bytes per flop: worth 5 % of padding
+      const int64_t cols = ((M + cand - 1) / cand) * cand;
+      if (best_bm == 0 || cols * 21 < best_cols * 20) {
+        best_bm = cand;
+        best_cols = cols;
+      }
+    }
+    if (best_cols * 100 <= static_cast<int64_t>(pl.m_tiles) * bm * 115) {
+      GemmPlan pp{};
+      pp.pair = 1;
+      pp.bm = best_bm;
+      pp.m_tiles = static_cast<int>(best_cols / best_bm);
+      pp.n_tiles = pl.n_tiles;
+      pp.splits = 1;
+      pp.kb_per_split = kblocks;
+      const int64_t positions = pp.m_tiles * np, punits = positions * kblocks;
+      if (pp.m_tiles > 1) {
+        const int64_t fit = (int64_t(32) << 20) / (static_cast<int64_t>(best_bm) * K);
+        pp.m_group = static_cast<int>(fit < 1 ? 1 : (fit > 8 ? 8 : fit));
+      }
+      if (positions >= 4 * pairs) {
+        pp.persist = 1;
+        pp.ctas = static_cast<int>(2 * pairs);
+        int64_t tail = positions % pairs;
+        if ((pairs - tail) * kblocks < 60 * pairs) tail = 0;  // too little to gain: leave the last round uneven
+        pp.tail_pos0 = static_cast<int>(positions - tail);
+        pp.base = static_cast<int>(tail * kblocks / pairs);
+        pp.rem = static_cast<int>(tail * kblocks % pairs);
+        return pp;
+      }
+      if (punits >= 8 && punits < (int64_t(1) << 30)) {
+        int64_t g = pairs < punits / 4 ? pairs : punits / 4;
+        if (g < 1) g = 1;
+        pp.stream = 1;
+        pp.ctas = static_cast<int>(2 * g);
+        pp.base = static_cast<int>(punits / g);
+        pp.rem = static_cast<int>(punits % g);
+        return pp;
+      }
+    }
+  }
   // CTAs per SM the kernel family is sized for at this tile
   // (the block-scaled kernel: always one; its launches with shared tiles are cooperative, and a cooperative
   // launch of a kernel that allocates tensor memory is given one CTA per SM)
@@ -681,36 +732,6 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout) {
     pl.base = static_cast<int>(tail_tiles * kblocks / g);
     pl.rem = static_cast<int>(tail_tiles * kblocks % g);
     pl.partial_floats = tail_tiles > 0 ? 2 * static_cast<size_t>(g) * bm * kTileN : 0;
-    if (wide && bm >= 192 && pl.n_tiles % 2 == 0 && sm_count() >= 2) {
-      // CTA pairs (two CTAs share each token tile and take two neighbouring channel tiles): whole tiles only,
-      // pair c walks the pair positions c, c + pairs, ...  The token tile (224 or 192 tokens: two accumulators)
-      // is the one with the fewest rounds x width; taken unless its last, incomplete round would cost more
-      // than the pairs save.
-      const int64_t pairs = sm_count() / 2, np = pl.n_tiles / 2;
-      int best_bm = 0;
-      int64_t best_cost = 0;
-      for (const int cand : {224, 192}) {
-        const int64_t mt = (M + cand - 1) / cand;
-        const int64_t cost = ((mt * np + pairs - 1) / pairs) * cand;
-        if (best_bm == 0 || cost < best_cost) {
-          best_bm = cand;
-          best_cost = cost;
-        }
-      }
-      const double single_cost = static_cast<double>(tiles) * bm / sm_count();
-      if (static_cast<double>(best_cost) <= 1.10 * single_cost) {
-        pl.pair = 1;
-        pl.bm = best_bm;
-        pl.m_tiles = static_cast<int>((M + best_bm - 1) / best_bm);
-        const int64_t positions = pl.m_tiles * np;
-        pl.ctas = static_cast<int>(2 * (positions < pairs ? positions : pairs));
-        pl.tail_pos0 = pl.m_tiles * pl.n_tiles;
-        pl.base = pl.rem = 0;
-        pl.partial_floats = 0;
-        const int64_t fit = (int64_t(32) << 20) / (static_cast<int64_t>(best_bm) * K);
-        pl.m_group = pl.m_tiles > 1 ? static_cast<int>(fit < 1 ? 1 : (fit > 8 ? 8 : fit)) : 0;
-      }
-    }
     return pl;
   }
   if ((mx || (mode != ZQ_SCALE_NONE && bm == 16 && pl.m_tiles == 1)) && tiles <= kWsMaxTiles && units >= 8 &&

@@ -54,7 +54,6 @@ struct Params {
                  // up to position tail_pos0; the tiles from there on are dealt out as unit ranges like stream == 1
   int tail_pos0;
   int dealt0;    // first unit of the units that are dealt out as ranges (0 when stream == 1)
-  int pair_end;  // CTA-pair kernel: pair positions [0, pair_end) are its work (see pair_tile)
   int m_group;   // the launch order runs through groups of this many token tiles (see raster_tile)
   int atomic_y;  // streaming launch with FP32 y: CTAs that share a tile add their share into a zeroed y
   int handover;  // cooperative launch: shared FP32 tiles are handed over through per-tile flags (one CTA stores,

@@ -105,15 +105,19 @@ struct MxCfg {
 struct Segments {
   int us, u1;
   int idx, step;
-  bool persist;
-  __device__ __forceinline__ explicit Segments(const Params& p) {
+  bool persist, pairs;
+  // `worker` of `workers`: a CTA of the grid, or (CTA-pair kernel) a pair of the grid's pairs, whose positions
+  // are pair positions (see pair_tile) and are handed back as they are
+  __device__ __forceinline__ explicit Segments(const Params& p, int worker = static_cast<int>(blockIdx.x),
+                                               int workers = static_cast<int>(gridDim.x), bool pair_positions = false) {
     persist = p.persist != 0;
-    idx = static_cast<int>(blockIdx.x);
-    step = static_cast<int>(gridDim.x);
+    pairs = pair_positions;
+    idx = worker;
+    step = workers;
     us = u1 = 0;
     if (p.stream || persist) {
-      us = p.dealt0 + range_start(p, blockIdx.x);
-      u1 = p.dealt0 + range_start(p, blockIdx.x + 1);
+      us = p.dealt0 + range_start(p, worker);
+      u1 = p.dealt0 + range_start(p, worker + 1);
     } else {
       const int z = blockIdx.x / p.tiles, pos = blockIdx.x % p.tiles;
       us = pos * p.kblocks + z * p.kb_per_split;
@@ -138,7 +142,7 @@ struct Segments {
       nkb = ue - us;
       us = ue;
     }
-    tile = raster_tile(p, pos);
+    tile = pairs ? pos : raster_tile(p, pos);
     return true;
   }
 };
@@ -794,7 +798,10 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
 // the leader's barrier), the leader's MMA thread issues for both, its commits release the stages and publish
 // the accumulators in both CTAs, and each CTA's epilogue warps finish their own 128 channels.  The token bytes
 // per CTA and K block are halved.
-// Whole output tiles only: pair `c` of the grid walks pair positions c, c + pairs, ... below p.pair_end.
+// Work partition: as above with pairs in place of CTAs and pair positions (token tile x two neighbouring channel
+// tiles) in place of tiles: whole positions in whole rounds, the rest dealt out as contiguous unit ranges; a
+// position shared by several pairs is handed over through per-CTA flags (FP32 y only): the last contributor in K
+// order stores, the others wait for its flag and add.  All pairs of the grid fit the device at once.
 template <int BM, bool W8>
 struct PairCfg {
   static constexpr int kThreads = 192;
@@ -915,12 +922,14 @@ w4a8_mx_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
       int s = 0, issued = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int pos = pair; ok && pos < p.pair_end; pos += pairs) {
+      Segments sg(p, pair, pairs, true);
+      int pos, tile_unused, kb0, nkb;
+      while (ok && sg.next(p, pos, tile_unused, kb0, nkb)) {
         int m_tile, n_pair;
         pair_tile(p, pos, m_tile, n_pair);
         const int nt = 2 * n_pair + static_cast<int>(rank);
         const int row0 = m_tile * BM + static_cast<int>(rank) * C::kHalf;
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        for (int kb = kb0; kb < kb0 + nkb; ++kb) {
           if (issued >= C::NS && !mbar_wait(&empty[s], ph ^ 1, s_abort)) {
             if (issuer) raise_error(p, s_abort, kErrProducer);
             ok = false;
@@ -959,7 +968,9 @@ w4a8_mx_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
       int s = 0, seg = 0;
       uint32_t ph = 0;
       bool failed = false;
-      for (int pos = pair; !failed && pos < p.pair_end; pos += pairs, ++seg) {
+      Segments sg(p, pair, pairs, true);
+      int pos, tile_unused, kb0, nkb;
+      for (; !failed && sg.next(p, pos, tile_unused, kb0, nkb); ++seg) {
         const int buf = seg % C::NB;
         if (seg >= C::NB && !mbar_wait(&acc_empty[buf], ((seg / C::NB) - 1) & 1, s_abort)) {
           failed = true;
@@ -967,7 +978,7 @@ w4a8_mx_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + buf * BM;
-        for (int kb = 0; kb < p.kblocks && !failed; ++kb) {
+        for (int kb = 0; kb < nkb && !failed; ++kb) {
           if (!mbar_wait(&full[s], ph, s_abort)) {
             failed = true;
             break;
@@ -986,7 +997,7 @@ w4a8_mx_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
                                  tmem_sfb, (kb > 0 || k > 0) ? 1u : 0u);
             }
             umma_commit_pair(&empty[s]);
-            if (kb + 1 == p.kblocks) umma_commit_pair(&acc_full[buf]);
+            if (kb + 1 == nkb) umma_commit_pair(&acc_full[buf]);
           }
           __syncwarp();
           if (++s == C::NS) {
@@ -1015,7 +1026,9 @@ w4a8_mx_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
     int m0_loaded = -1;
     pdl_wait();  // sx, t and y may still be in use by the kernel ahead in the stream
     int seg = 0;
-    for (int pos = pair; pos < p.pair_end; pos += pairs, ++seg) {
+    Segments sg(p, pair, pairs, true);
+    int pos, tile_unused, kb0, nkb;
+    for (; sg.next(p, pos, tile_unused, kb0, nkb); ++seg) {
       int m_tile, n_pair;
       pair_tile(p, pos, m_tile, n_pair);
       const int m0 = m_tile * BM;
@@ -1054,17 +1067,59 @@ w4a8_mx_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
         failed = true;
       }
       tc_fence_after_sync();
-      if (!failed) {
-        float nxt[EC];
-        tmem_ld_issue<EC>(t_lane, nxt);
+      if (nkb == p.kblocks) {
+        if (!failed) {
+          float nxt[EC];
+          tmem_ld_issue<EC>(t_lane, nxt);
 #pragma unroll 1
-        for (int c = 0; c < BM; c += EC) {
-          float v[EC];
-          tmem_ld_wait_regs<EC>(nxt);
+          for (int c = 0; c < BM; c += EC) {
+            float v[EC];
+            tmem_ld_wait_regs<EC>(nxt);
 #pragma unroll
-          for (int e = 0; e < EC; ++e) v[e] = nxt[e];
-          if (c + EC < BM) tmem_ld_issue<EC>(t_lane + c + EC, nxt);
-          if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t);
+            for (int e = 0; e < EC; ++e) v[e] = nxt[e];
+            if (c + EC < BM) tmem_ld_issue<EC>(t_lane + c + EC, nxt);
+            if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t);
+          }
+        }
+      } else {
+        // Several pairs share this position (FP32 y).  Its last contributor in K order meets it as the first
+        // segment of its range, i.e. early: it STORES its share (with the LoRC term) and raises this CTA's flag of
+        // the position.  The others meet it at the end of their ranges: they wait for the flag and ADD their
+        // shares.  The adder that finds all others done leaves the flag at zero for the next call.
+        int first, count;
+        contributors(p, pos, &first, &count);
+        const bool storer = pair == first + count - 1;
+        int* flag = p.counters + 2 * pos + static_cast<int>(rank);
+        if (!storer) {
+          if (threadIdx.x == 0) {
+            const uint64_t t0 = global_timer_ns();
+            bool ok = false;
+            for (uint32_t spin = 0; spin < kSpinLimit && !ok; ++spin) {
+              ok = *reinterpret_cast<volatile int*>(flag) != 0 || *s_abort != 0;
+              if (!ok && (spin & 63u) == 63u && global_timer_ns() - t0 > kWaitLimitNs) break;
+            }
+            if (!ok) raise_error(p, s_abort, kErrHandover);
+            __threadfence();
+          }
+          named_bar_sync(2, C::kEpiThreads);
+          if (*s_abort) failed = true;
+        }
+        if (!failed) {
+#pragma unroll 1
+          for (int c = 0; c < BM; c += EC) {
+            float v[EC];
+            tmem_ld_cols<EC>(t_lane + c, v);
+            if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t, !storer, storer);
+          }
+        }
+        __threadfence();  // this thread's stores / adds are performed before the flag moves
+        named_bar_sync(2, C::kEpiThreads);
+        if (threadIdx.x == 0 && !*s_abort) {
+          if (storer) {
+            atomicExch(flag, 1);
+          } else if (atomicAdd(flag, 1) == count - 1) {
+            atomicExch(flag, 0);  // storer + all other adders were counted before this one
+          }
         }
       }
       // this warp has read the buffer: tell the leader's MMA thread
@@ -1210,10 +1265,9 @@ int launch_pair_cfg(const GemmArgs& a, const GemmPlan& plan, Params p, cudaStrea
       !make_token_map(&tm_q, a.q, static_cast<uint64_t>(a.K), static_cast<uint64_t>(a.M), C::kHalf, 1) ||
       !make_scale_map(&tm_sf, a.codes, static_cast<uint64_t>(plan.n_tiles), static_cast<uint64_t>(p.kblocks), W8))
     return ZQ_ERR_CUDA;
-  const int positions = plan.m_tiles * (plan.n_tiles / 2);
-  p.pair_end = positions;
-  const int pairs = positions < max_pairs ? positions : max_pairs;
-  const cudaError_t err = launch_chained(kernel, dim3(2 * pairs), dim3(C::kThreads), C::kSmemBytes, st, false, tm_w,
+  // shared positions are handed over by flags between pairs that must all be running: the plan's grid has to fit
+  if (plan.ctas / 2 > max_pairs) return kPairNotTaken;
+  const cudaError_t err = launch_chained(kernel, dim3(plan.ctas), dim3(C::kThreads), C::kSmemBytes, st, false, tm_w,
                                          tm_q, tm_sf, p);
   count_launch();
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
@@ -1222,7 +1276,23 @@ int launch_pair_cfg(const GemmArgs& a, const GemmPlan& plan, Params p, cudaStrea
 }  // namespace
 
 int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
-  const GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode, ZQ_WEIGHTS_MX);
+  GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode, ZQ_WEIGHTS_MX);
+  if (plan.pair) {
+    // positions shared between pairs are added into an FP32 y; a bf16 y takes the single CTAs, and so does a
+    // device that grants the pair kernel fewer pairs than planned
+    const bool shared = plan.stream || plan.tail_pos0 < plan.m_tiles * (plan.n_tiles / 2);
+    int e = kPairNotTaken;
+    if (!(shared && a.ydt != ZQ_OUT_F32)) {
+      Params pp = make_params(a, plan);
+      const bool w8p = a.layout == ZQ_WEIGHTS_MX_FP8;
+      switch (plan.bm) {
+        case 192: e = w8p ? launch_pair_cfg<192, true>(a, plan, pp, st) : launch_pair_cfg<192, false>(a, plan, pp, st); break;
+        case 224: e = w8p ? launch_pair_cfg<224, true>(a, plan, pp, st) : launch_pair_cfg<224, false>(a, plan, pp, st); break;
+      }
+    }
+    if (e != kPairNotTaken) return e;
+    plan = plan_gemm(a.M, a.N, a.K, a.mode, ZQ_WEIGHTS_MX, false);
+  }
   if (plan.partial_floats > a.partial_floats) return ZQ_ERR_WORKSPACE;
   Params p = make_params(a, plan);
   const bool w8 = a.layout == ZQ_WEIGHTS_MX_FP8;
@@ -1244,16 +1314,6 @@ int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
       case 128: return launch_mx_cfg<128, false, false, true>(a, plan, p, st);
     }
     return ZQ_ERR_SHAPE;
-  }
-  if (plan.pair) {
-    // many tokens, whole tiles: CTA pairs sharing each token tile
-    int e = kPairNotTaken;
-    switch (plan.bm) {
-      case 192: e = w8 ? launch_pair_cfg<192, true>(a, plan, p, st) : launch_pair_cfg<192, false>(a, plan, p, st); break;
-      case 224: e = w8 ? launch_pair_cfg<224, true>(a, plan, p, st) : launch_pair_cfg<224, false>(a, plan, p, st); break;
-    }
-    if (e != kPairNotTaken) return e;
-    return ZQ_ERR_CUDA;  // the device grants this kernel no CTA pair
   }
 #define ZQ_MX_CASE(BM_) \
   case BM_: return w8 ? launch_mx_cfg<BM_, true, false, false>(a, plan, p, st) : launch_mx_cfg<BM_, false, false, false>(a, plan, p, st)

@@ -116,10 +116,13 @@ struct GemmPlan {
   int kb_per_split;  // stream == 0: 128-element K blocks per split
   int base, rem;     // stream == 1: units per CTA (the first `rem` CTAs take one more)
   int m_group;       // the launch order runs through groups of this many token tiles (0 or 1: along N only)
-  int pair;          // 1 (with persist): CTA pairs; pair c = CTAs 2c, 2c + 1 walks pair positions c, c + ctas / 2, ...
+  int pair;          // 1: CTA pairs (CTAs 2c, 2c + 1 = pair c).  Positions, tail_pos0 and the units of base / rem then
+                     //    count pair positions (token tile x two neighbouring channel tiles) and pairs, not tiles and CTAs
   size_t partial_floats;
 };
-GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout);
+// allow_pair = false: the plan for single CTAs (shared output tiles of a bf16 y go through the workspace, which
+// the pair kernel does not do).
+GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout, bool allow_pair = true);
 int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st);           // ZQ_WEIGHTS_CAST
 int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st);        // ZQ_WEIGHTS_MX
 int sm_count();

@@ -125,6 +125,36 @@ def test_linear_cta_pairs(M, N, K, r, mode, layout, out_dtype):
     check_linear(x_bits, W, U, V, 128, mode, layout=layout, rows=rows, out_dtype=out_dtype)
 
 
+@pytest.mark.parametrize("M,N,K,out_dtype", [
+    (500, 128 * 6, 2048, torch.float32),      # 3 x 3 positions x 16 K blocks dealt out as ranges: most positions shared
+    (500, 128 * 6, 2048, torch.bfloat16),     # bf16 y with shared tiles: the single CTAs take it (workspace partial sums)
+    (192, 128 * 150, 512, torch.float32),     # one row of 192-token tiles
+    (1120, 128 * 120, 9216, torch.float32),   # four whole rounds, then four positions dealt out to all 74 pairs
+])
+def test_linear_cta_pairs_shared_positions(M, N, K, out_dtype):
+    """Pair positions whose K range is split between pairs: the last contributor stores, the others wait for its
+    flag and add; a second call on the same workspace must find the flags as the first one did."""
+    pl = binding.linear_plan(M, N, K, "M2", MX)
+    assert pl["pair"] == 1 and (pl["stream"] == 1 or pl["tail_pos0"] < pl["m_tiles"] * pl["n_tiles"] // 2)
+    x_bits, W, U, V = _layer(93, M, N, K, 8)
+    bm = pl["bm"]
+    rows = sorted({0, bm // 2 - 1, bm // 2, bm - 1, min(bm, M - 1), M // 2, M - 2, M - 1})
+    q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
+    c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, 128, "M2")
+    y_o = oracle.w4a8_linear(q_o, sx_o, c_o, sh_o, sc_o, 128, "M2", U, t_o, rows=rows)
+    pw = binding.pack_weight_fp4(up(W), 128, "M2", MX)
+    ws = binding.make_workspace(binding.linear_workspace_bytes(M, N, K, 8))
+    q, sx, t = binding.quantize_act_fp8(to_bf16(x_bits), up(V))
+    for _ in range(3):
+        y = binding.w4a8_linear(pw, q=q, sx=sx, t=t, U=up(U), out_dtype=out_dtype, workspace=ws)
+        assert binding.device_status(ws) == (0, 0)
+        yh = host(y.float()).astype(np.float64)[rows]
+        tol = TOL_REL * np.abs(y_o).max()
+        if out_dtype == torch.bfloat16:
+            tol = tol + 2.0 ** (np.floor(np.log2(np.maximum(np.abs(y_o), 1e-30))) - 7)
+        assert np.all(np.abs(yh - y_o) <= tol)
+
+
 def test_linear_cta_pairs_fp8_weights():
     M, N, K, r = 1120, 128 * 120, 384, 8
     assert binding.linear_plan(M, N, K, "M2", binding.WEIGHTS_MX_FP8)["pair"] == 1

@@ -42,16 +42,28 @@ def units_of_cta(pl, c, kblocks):
         end = first_unit + (c + 1) * pl["base"] + min(c + 1, pl["rem"])
         return [(u // kblocks, u % kblocks) for u in range(start, end)]
 
+    if pl["pair"]:
+        # CTAs 2c and 2c + 1 are pair c: they share the token tile of each of the pair's positions and CTA 2c + h
+        # takes the channel tile 2 * n_pair + h.  Positions, tail_pos0 and base / rem count pair positions and pairs.
+        # Units are reported by tile index here, not by launch position.
+        pairs, (pair, half) = pl["ctas"] // 2, divmod(c, 2)
+
+        def dealt_pair(first_unit):
+            start = first_unit + pair * pl["base"] + min(pair, pl["rem"])
+            end = first_unit + (pair + 1) * pl["base"] + min(pair + 1, pl["rem"])
+            return [(u // kblocks, u % kblocks) for u in range(start, end)]
+
+        if pl["stream"]:
+            us = dealt_pair(0)
+        else:
+            us = [(pp, kb) for pp in range(pair, pl["tail_pos0"], pairs) for kb in range(kblocks)]
+            us += dealt_pair(pl["tail_pos0"] * kblocks)
+        for pp, kb in us:
+            m_tile, n_pair = pair_raster(pp, pl["m_tiles"], pl["n_tiles"] // 2, pl["m_group"])
+            out.append((m_tile * pl["n_tiles"] + 2 * n_pair + half, kb))
+        return out
     if pl["stream"]:
         return dealt(0)
-    if pl["pair"]:
-        # CTAs 2c and 2c + 1 share the token tile of every pair position c, c + pairs, ...; CTA 2c + h takes the
-        # channel tile 2 * pair + h.  Units are reported by tile index here, not by launch position.
-        pairs, (pair, half) = pl["ctas"] // 2, divmod(c, 2)
-        for pp in range(pair, pl["m_tiles"] * (pl["n_tiles"] // 2), pairs):
-            m_tile, n_pair = pair_raster(pp, pl["m_tiles"], pl["n_tiles"] // 2, pl["m_group"])
-            out += [(m_tile * pl["n_tiles"] + 2 * n_pair + half, kb) for kb in range(kblocks)]
-        return out
     if pl["persist"]:
         for pos in range(c, pl["tail_pos0"], pl["ctas"]):
             out += [(pos, kb) for kb in range(kblocks)]
@@ -93,7 +105,9 @@ def test_plan_covers_every_unit_once(M, N, K, layout, mode):
     shared = sharers > 1
     if shared.any():
         assert tiles <= 16384, "shared tiles are counted in the workspace's tile counters"
-        if pl["stream"] or pl["persist"]:
+        if pl["pair"]:
+            assert max_partial_tiles <= 2   # shared tiles are handed over by flags into an FP32 y: no scratch
+        elif pl["stream"] or pl["persist"]:
             assert max_partial_tiles <= 2
             assert pl["partial_floats"] >= 2 * ctas * bm * 128
         else:
@@ -106,13 +120,19 @@ def test_plan_tile_choices_of_the_block_scaled_kernel():
     # one row of tiles up to 256 tokens, then 192 / 224 (two accumulators) or 256 (long rows, many tiles)
     assert [binding.linear_plan(M, 28672, 7168, "M2", "mx")["bm"] for M in (1, 16, 17, 64, 100, 192, 256)] == \
         [16, 16, 32, 64, 128, 192, 256]
-    assert binding.linear_plan(512, 28672, 7168, "M2", "mx")["bm"] == 192
+    assert binding.linear_plan(512, 28672 + 128, 7168, "M2", "mx")["bm"] == 192
     assert binding.linear_plan(8192, 28672, 7168, "M2", "mx")["bm"] == 224
     # many tokens, an even number of channel tiles: CTA pairs on whole tiles, the tile width with the fewest
     # rounds x width (37 x 28 pair positions of 224 tokens are 14 whole rounds of 74 pairs)
     p = binding.linear_plan(8192, 7168, 28672, "M2", "mx")
     if p["sms"] == 148:
         assert p["pair"] == 1 and p["persist"] == 1 and p["bm"] == 224 and p["ctas"] == 148 and p["partial_floats"] == 0
+        assert p["tail_pos0"] == 37 * 28                      # 14 whole rounds, nothing left to deal out
+        p = binding.linear_plan(2048, 7168, 28672, "M2", "mx")     # 11 x 28 positions: 4 rounds, 12 positions dealt out
+        assert p["pair"] == 1 and p["persist"] == 1 and p["bm"] == 192 and p["tail_pos0"] == 4 * 74
+        assert p["base"] * 74 + p["rem"] == 12 * 224
+        p = binding.linear_plan(512, 7168, 28672, "M2", "mx")      # 3 x 28 positions: fewer than four rounds, all dealt out
+        assert p["pair"] == 1 and p["stream"] == 1 and p["bm"] == 192 and p["base"] * 74 + p["rem"] == 84 * 224
     # an odd number of channel tiles: single CTAs, whole rounds of whole tiles and a dealt-out last round
     p = binding.linear_plan(8192, 7168 + 128, 28672, "M2", "mx")
     assert p["pair"] == 0 and p["persist"] == 1 and p["bm"] == 256
