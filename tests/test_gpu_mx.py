@@ -282,10 +282,10 @@ def test_host_buffer_entry_point_in_row_chunks(layout):
     assert np.abs(yh.numpy() - y_d).max() <= 1e-5 * np.abs(y_d).max()
 
 
-@pytest.mark.parametrize("M,N,K", [(8, 640, 4096), (40, 200, 2048), (300, 384, 512), (1120, 15360, 256)])
+@pytest.mark.parametrize("M,N,K", [(8, 640, 4096), (40, 200, 2048), (300, 384, 512), (1120, 15360, 256), (500, 768, 2048)])
 def test_strided_output_leaves_the_gaps_alone(M, N, K):
-    # y with a leading dimension larger than N: shared tiles (store / flag / add), whole tiles and the
-    # persistent launch must write exactly the M x N block
+    # y with a leading dimension larger than N: shared tiles (store / flag / add), whole tiles, the persistent
+    # launch and the CTA pairs (whole and shared positions) must write exactly the M x N block
     x_bits, W, U, V = _layer(98, M, N, K, 8)
     pw = binding.pack_weight_fp4(up(W), 128, "M2", MX)
     q, sx, t = binding.quantize_act_fp8(to_bf16(x_bits), up(V))
