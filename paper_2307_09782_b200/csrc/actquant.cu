@@ -7,6 +7,8 @@
 #include <cooperative_groups.h>
 #include <cuda_fp16.h>
 
+#include <mutex>
+
 #include "act_cast.cuh"
 #include "zq_common.cuh"
 
@@ -244,6 +246,184 @@ act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec
   }
 }
 
+// ---- a few hundred tokens: eight rows per cluster, the rows held in shared memory --------------------
+// Between the two kernels around it: too few tokens for the eight-row CTAs above to fill the device, too many
+// for a cluster per row below, whose every cluster reads all of V.  Here a cluster of C CTAs takes eight rows
+// and each CTA a slice of at most 4096 columns of them, which one thread fetches into shared memory with
+// eight bulk copies: the rows are read from HBM exactly once, V once per eight rows, absmax and the LoRC sums
+// meet through distributed shared memory, and the cast reads shared memory.
+// The wait for the copies is bounded like every wait of this library; the quantizer has no status word, so a
+// wait that ran out shows as sx = +inf (and no codes written) for the rows concerned.
+constexpr int kTileThreads = 384;
+constexpr int kTileWarps = kTileThreads / 32;
+constexpr int kTileMaxVec = 512;  // 16-byte vectors (8 elements) of a row one CTA holds
+constexpr int kTilePadVec = 4;    // row pitch = slice + 64 bytes: the two rows of a quarter-warp hit disjoint banks
+constexpr int kTileMaxCluster = 8;
+constexpr int kTileMinTokens = 32;
+
+template <bool HAS_V, int C>
+__global__ void __cluster_dims__(C, 1, 1) __launch_bounds__(kTileThreads, 3)
+act_quant_tile_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec, int vec_per_cta,
+                      uint8_t* __restrict__ q, float* __restrict__ sx, const uint4* __restrict__ V,
+                      float* __restrict__ t) {
+  namespace cg = cooperative_groups;
+  extern __shared__ uint4 s_x[];  // [kRows][vec_per_cta + kTilePadVec]
+  __shared__ float s_amax[kTileWarps][kRows];
+  __shared__ float s_acc[kTileWarps][kRows * 8];
+  __shared__ float s_part_amax[kRows];   // this CTA's partial absmax per row (read by the whole cluster)
+  __shared__ float s_part_t[kRows * 8];  // this CTA's partial LoRC sums [token][j] (read by rank 0)
+  __shared__ float s_inv[kRows];
+  __shared__ __align__(8) uint64_t s_bar;
+  __shared__ int s_abort;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = C == 1 ? 0 : static_cast<int>(cluster.block_rank());
+  const int m0 = blockIdx.y * kRows;
+  const int nrows = min(kRows, M - m0);
+  const int nvec = K / 8;
+  const int v_begin = rank * vec_per_cta;
+  const int nv = max(0, min(nvec, v_begin + vec_per_cta) - v_begin);  // vectors of this CTA's slice
+  const int pitch = vec_per_cta + kTilePadVec;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, tig = lane & 3;  // g: token row of this lane, and its row of V
+  const uint4* xr = x + static_cast<int64_t>(m0) * ldx_vec + v_begin;
+  if (tid == 0) {
+    mbar_init(&s_bar, 1);
+    s_abort = 0;
+    fence_mbar_init();
+  }
+  pdl_launch_dependents();
+  __syncthreads();
+  if (tid == 0 && nv > 0) {
+    pdl_wait();  // x may be the output of the kernel before this one
+    mbar_arrive_expect_tx(&s_bar, static_cast<uint32_t>(nrows) * nv * 16u);
+    for (int r = 0; r < nrows; ++r)
+      bulk_load(s_x + r * pitch, xr + static_cast<int64_t>(r) * ldx_vec, nv * 16u, &s_bar);
+  }
+  const uint4* vrow = V + static_cast<int64_t>(g) * nvec + v_begin;
+  const uint4* srow = s_x + g * pitch;
+  const bool row_ok = g < nrows;
+
+  float amax = 0.0f;
+  float d[4] = {0.0f, 0.0f, 0.0f, 0.0f};  // d[0], d[1]: t[token 2 tig, 2 tig + 1][j = g] over this warp's columns
+  bool arrived = false;
+  for (int base = warp * kRowsUnroll * 4; base < nv; base += kTileWarps * kRowsUnroll * 4) {
+    uint4 vv[kRowsUnroll];
+    if (HAS_V) {  // V does not depend on the copies: its loads go out before the wait
+#pragma unroll
+      for (int i = 0; i < kRowsUnroll; ++i) {
+        const int u = base + i * 4 + tig;
+        vv[i] = u < nv ? __ldg(vrow + u) : make_uint4(0, 0, 0, 0);
+      }
+    }
+    if (!arrived) {
+      if (!mbar_wait(&s_bar, 0, &s_abort)) s_abort = 1;
+      arrived = true;
+    }
+#pragma unroll
+    for (int i = 0; i < kRowsUnroll; ++i) {
+      const int u = base + i * 4 + tig;
+      const uint4 xv = (u < nv && row_ok) ? srow[u] : make_uint4(0, 0, 0, 0);
+      amax = absmax8(xv, amax);
+      if (HAS_V) {
+        const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+        const uint32_t vw[4] = {vv[i].x, vv[i].y, vv[i].z, vv[i].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __half2 h;
+          *reinterpret_cast<uint32_t*>(&h) = vw[e];
+          const float2 vf = __half22float2(h);
+          // elements 2e and 2e+1 of both 8-element pieces stand at MMA-K positions tig and tig + 4
+          mma_tf32_16x8x8(d, __float_as_uint(vf.x), __float_as_uint(vf.y), xw[e] << 16, xw[e] & 0xFFFF0000u);
+        }
+      }
+    }
+  }
+  if (!arrived && nv > 0 && !mbar_wait(&s_bar, 0, &s_abort)) s_abort = 1;  // the cast below reads the slice too
+  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+  if (tig == 0) s_amax[warp][g] = amax;
+  if (HAS_V) {
+    s_acc[warp][(2 * tig) * 8 + g] = d[0];  // [token][j]
+    s_acc[warp][(2 * tig + 1) * 8 + g] = d[1];
+  }
+  __syncthreads();
+  const bool failed = s_abort != 0;
+  if (tid < kRows) {
+    float a = s_amax[0][tid];
+    for (int w = 1; w < kTileWarps; ++w) a = fmaxf(a, s_amax[w][tid]);
+    s_part_amax[tid] = failed ? __int_as_float(0x7F800000) : a;
+  }
+  if (HAS_V && tid >= 64 && tid < 64 + kRows * 8) {
+    float v = 0.0f;
+    for (int w = 0; w < kTileWarps; ++w) v += s_acc[w][tid - 64];
+    s_part_t[tid - 64] = v;
+  }
+  if (C > 1) cluster.sync(); else __syncthreads();  // every CTA's partial results are written and visible
+  if (tid < kRows) {
+    float a = 0.0f;
+    if (C == 1) {
+      a = s_part_amax[tid];
+    } else {
+      for (int k = 0; k < C; ++k) a = fmaxf(a, cluster.map_shared_rank(s_part_amax, k)[tid]);
+    }
+    float s = 1.0f, inv = 1.0f;
+    if (a != 0.0f) {
+      s = __fdiv_rn(a, 448.0f);
+      inv = __fdiv_rn(448.0f, a);
+    }
+    s_inv[tid] = inv;
+    if (rank == 0 && tid < nrows) sx[m0 + tid] = s;
+  }
+  if (HAS_V && rank == 0 && tid >= 64 && tid < 64 + kRows * 8 && ((tid - 64) >> 3) < nrows) {
+    float v = 0.0f;
+    if (C == 1) {
+      v = s_part_t[tid - 64];
+    } else {
+      for (int k = 0; k < C; ++k) v += cluster.map_shared_rank(s_part_t, k)[tid - 64];
+    }
+    t[static_cast<int64_t>(m0) * 8 + (tid - 64)] = v;
+  }
+  __syncthreads();
+  // cast from shared memory: a thread's unit is one 16-byte vector in, eight bytes out
+  if (!failed) {
+    uint2* qv = reinterpret_cast<uint2*>(q);
+    for (int idx = tid; idx < nrows * nv; idx += kTileThreads) {
+      const int r = idx / nv, u = idx - r * nv;
+      qv[static_cast<int64_t>(m0 + r) * nvec + v_begin + u] = cast8(s_x[r * pitch + u], s_inv[r]);
+    }
+  }
+  if (C > 1) cluster.sync();  // no CTA may exit while a peer can still read its shared memory
+}
+
+template <bool HAS_V, int C>
+cudaError_t launch_tile(const void* x, int64_t M, int64_t K, int64_t ldx, int vec_per_cta, uint8_t* q, float* sx,
+                        const void* V, float* t, cudaStream_t st) {
+  auto kernel = act_quant_tile_kernel<HAS_V, C>;
+  const size_t smem = static_cast<size_t>(kRows) * (vec_per_cta + kTilePadVec) * sizeof(uint4);
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [&] {
+    attr_err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kRows * (kTileMaxVec + kTilePadVec) * static_cast<int>(sizeof(uint4)));
+  });
+  if (attr_err != cudaSuccess) return attr_err;
+  dim3 grid(C, static_cast<unsigned>((M + kRows - 1) / kRows));
+  return launch_chained(kernel, grid, dim3(kTileThreads), smem, st, false, static_cast<const uint4*>(x),
+                        static_cast<int>(M), static_cast<int>(K), ldx / 8, vec_per_cta, q, sx,
+                        static_cast<const uint4*>(V), t);
+}
+
+template <bool HAS_V>
+cudaError_t launch_tile_c(int c, const void* x, int64_t M, int64_t K, int64_t ldx, int vec_per_cta, uint8_t* q,
+                          float* sx, const void* V, float* t, cudaStream_t st) {
+  switch (c) {
+    case 1: return launch_tile<HAS_V, 1>(x, M, K, ldx, vec_per_cta, q, sx, V, t, st);
+    case 2: return launch_tile<HAS_V, 2>(x, M, K, ldx, vec_per_cta, q, sx, V, t, st);
+    case 4: return launch_tile<HAS_V, 4>(x, M, K, ldx, vec_per_cta, q, sx, V, t, st);
+    default: return launch_tile<HAS_V, 8>(x, M, K, ldx, vec_per_cta, q, sx, V, t, st);
+  }
+}
+
 // ---- few tokens: a cluster of eight CTAs per row -------------------------------------------------
 // With one CTA per token a decode-size call (1-64 tokens) leaves most SMs idle and its latency is one
 // CTA walking a whole row and all of V.  Here eight CTAs of a thread-block cluster share a row: each
@@ -375,6 +555,19 @@ int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* 
       err = launch_chained(act_quant_rows_kernel<false>, grid, dim3(kRowsThreads), 0, st, false,
                            static_cast<const uint4*>(x), static_cast<int>(M), static_cast<int>(K), ldx / 8, q, sx,
                            static_cast<const uint4*>(nullptr), t);
+    count_launch();
+    return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
+  }
+  // a few hundred tokens: eight rows per cluster of as many CTAs as make slices of at most 2048 columns (as long
+  // as the cluster allows), so that even 64 tokens spread over dozens of SMs
+  if (M >= kTileMinTokens && M < kRowsMinTokens && (V == nullptr || r == 8) && K >= 1024 &&
+      K / 8 <= kTileMaxCluster * kTileMaxVec) {
+    const int nvec = static_cast<int>(K / 8);
+    int c = 1;
+    while (c < kTileMaxCluster && (nvec + c - 1) / c > kTileMaxVec / 2) c *= 2;
+    const int vec_per_cta = ((nvec + c - 1) / c + 3) / 4 * 4;
+    err = V ? launch_tile_c<true>(c, x, M, K, ldx, vec_per_cta, q, sx, V, t, st)
+            : launch_tile_c<false>(c, x, M, K, ldx, vec_per_cta, q, sx, nullptr, t, st);
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
   }

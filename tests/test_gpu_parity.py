@@ -45,8 +45,30 @@ def test_act_quant_many_rows_kernel(M, K, lorc):
         assert np.abs(host(t) - t_o).max() <= 1e-4 * np.abs(t_o).max()
 
 
+@pytest.mark.parametrize("M,K,lorc", [(64, 1024, True), (100, 7168, True), (128, 28672, True), (383, 4096, True),
+                                      (200, 28704, True), (65, 2048, False), (130, 16, True), (72, 40960, True),
+                                      (63, 7168, True), (77, 3600, True), (32, 7168, True), (31, 7168, True),
+                                      (40, 28672, True)])
+def test_act_quant_a_few_hundred_rows(M, K, lorc):
+    """Token counts between the cluster-per-row kernel and the eight-row CTAs: eight rows per cluster with the rows
+    in shared memory (and, outside its limits on K, the kernels around it)."""
+    x_bits = synth.make_x(500 + M, M, K, max(1, K // 100), 20.0)
+    x_bits[min(5, M - 1)] = 0                      # an all-zero token
+    V = synth.make_lorc(500 + M, 8, K, 8)[1] if lorc else None
+    q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
+    q, sx, t = binding.quantize_act_fp8(to_bf16(x_bits), up(V))
+    assert np.array_equal(host(q), q_o)
+    assert np.array_equal(host(sx).view(np.uint32), sx_o.view(np.uint32))
+    if lorc:
+        assert np.abs(host(t) - t_o).max() <= 1e-4 * np.abs(t_o).max()
+
+
 def test_act_quant_many_rows_strided_input():
-    M, K = 517, 7168
+    _strided_quant_case(517, 7168)
+    _strided_quant_case(150, 7168)
+
+
+def _strided_quant_case(M, K):
     x_bits = synth.make_x(77, M, K, 70, 20.0)
     V = synth.make_lorc(77, 8, K, 8)[1]
     wide = torch.full((M, K + 264), 1e30, dtype=torch.bfloat16, device=dev())
