@@ -649,8 +649,8 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout, bool a
   const int64_t tiles = static_cast<int64_t>(pl.m_tiles) * pl.n_tiles;
   const int kblocks = static_cast<int>(K / kBlockK);
   if (tiles <= 0 || kblocks <= 0) return pl;  // nothing to do: an empty plan (ctas == 0)
-  if (wide && allow_pair && bm >= 192 && pl.n_tiles % 2 == 0 && sm_count() >= 2 && tiles <= kWsMaxTiles) {
-    // CTA pairs: the two CTAs of a cluster share each token tile (192 or 224 tokens, two accumulators) and
+  if (wide && allow_pair && bm >= 128 && pl.n_tiles % 2 == 0 && sm_count() >= 2 && tiles <= kWsMaxTiles) {
+    // CTA pairs: the two CTAs of a cluster share each token tile (128, 192 or 224 tokens, two accumulators) and
     // take two neighbouring channel tiles.  Work is counted in units of one K block of one pair position
     // (token tile x channel-tile pair) and partitioned among the pairs like the single CTAs' below: whole
     // positions in whole rounds where there are at least four rounds, the rest (or everything) dealt out as
@@ -659,7 +659,8 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout, bool a
     const int64_t pairs = sm_count() / 2, np = pl.n_tiles / 2;
     int best_bm = 0;
     int64_t best_cols = 0;
-    for (const int cand : {224, 192}) {  // 224 tokens move fewer shared-memory bytes per flop: worth 5 % of padding
+    for (const int cand : {224, 192, 128}) {  // wider tiles move fewer shared-memory bytes per flop: worth 5 % of padding
+      if (cand == 128 && M > 128) continue;   // 128-token tiles: one row of them only
       const int64_t cols = ((M + cand - 1) / cand) * cand;
       if (best_bm == 0 || cols * 21 < best_cols * 20) {
         best_bm = cand;

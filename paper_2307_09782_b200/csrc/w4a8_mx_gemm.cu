@@ -1286,6 +1286,7 @@ int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
       Params pp = make_params(a, plan);
       const bool w8p = a.layout == ZQ_WEIGHTS_MX_FP8;
       switch (plan.bm) {
+        case 128: e = w8p ? launch_pair_cfg<128, true>(a, plan, pp, st) : launch_pair_cfg<128, false>(a, plan, pp, st); break;
         case 192: e = w8p ? launch_pair_cfg<192, true>(a, plan, pp, st) : launch_pair_cfg<192, false>(a, plan, pp, st); break;
         case 224: e = w8p ? launch_pair_cfg<224, true>(a, plan, pp, st) : launch_pair_cfg<224, false>(a, plan, pp, st); break;
       }

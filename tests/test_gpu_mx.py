@@ -129,6 +129,8 @@ def test_linear_cta_pairs(M, N, K, r, mode, layout, out_dtype):
     (500, 128 * 6, 2048, torch.float32),      # 3 x 3 positions x 16 K blocks dealt out as ranges: most positions shared
     (500, 128 * 6, 2048, torch.bfloat16),     # bf16 y with shared tiles: the single CTAs take it (workspace partial sums)
     (192, 128 * 150, 512, torch.float32),     # one row of 192-token tiles
+    (100, 128 * 20, 1024, torch.float32),     # one row of 128-token tiles, 20 pairs
+    (128, 128 * 150, 256, torch.float32),     # one row of 128-token tiles, all 74 pairs
     (1120, 128 * 120, 9216, torch.float32),   # four whole rounds, then four positions dealt out to all 74 pairs
 ])
 def test_linear_cta_pairs_shared_positions(M, N, K, out_dtype):
@@ -138,7 +140,7 @@ def test_linear_cta_pairs_shared_positions(M, N, K, out_dtype):
     assert pl["pair"] == 1 and (pl["stream"] == 1 or pl["tail_pos0"] < pl["m_tiles"] * pl["n_tiles"] // 2)
     x_bits, W, U, V = _layer(93, M, N, K, 8)
     bm = pl["bm"]
-    rows = sorted({0, bm // 2 - 1, bm // 2, bm - 1, min(bm, M - 1), M // 2, M - 2, M - 1})
+    rows = sorted({min(v, M - 1) for v in (0, bm // 2 - 1, bm // 2, bm - 1, bm, M // 2, M - 2, M - 1)})
     q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
     c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, 128, "M2")
     y_o = oracle.w4a8_linear(q_o, sx_o, c_o, sh_o, sc_o, 128, "M2", U, t_o, rows=rows)
