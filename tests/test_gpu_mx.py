@@ -157,6 +157,35 @@ def test_linear_cta_pairs_shared_positions(M, N, K, out_dtype):
         assert np.all(np.abs(yh - y_o) <= tol)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_linear_cta_pairs_seeded_random_shapes(seed):
+    """Seeded random shapes with an even number of channel tiles (ragged last tile, any K, ranks 0 / 8 / 16, both
+    output types): whatever partition the plan picks, sampled rows must match the oracle, twice on one workspace."""
+    rng = np.random.default_rng(4242 + seed)
+    M = int(rng.choice([rng.integers(65, 129), rng.integers(129, 600), rng.integers(600, 2600)]))
+    N = 256 * int(rng.integers(1, 80)) - int(rng.integers(0, 128))
+    K = 128 * int(rng.integers(1, 40))
+    r = int(rng.choice([0, 8, 8, 16]))
+    mode = str(rng.choice(["M1", "M2"]))
+    out_dtype = torch.float32 if rng.random() < 0.75 else torch.bfloat16
+    assert binding.linear_plan(M, N, K, mode, MX)["pair"] == 1 or M > 224
+    x_bits, W, U, V = _layer(2000 + seed, M, N, K, r)
+    rows = sorted(set(int(v) for v in rng.integers(0, M, 10)) | {0, M - 1})
+    q_o, sx_o, t_o = oracle.quantize_act_fp8(x_bits, V)
+    c_o, sh_o, sc_o = oracle.pack_weight_fp4(W, 128, mode)
+    y_o = oracle.w4a8_linear(q_o, sx_o, c_o, sh_o, sc_o, 128, mode, U, t_o, rows=rows)
+    pw = binding.pack_weight_fp4(up(W), 128, mode, MX)
+    ws = binding.make_workspace(binding.linear_workspace_bytes(M, N, K, r))
+    q, sx, t = binding.quantize_act_fp8(to_bf16(x_bits), up(V))
+    tol = TOL_REL * np.abs(y_o).max()
+    if out_dtype == torch.bfloat16:
+        tol = tol + 2.0 ** (np.floor(np.log2(np.maximum(np.abs(y_o), 1e-30))) - 7)
+    for _ in range(2):
+        y = binding.w4a8_linear(pw, q=q, sx=sx, t=t, U=up(U), out_dtype=out_dtype, workspace=ws)
+        assert binding.device_status(ws) == (0, 0)
+        assert np.all(np.abs(host(y.float()).astype(np.float64)[rows] - y_o) <= tol)
+
+
 def test_linear_cta_pairs_fp8_weights():
     M, N, K, r = 1120, 128 * 120, 384, 8
     assert binding.linear_plan(M, N, K, "M2", binding.WEIGHTS_MX_FP8)["pair"] == 1
