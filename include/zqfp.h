@@ -175,6 +175,34 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
                    size_t workspace_bytes, void* stream);
 
 /*
+ * Fusion on the output side of the layer (Section 3: the next layer quantizes this layer's output token-wise
+ * to FP8, Appendix A): zq_w4a8_linear with two additions.
+ *   relu      non-zero: y = max(y, 0) before the store (the MLP non-linearity of the OPT family).
+ *   y_absmax  device float [M] or NULL: receives, per token, the maximum of |y| over all N outputs, of the
+ *             values as they are stored (after relu; after the rounding to bf16 when ydt is bf16).  The call
+ *             clears the array first (on the stream) and the epilogues add in with atomic maxima.
+ * With these maxima the next layer's quantizer needs no reduction: zq_quantize_act_fp8_scaled below.
+ * Output tiles shared by several CTAs take the partial-sum route through the workspace here (as for a bf16 y):
+ * nobody adds into y, because the final value must be known to the CTA that forms the maximum.
+ * Everything else (arguments, workspace, errors) as zq_w4a8_linear.
+ */
+int zq_w4a8_linear_fused_out(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M,
+                             int64_t N, int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout,
+                             const uint8_t* codes, const uint8_t* shift, const float* scale, const void* U_f16,
+                             const void* V_f16, const float* t, int r, void* y, zq_out_dtype ydt, int64_t ldy,
+                             void* workspace, size_t workspace_bytes, void* stream, int relu, float* y_absmax);
+
+/*
+ * zq_quantize_act_fp8 for a caller that already has the tokens' absolute maxima (Section 3, Appendix A, Eq. 1 with
+ * Z = 0: s_x = absmax / 448, q = RNE_E4M3(x * (448 / absmax))): one pass over x, no reduction.
+ *   absmax  device float [M]: max_k |x[m, k]| exactly (e.g. from zq_w4a8_linear_fused_out of the layer before);
+ *           a value that is not the row's maximum gives codes that differ from zq_quantize_act_fp8's.
+ * Other arguments, outputs and errors as zq_quantize_act_fp8.
+ */
+int zq_quantize_act_fp8_scaled(const void* x_bf16, int64_t M, int64_t K, int64_t ldx, const float* absmax,
+                               uint8_t* q, float* sx, const void* V_f16, int r, float* t, void* stream);
+
+/*
  * How zq_w4a8_linear would partition a problem on the current device (no launch; host only).  Not an
  * operation of the paper: it exposes the launch plan so that its arithmetic can be checked without a GPU.
  * Work is counted in units of one 128-element K block of one output tile (128 channels x bm tokens);

@@ -27,6 +27,7 @@ EXPORTS = [
     "zq_w4a8_linear_workspace_bytes", "zq_workspace_init", "zq_w4a8_linear",
     "zq_w4a8_linear_host_workspace_bytes", "zq_w4a8_linear_host", "zq_device_status", "zq_launch_count",
     "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc", "zq_w4a8_linear_noalloc_status", "zq_w4a8_linear_plan", "zq_selftest_bounded_wait", "zq_lorc_workspace_bytes", "zq_lorc_factors",
+    "zq_w4a8_linear_fused_out", "zq_quantize_act_fp8_scaled",
 ]
 PLAN_FIELDS = ("bm", "m_tiles", "n_tiles", "ctas", "stream", "persist", "splits", "kb_per_split", "base", "rem",
                "tail_pos0", "m_group", "partial_floats", "sms", "pair")
@@ -86,6 +87,10 @@ def lib() -> C.CDLL:
         L.zq_lorc_workspace_bytes.argtypes = [i64, i64, ci]
         L.zq_lorc_factors.restype = ci
         L.zq_lorc_factors.argtypes = [vp, i64, i64, ci, ci, vp, vp, ci, vp, ci, vp, vp, vp, vp, sz, vp]
+        L.zq_w4a8_linear_fused_out.restype = ci
+        L.zq_w4a8_linear_fused_out.argtypes = L.zq_w4a8_linear.argtypes + [ci, vp]
+        L.zq_quantize_act_fp8_scaled.restype = ci
+        L.zq_quantize_act_fp8_scaled.argtypes = [vp, i64, i64, i64, vp, vp, vp, vp, ci, vp, vp]
         _lib = L
     return _lib
 
@@ -127,8 +132,9 @@ def packed_weight_sizes(N: int, K: int, group: int, mode, layout=WEIGHTS_CAST):
     return a.value, b.value, c.value
 
 
-def quantize_act_fp8(x: torch.Tensor, V: Optional[torch.Tensor] = None):
-    """x: bf16 [M, K] (row stride allowed).  Returns (q uint8 [M,K], sx float32 [M], t float32 [M,r] | None)."""
+def quantize_act_fp8(x: torch.Tensor, V: Optional[torch.Tensor] = None, absmax: Optional[torch.Tensor] = None):
+    """x: bf16 [M, K] (row stride allowed).  Returns (q uint8 [M,K], sx float32 [M], t float32 [M,r] | None).
+    With ``absmax`` (float32 [M], the rows' exact absolute maxima): ``zq_quantize_act_fp8_scaled``, one pass."""
     assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
     M, K = x.shape
     q = torch.empty((M, K), dtype=torch.uint8, device=x.device)
@@ -139,6 +145,11 @@ def quantize_act_fp8(x: torch.Tensor, V: Optional[torch.Tensor] = None):
         r = V.shape[0]
         t = torch.empty((M, r), dtype=torch.float32, device=x.device)
     ldx = x.stride(0) if M > 1 else K
+    if absmax is not None:
+        assert absmax.dtype == torch.float32 and absmax.is_contiguous() and absmax.shape == (M,)
+        _check(lib().zq_quantize_act_fp8_scaled(_ptr(x), M, K, ldx, _ptr(absmax), _ptr(q), _ptr(sx), _ptr(V), r,
+                                                _ptr(t), _stream()), "zq_quantize_act_fp8_scaled")
+        return q, sx, t
     _check(lib().zq_quantize_act_fp8(_ptr(x), M, K, ldx, _ptr(q), _ptr(sx), _ptr(V), r, _ptr(t), _stream()),
            "zq_quantize_act_fp8")
     return q, sx, t
@@ -201,8 +212,10 @@ def make_workspace(nbytes: int, device="cuda") -> torch.Tensor:
 
 
 def w4a8_linear(w: PackedWeight, *, q=None, sx=None, t=None, x=None, U=None, V=None,
-                out_dtype=torch.float32, workspace: Optional[torch.Tensor] = None, y=None):
-    """y [M, N] = the quantized linear layer; activations either (q, sx[, t]) or raw bf16 ``x`` (then V when U)."""
+                out_dtype=torch.float32, workspace: Optional[torch.Tensor] = None, y=None, relu=False,
+                y_absmax: Optional[torch.Tensor] = None):
+    """y [M, N] = the quantized linear layer; activations either (q, sx[, t]) or raw bf16 ``x`` (then V when U).
+    ``relu`` / ``y_absmax`` (float32 [M], written): ``zq_w4a8_linear_fused_out``."""
     codes, shift, scale, group, mode, N, K = w.codes, w.shift, w.scale, w.group, w.mode, w.N, w.K
     if x is not None:
         M, ldx = x.shape[0], (x.stride(0) if x.shape[0] > 1 else K)
@@ -215,6 +228,14 @@ def w4a8_linear(w: PackedWeight, *, q=None, sx=None, t=None, x=None, U=None, V=N
         y = torch.empty((M, N), dtype=out_dtype, device=codes.device)
     ydt = OUT_F32 if y.dtype == torch.float32 else OUT_BF16
     ldy = y.stride(0) if M > 1 else N
+    if relu or y_absmax is not None:
+        assert y_absmax is None or (y_absmax.dtype == torch.float32 and y_absmax.is_contiguous() and
+                                    y_absmax.shape == (M,))
+        _check(lib().zq_w4a8_linear_fused_out(_ptr(q), _ptr(sx), _ptr(x), ldx, M, N, K, group, _mode(mode), w.layout,
+                                              _ptr(codes), _ptr(shift), _ptr(scale), _ptr(U), _ptr(V), _ptr(t), r,
+                                              _ptr(y), ydt, ldy, _ptr(workspace), workspace.numel(), _stream(),
+                                              1 if relu else 0, _ptr(y_absmax)), "zq_w4a8_linear_fused_out")
+        return y
     _check(lib().zq_w4a8_linear(_ptr(q), _ptr(sx), _ptr(x), ldx, M, N, K, group, _mode(mode), w.layout, _ptr(codes),
                                 _ptr(shift), _ptr(scale), _ptr(U), _ptr(V), _ptr(t), r, _ptr(y), ydt, ldy,
                                 _ptr(workspace), workspace.numel(), _stream()), "zq_w4a8_linear")

@@ -31,10 +31,13 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// amax_in != nullptr: the caller knows the tokens' absolute maxima (the epilogue of the layer before collected
+// them): no reduction; the row is still kept in registers for the LoRC product.
 template <bool CACHED>
 __global__ void __launch_bounds__(kMaxThreads)
 act_quant_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, uint8_t* __restrict__ q,
-                 float* __restrict__ sx, const uint4* __restrict__ V, int r, float* __restrict__ t) {
+                 float* __restrict__ sx, const uint4* __restrict__ V, int r, float* __restrict__ t,
+                 const float* __restrict__ amax_in) {
   pdl_launch_dependents();
   pdl_wait();  // x may be the output of the kernel before this one
   const int64_t m = blockIdx.x;
@@ -69,6 +72,7 @@ act_quant_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, uint8_t* _
   __syncthreads();
   a = red[0];
   for (int w = 1; w < (T >> 5); ++w) a = fmaxf(a, red[w]);
+  if (amax_in != nullptr) a = __ldg(amax_in + m);
 
   float s = 1.0f, inv = 1.0f;
   if (a != 0.0f) {
@@ -162,15 +166,18 @@ __device__ __forceinline__ void mma_tf32_16x8x8(float (&d)[4], uint32_t a0, uint
       : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 
-template <bool HAS_V>
+// SCALED: the tokens' absolute maxima are given (amax_in), so the codes are written in the one pass that also
+// forms t, and nothing is read twice.
+template <bool HAS_V, bool SCALED>
 __global__ void __launch_bounds__(kRowsThreads, 1)
 act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec, uint8_t* __restrict__ q,
-                      float* __restrict__ sx, const uint4* __restrict__ V, float* __restrict__ t) {
+                      float* __restrict__ sx, const uint4* __restrict__ V, float* __restrict__ t,
+                      const float* __restrict__ amax_in) {
   __shared__ float s_amax[kRowsWarps][kRows];
   __shared__ float s_acc[kRowsWarps][kRows * 8];
   __shared__ float s_inv[kRows];
   pdl_launch_dependents();
-  pdl_wait();  // x may be the output of the kernel before this one
+  pdl_wait();  // x (and amax_in) may be the output of the kernel before this one
   const int m0 = blockIdx.x * kRows;
   const int nrows = min(kRows, M - m0);
   const int nvec = K / 8;  // 16-byte vectors per row
@@ -180,6 +187,22 @@ act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec
   const uint4* xrow = xr + static_cast<int64_t>(g) * ldx_vec;
   const uint4* vrow = V + static_cast<int64_t>(g) * nvec;
   const bool row_ok = g < nrows;
+  float inv_g = 1.0f;
+  if (SCALED) {
+    if (tid < kRows) {
+      const float a = tid < nrows ? __ldg(amax_in + m0 + tid) : 0.0f;
+      float s = 1.0f, inv = 1.0f;
+      if (a != 0.0f) {
+        s = __fdiv_rn(a, 448.0f);
+        inv = __fdiv_rn(448.0f, a);
+      }
+      s_inv[tid] = inv;
+      if (tid < nrows) sx[m0 + tid] = s;
+    }
+    __syncthreads();
+    inv_g = s_inv[g];
+  }
+  uint2* qrow8 = reinterpret_cast<uint2*>(q + static_cast<int64_t>(m0 + (row_ok ? g : 0)) * K);
 
   float amax = 0.0f;
   float d[4] = {0.0f, 0.0f, 0.0f, 0.0f};  // d[0], d[1]: t[token 2 tig, 2 tig + 1][j = g], partial over this warp's K
@@ -195,7 +218,12 @@ act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec
     }
 #pragma unroll
     for (int i = 0; i < kRowsUnroll; ++i) {
-      amax = absmax8(xv[i], amax);
+      if (SCALED) {
+        const int u = base + i * 4 + tig;
+        if (u < nvec && row_ok) qrow8[u] = cast8(xv[i], inv_g);
+      } else {
+        amax = absmax8(xv[i], amax);
+      }
       if (HAS_V) {
         const uint32_t xw[4] = {xv[i].x, xv[i].y, xv[i].z, xv[i].w};
         const uint32_t vw[4] = {vv[i].x, vv[i].y, vv[i].z, vv[i].w};
@@ -219,7 +247,7 @@ act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec
     s_acc[warp][(2 * tig + 1) * 8 + g] = d[1];
   }
   __syncthreads();
-  if (tid < kRows) {
+  if (!SCALED && tid < kRows) {
     float a = s_amax[0][tid];
     for (int w = 1; w < kRowsWarps; ++w) a = fmaxf(a, s_amax[w][tid]);
     float s = 1.0f, inv = 1.0f;
@@ -235,6 +263,7 @@ act_quant_rows_kernel(const uint4* __restrict__ x, int M, int K, int64_t ldx_vec
     for (int w = 0; w < kRowsWarps; ++w) v += s_acc[w][tid - 64];
     t[static_cast<int64_t>(m0) * 8 + (tid - 64)] = v;
   }
+  if (SCALED) return;  // the codes were written in the pass above
   __syncthreads();
   const int nunits = K / kUnit;
   for (int idx = tid; idx < nrows * nunits; idx += kRowsThreads) {
@@ -540,27 +569,39 @@ act_quant_cluster_kernel(const uint4* __restrict__ x, int K, int64_t ldx_vec, ui
 }  // namespace
 
 int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
-                     const void* V, int r, float* t, cudaStream_t st) {
+                     const void* V, int r, float* t, cudaStream_t st, const float* amax_in) {
   if (M == 0) return ZQ_OK;
   cudaError_t err = cudaSuccess;
-  // enough rows for the eight-row CTAs to beat one row per CTA (measured: from about 50 CTAs on), and the
-  // rank the row kernel is written for
-  if (M >= kRowsMinTokens && (V == nullptr || r == 8)) {
+  const uint4* xv = static_cast<const uint4*>(x);
+  const uint4* Vv = static_cast<const uint4*>(V);
+  if (amax_in != nullptr && (V == nullptr || r == 8)) {
+    // the absolute maxima are known: one streaming pass, eight rows per CTA whatever the token count
     dim3 grid(static_cast<unsigned>((M + kRows - 1) / kRows));
     if (V)
-      err = launch_chained(act_quant_rows_kernel<true>, grid, dim3(kRowsThreads), 0, st, false,
-                           static_cast<const uint4*>(x), static_cast<int>(M), static_cast<int>(K), ldx / 8, q, sx,
-                           static_cast<const uint4*>(V), t);
+      err = launch_chained(act_quant_rows_kernel<true, true>, grid, dim3(kRowsThreads), 0, st, false, xv,
+                           static_cast<int>(M), static_cast<int>(K), ldx / 8, q, sx, Vv, t, amax_in);
     else
-      err = launch_chained(act_quant_rows_kernel<false>, grid, dim3(kRowsThreads), 0, st, false,
-                           static_cast<const uint4*>(x), static_cast<int>(M), static_cast<int>(K), ldx / 8, q, sx,
-                           static_cast<const uint4*>(nullptr), t);
+      err = launch_chained(act_quant_rows_kernel<false, true>, grid, dim3(kRowsThreads), 0, st, false, xv,
+                           static_cast<int>(M), static_cast<int>(K), ldx / 8, q, sx, Vv, t, amax_in);
+    count_launch();
+    return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
+  }
+  // enough rows for the eight-row CTAs to beat one row per CTA (measured: from about 50 CTAs on), and the
+  // rank the row kernel is written for
+  if (amax_in == nullptr && M >= kRowsMinTokens && (V == nullptr || r == 8)) {
+    dim3 grid(static_cast<unsigned>((M + kRows - 1) / kRows));
+    if (V)
+      err = launch_chained(act_quant_rows_kernel<true, false>, grid, dim3(kRowsThreads), 0, st, false, xv,
+                           static_cast<int>(M), static_cast<int>(K), ldx / 8, q, sx, Vv, t, amax_in);
+    else
+      err = launch_chained(act_quant_rows_kernel<false, false>, grid, dim3(kRowsThreads), 0, st, false, xv,
+                           static_cast<int>(M), static_cast<int>(K), ldx / 8, q, sx, Vv, t, amax_in);
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
   }
   // a few hundred tokens: eight rows per cluster of as many CTAs as make slices of at most 2048 columns (as long
-  // as the cluster allows), so that even 64 tokens spread over dozens of SMs
-  if (M >= kTileMinTokens && M < kRowsMinTokens && (V == nullptr || r == 8) && K >= 1024 &&
+  // as the cluster allows), so that even 32 tokens spread over dozens of SMs
+  if (amax_in == nullptr && M >= kTileMinTokens && M < kRowsMinTokens && (V == nullptr || r == 8) && K >= 1024 &&
       K / 8 <= kTileMaxCluster * kTileMaxVec) {
     const int nvec = static_cast<int>(K / 8);
     int c = 1;
@@ -571,13 +612,12 @@ int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* 
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
   }
-  // fewer tokens than the eight-row kernel needs, rows long enough to be worth sharing: a cluster of eight CTAs per row
-  if (M < kRowsMinTokens && (M <= 256 || K >= 16384) && K >= 2048 &&
+  // fewer tokens than that, rows long enough to be worth sharing: a cluster of eight CTAs per row
+  if (amax_in == nullptr && M < kRowsMinTokens && (M <= 256 || K >= 16384) && K >= 2048 &&
       K / kUnit <= kClusterSize * kClusterThreads * kClusterVpt) {
     dim3 grid(kClusterSize, static_cast<unsigned>(M));
-    err = launch_chained(act_quant_cluster_kernel, grid, dim3(kClusterThreads), 0, st, false,
-                         static_cast<const uint4*>(x), static_cast<int>(K), ldx / 8, q, sx,
-                         static_cast<const uint4*>(V), r, t);
+    err = launch_chained(act_quant_cluster_kernel, grid, dim3(kClusterThreads), 0, st, false, xv, static_cast<int>(K),
+                         ldx / 8, q, sx, Vv, r, t);
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
   }
@@ -587,11 +627,11 @@ int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* 
   const bool cached = nunits <= threads * kVpt;
   dim3 grid(static_cast<unsigned>(M));
   if (cached)
-    err = launch_chained(act_quant_kernel<true>, grid, dim3(threads), 0, st, false, static_cast<const uint4*>(x),
-                         static_cast<int>(K), ldx / 8, q, sx, static_cast<const uint4*>(V), r, t);
+    err = launch_chained(act_quant_kernel<true>, grid, dim3(threads), 0, st, false, xv, static_cast<int>(K), ldx / 8, q,
+                         sx, Vv, r, t, amax_in);
   else
-    err = launch_chained(act_quant_kernel<false>, grid, dim3(threads), 0, st, false, static_cast<const uint4*>(x),
-                         static_cast<int>(K), ldx / 8, q, sx, static_cast<const uint4*>(V), r, t);
+    err = launch_chained(act_quant_kernel<false>, grid, dim3(threads), 0, st, false, xv, static_cast<int>(K), ldx / 8,
+                         q, sx, Vv, r, t, amax_in);
   count_launch();
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? ZQ_OK : ZQ_ERR_CUDA;
 }

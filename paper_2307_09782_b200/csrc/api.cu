@@ -124,15 +124,28 @@ const char* zq_status_string(int status) {
 
 int64_t zq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
-int zq_quantize_act_fp8(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
-                        const void* V, int r, float* t, void* stream) {
+namespace {
+int quantize_act(const void* x, int64_t M, int64_t K, int64_t ldx, const float* absmax, bool scaled, uint8_t* q,
+                 float* sx, const void* V, int r, float* t, void* stream) {
   if (M < 0 || K < 16 || K % 16 || ldx < K || K > (int64_t(1) << 30) || M > 0x7FFFFFFF) return ZQ_ERR_SHAPE;
   if (V && (r <= 0 || r > 64)) return ZQ_ERR_SHAPE;
   if (M == 0) return ZQ_OK;
-  if (!x || !q || !sx || (V && !t)) return ZQ_ERR_NULL;
+  if (!x || !q || !sx || (V && !t) || (scaled && !absmax)) return ZQ_ERR_NULL;
   if (!aligned16(x) || !aligned16(q) || ldx % 8 || (V && !aligned16(V))) return ZQ_ERR_ALIGN;
   if (int e = check_device_sm100()) return e;
-  return launch_act_quant(x, M, K, ldx, q, sx, V, V ? r : 0, t, static_cast<cudaStream_t>(stream));
+  return launch_act_quant(x, M, K, ldx, q, sx, V, V ? r : 0, t, static_cast<cudaStream_t>(stream),
+                          scaled ? absmax : nullptr);
+}
+}  // namespace
+
+int zq_quantize_act_fp8(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
+                        const void* V, int r, float* t, void* stream) {
+  return quantize_act(x, M, K, ldx, nullptr, false, q, sx, V, r, t, stream);
+}
+
+int zq_quantize_act_fp8_scaled(const void* x, int64_t M, int64_t K, int64_t ldx, const float* absmax, uint8_t* q,
+                               float* sx, const void* V, int r, float* t, void* stream) {
+  return quantize_act(x, M, K, ldx, absmax, true, q, sx, V, r, t, stream);
 }
 
 int zq_packed_weight_sizes(int64_t N, int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout,
@@ -178,10 +191,12 @@ int zq_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
                                                                                                        : ZQ_ERR_CUDA;
 }
 
-int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M, int64_t N,
-                   int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout, const uint8_t* codes,
-                   const uint8_t* shift, const float* scale, const void* U, const void* V, const float* t, int r,
-                   void* y, zq_out_dtype ydt, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+namespace {
+int linear_impl(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M, int64_t N,
+                int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout, const uint8_t* codes,
+                const uint8_t* shift, const float* scale, const void* U, const void* V, const float* t, int r,
+                void* y, zq_out_dtype ydt, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream,
+                int relu, float* y_absmax) {
   if (!valid_mode(mode) || !valid_layout(layout, mode) || (ydt != ZQ_OUT_F32 && ydt != ZQ_OUT_BF16))
     return ZQ_ERR_MODE;
   if (!valid_linear_shape(M, N, K, r) || !valid_group(group, mode) || K % group || ldy < N) return ZQ_ERR_SHAPE;
@@ -208,6 +223,9 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
+  // the epilogues add the tokens' maxima in with atomic max: start from zero
+  if (y_absmax && cudaMemsetAsync(y_absmax, 0, static_cast<size_t>(M) * sizeof(float), st) != cudaSuccess)
+    return ZQ_ERR_CUDA;
   if (x_bf16 && layout_is_mx(layout) && mode != ZQ_SCALE_NONE && M <= kFusedMaxTokens) {
     // Few tokens (decode): the block-scaled kernel quantizes the activations itself, so the layer is one
     // launch.  If that launch is refused, the two-kernel path below runs instead.
@@ -235,6 +253,8 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
     f.ldx = ldx;
     f.V = r > 0 ? V : nullptr;
     f.fused_scratch = ws + kWsStatusBytes + kWsCounterBytes;
+    f.relu = relu;
+    f.y_amax = y_absmax;
     const int e = launch_w4a8_mx_gemm(f, st);
     if (e != kFusedLaunchRefused) return e;
   }
@@ -270,7 +290,27 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
   a.counters = reinterpret_cast<int*>(ws + kWsStatusBytes);
   a.partials = reinterpret_cast<float*>(ws + w.off_partials);
   a.partial_floats = w.partial_floats;
+  a.relu = relu;
+  a.y_amax = y_absmax;
   return layout_is_mx(layout) ? launch_w4a8_mx_gemm(a, st) : launch_w4a8_gemm(a, st);
+}
+}  // namespace
+
+int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M, int64_t N,
+                   int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout, const uint8_t* codes,
+                   const uint8_t* shift, const float* scale, const void* U, const void* V, const float* t, int r,
+                   void* y, zq_out_dtype ydt, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+  return linear_impl(q, sx, x_bf16, ldx, M, N, K, group, mode, layout, codes, shift, scale, U, V, t, r, y, ydt, ldy,
+                     workspace, workspace_bytes, stream, 0, nullptr);
+}
+
+int zq_w4a8_linear_fused_out(const uint8_t* q, const float* sx, const void* x_bf16, int64_t ldx, int64_t M,
+                             int64_t N, int64_t K, int group, zq_scale_mode mode, zq_weight_layout layout,
+                             const uint8_t* codes, const uint8_t* shift, const float* scale, const void* U,
+                             const void* V, const float* t, int r, void* y, zq_out_dtype ydt, int64_t ldy,
+                             void* workspace, size_t workspace_bytes, void* stream, int relu, float* y_absmax) {
+  return linear_impl(q, sx, x_bf16, ldx, M, N, K, group, mode, layout, codes, shift, scale, U, V, t, r, y, ydt, ldy,
+                     workspace, workspace_bytes, stream, relu ? 1 : 0, y_absmax);
 }
 
 int zq_w4a8_linear_plan(int64_t M, int64_t N, int64_t K, zq_scale_mode mode, zq_weight_layout layout,

@@ -483,7 +483,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
             if (!failed) {
 #pragma unroll
               for (int c = 0; c < BM; c += EC)
-                if (n_ok) finalize<EC, BM>(p, run + c, m0, c, n, cs, u, s_sx, s_t);
+                if (n_ok || p.y_amax) finalize<EC, BM>(p, run + c, m0, c, n, cs, u, s_sx, s_t, false, true, n_ok);
             }
           } else if (!failed && has_cols) {
             // the next step's accumulator columns are in flight while this step's are finished
@@ -496,7 +496,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
 #pragma unroll
               for (int e = 0; e < EC; ++e) v[e] = nxt[e];
               if (c + EC < kMyCols) tmem_ld_issue<EC>(t_lane + col0 + c + EC, nxt);
-              if (n_ok) finalize<EC, BM>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+              if (n_ok || p.y_amax) finalize<EC, BM>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t, false, true, n_ok);
             }
           }
         } else if (!NONE && p.atomic_y) {
@@ -556,7 +556,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tm_q, const Params p) {
 #pragma unroll
                 for (int e = 0; e < EC; ++e) v[e] += __ldcg(src + e * kTileN);
               }
-              if (n_ok) finalize<EC, BM>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t);
+              if (n_ok || p.y_amax) finalize<EC, BM>(p, v, m0, col0 + c, n, cs, u, s_sx, s_t, false, true, n_ok);
             }
           }
           named_bar_sync(1, C::kEpiThreads);  // s_last is reused by the next segment

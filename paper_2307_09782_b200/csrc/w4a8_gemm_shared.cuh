@@ -80,6 +80,9 @@ struct Params {
   const __half* V;
   uint8_t* q_out;
   FusedScratch* fq;
+  // fusion on the output side (see GemmArgs)
+  int relu;
+  float* y_amax;
 };
 
 constexpr int cmin(int a, int b) { return a < b ? a : b; }
@@ -139,10 +142,12 @@ __device__ __forceinline__ size_t partial_slot(const Params& p, int tile, int fi
 // other ranks read t and U through the cache.
 // `add`: y was zeroed by the launcher and this CTA holds only part of the K range, so it adds (FP32 atomics,
 // order-dependent in the last bit); `lorc`: this CTA is the one that contributes the LoRC term.
+// `store_ok` == false: the channel lies beyond N; the thread is here only for the warp-wide maximum of p.y_amax.
 template <int NC, int BM>
 __device__ __forceinline__ void finalize(const Params& p, const float* v, int m0, int c0, int n, float cs,
                                          const uint64_t* u2, const float* __restrict__ s_sx,
-                                         const float* __restrict__ s_tT, bool add = false, bool lorc = true) {
+                                         const float* __restrict__ s_tT, bool add = false, bool lorc = true,
+                                         bool store_ok = true) {
   // All NC results are computed before the first store, so that the columns' loads and FMA chains
   // interleave instead of running one column at a time behind each store.
   static_assert(NC % 4 == 0, "columns are taken four at a time");
@@ -180,6 +185,26 @@ __device__ __forceinline__ void finalize(const Params& p, const float* v, int m0
       }
     }
   }
+  if (p.relu && !add) {
+#pragma unroll
+    for (int c = 0; c < NC; ++c) out[c] = fmaxf(out[c], 0.0f);
+  }
+  if (p.y_amax != nullptr && !add) {
+    // Per-token max |y| over this warp's 32 channels, of the values as they are stored (rounding to bf16 is
+    // monotone, so it commutes with the maximum); one atomic max per token and warp.  Every lane of the warp is
+    // here (a channel beyond N comes with store_ok == false and counts as zero).
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      float a = p.ydt == ZQ_OUT_F32 ? fabsf(out[c]) : fabsf(__bfloat162float(__float2bfloat16_rn(out[c])));
+      if (!store_ok) a = 0.0f;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
+      const int m = m0 + c0 + c;
+      if ((threadIdx.x & 31) == 0 && m < p.M && a > 0.0f)
+        atomicMax(reinterpret_cast<unsigned int*>(p.y_amax) + m, __float_as_uint(a));
+    }
+  }
+  if (!store_ok) return;
   const int64_t base = static_cast<int64_t>(m0 + c0) * p.ldy + n;
   if (add) {
     float* y = static_cast<float*>(p.y) + base;
@@ -260,7 +285,9 @@ inline Params make_params(const GemmArgs& a, const GemmPlan& plan) {
   p.tail_pos0 = plan.tail_pos0;
   p.dealt0 = plan.persist ? plan.tail_pos0 * p.kblocks : 0;
   p.m_group = plan.m_group;
-  p.atomic_y = (plan.stream && a.ydt == ZQ_OUT_F32 && plan.partial_floats > 0) ? 1 : 0;
+  p.relu = a.relu;
+  p.y_amax = a.y_amax;
+  p.atomic_y = (plan.stream && a.ydt == ZQ_OUT_F32 && plan.partial_floats > 0 && !a.relu && !a.y_amax) ? 1 : 0;
   p.splits = plan.splits;
   p.kb_per_split = plan.kb_per_split;
   p.base = plan.base;

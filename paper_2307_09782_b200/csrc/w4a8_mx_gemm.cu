@@ -657,7 +657,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
 #pragma unroll
             for (int e = 0; e < EC; ++e) v[e] = nxt[e];
             if (c + EC < BM) tmem_ld_issue<EC>(t_lane + c + EC, nxt);
-            if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t);
+            if (n_ok || p.y_amax) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t, false, true, n_ok);
           }
         }
       } else if (p.atomic_y && p.handover) {
@@ -751,7 +751,7 @@ w4a8_mx_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
 #pragma unroll
               for (int e = 0; e < EC; ++e) v[e] += __ldcg(src + e * kTileN);
             }
-            if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t);
+            if (n_ok || p.y_amax) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t, false, true, n_ok);
           }
         }
         named_bar_sync(1, C::kEpiThreads);  // s_last is reused by the next segment
@@ -1078,7 +1078,7 @@ w4a8_mx_pair_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_
 #pragma unroll
             for (int e = 0; e < EC; ++e) v[e] = nxt[e];
             if (c + EC < BM) tmem_ld_issue<EC>(t_lane + c + EC, nxt);
-            if (n_ok) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t);
+            if (n_ok || p.y_amax) finalize<EC, BM>(p, v, m0, c, n, cs, u, s_sx, s_t, false, true, n_ok);
           }
         }
       } else {
@@ -1184,8 +1184,9 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
   });
   if (attr_err != cudaSuccess) return ZQ_ERR_CUDA;
   dim3 grid(static_cast<unsigned>(plan.ctas));
+  const bool fused_out = a.relu || a.y_amax;  // final values must be known to one CTA: no adding into y
   const bool shared_f32 =
-      a.ydt == ZQ_OUT_F32 && (p.atomic_y || (plan.persist && plan.tail_pos0 < p.tiles));
+      a.ydt == ZQ_OUT_F32 && !fused_out && (p.atomic_y || (plan.persist && plan.tail_pos0 < p.tiles));
   if (shared_f32 || FUSEQ) {
     // Output tiles are shared by CTAs that accumulate into FP32 y.  In a cooperative launch (all CTAs
     // resident, which the plan's grid is sized for) they hand over through per-tile flags: one stores,
@@ -1278,11 +1279,11 @@ int launch_pair_cfg(const GemmArgs& a, const GemmPlan& plan, Params p, cudaStrea
 int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
   GemmPlan plan = plan_gemm(a.M, a.N, a.K, a.mode, ZQ_WEIGHTS_MX);
   if (plan.pair) {
-    // positions shared between pairs are added into an FP32 y; a bf16 y takes the single CTAs, and so does a
-    // device that grants the pair kernel fewer pairs than planned
+    // positions shared between pairs are added into an FP32 y; a bf16 y (or one with ReLU / the tokens' maxima
+    // fused in) takes the single CTAs, and so does a device that grants the pair kernel fewer pairs than planned
     const bool shared = plan.stream || plan.tail_pos0 < plan.m_tiles * (plan.n_tiles / 2);
     int e = kPairNotTaken;
-    if (!(shared && a.ydt != ZQ_OUT_F32)) {
+    if (!(shared && (a.ydt != ZQ_OUT_F32 || a.relu || a.y_amax))) {
       Params pp = make_params(a, plan);
       const bool w8p = a.layout == ZQ_WEIGHTS_MX_FP8;
       switch (plan.bm) {

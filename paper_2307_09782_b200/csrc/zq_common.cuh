@@ -69,8 +69,9 @@ inline size_t tile_bytes(int layout) {
 inline bool layout_is_mx(int layout) { return layout == ZQ_WEIGHTS_MX || layout == ZQ_WEIGHTS_MX_FP8; }
 
 // ---- launchers implemented in the .cu files ------------------------------------------------------
+// amax_in: the tokens' absolute maxima when the caller already has them (one pass: no reduction, no second read)
 int launch_act_quant(const void* x, int64_t M, int64_t K, int64_t ldx, uint8_t* q, float* sx,
-                     const void* V, int r, float* t, cudaStream_t st);
+                     const void* V, int r, float* t, cudaStream_t st, const float* amax_in = nullptr);
 int launch_pack_weight(const float* W, int64_t N, int64_t K, int group, int mode, int layout, uint8_t* codes,
                        uint8_t* shift, float* scale, cudaStream_t st);
 
@@ -99,6 +100,12 @@ struct GemmArgs {
   int64_t ldx;
   const void* V;         // fp16 [r, K] or NULL
   void* fused_scratch;   // kWsFusedBytes of the workspace head
+  // fusion on the output side: y = max(y, 0) before the store, and / or the per-token max |y| (of the values as
+  // stored) added with atomic max into y_amax [M] for the next layer's quantizer.  Either one keeps shared output
+  // tiles off the paths that add into y (their final values are known to no CTA): partial sums go through the
+  // workspace instead, as for a bf16 y.
+  int relu;
+  float* y_amax;
 };
 // Returned by launch_w4a8_mx_gemm when that launch was refused (the grid cannot be resident at once): nothing
 // ran; the caller quantizes with the separate kernel and launches the plain GEMM.
