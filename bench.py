@@ -501,6 +501,7 @@ def run_ours(args):
     # ---- further rows the configurations ask for (not part of the timed step)
     extra_rows = []
     lorc_ms = None
+    mlp_chain = None
     if not args.case and not args.no_extra:
         def extra(wl_, shape, M, md, lay, r_):
             ly = B.make_layer(wl_, shape, M, md, lay, rank_lorc=r_)
@@ -561,6 +562,76 @@ def run_ours(args):
                         "layer before (zq_w4a8_linear_fused_out), so x is read once and nothing is reduced",
                 "us": round(us1, 2), "achieved": round(gbs1, 1), "frac": round(gbs1 / peaks["hbm_gbs"], 4)}
         del ly, amax
+        # The two layers chained as an MLP block at the largest token count, fc1 -> ReLU -> fc2, with and without
+        # the fusion on the output side: fused = fc1 with ReLU and the token maxima in its epilogue (bf16 y), the
+        # one-pass quantizer, fc2; unfused = fc1 (bf16 y), a separate ReLU pass, the two-pass quantizer, fc2.
+        if len(shapes) == 2 and shapes[0].N == shapes[1].K:
+            l1 = B.make_layer(wl, shapes[0], Mmax, mode, args.layout, copies=1)
+            l2 = B.make_layer(wl, shapes[1], Mmax, mode, args.layout, copies=1)
+            y1 = torch.empty((Mmax, shapes[0].N), dtype=torch.bfloat16, device=dev)
+            am1 = torch.empty((Mmax,), dtype=torch.float32, device=dev)
+            vp_ = B.vp
+
+            def fc(ly, x_raw, q_, sx_, t_, y_, ydt, relu, amax_):
+                c_, sh_, sc_ = ly["copies"][0]
+                args_ = (vp_(q_), vp_(sx_), vp_(x_raw), ly["K"], Mmax, ly["N"], ly["K"], GROUP, ly["mode"], ly["layout"],
+                         vp_(c_), vp_(sh_), vp_(sc_), vp_(ly["U"]), vp_(ly["V"]) if x_raw is not None else None,
+                         vp_(t_) if (t_ is not None and ly["r"]) else None, ly["r"], vp_(y_), ydt, ly["N"], vp_(ly["ws"]),
+                         ly["ws"].numel(), B.sp)
+                rc = (B.L.zq_w4a8_linear_fused_out(*args_, 1 if relu else 0, vp_(amax_)) if (relu or amax_ is not None)
+                      else B.L.zq_w4a8_linear(*args_))
+                if rc:
+                    raise RuntimeError(f"linear failed in the MLP chain: {rc}")
+
+            def quant2(scaled):
+                a_ = (vp_(y1), Mmax, l2["K"], l2["K"])
+                b_ = (vp_(l2["q"]), vp_(l2["sx"]), vp_(l2["V"]), l2["r"], vp_(l2["t"]) if l2["r"] else None, B.sp)
+                rc = (B.L.zq_quantize_act_fp8_scaled(*a_, vp_(am1), *b_) if scaled else B.L.zq_quantize_act_fp8(*a_, *b_))
+                if rc:
+                    raise RuntimeError(f"quantizer failed in the MLP chain: {rc}")
+
+            def fused():
+                fc(l1, l1["x"], None, None, None, y1, 1, True, am1)
+                quant2(True)
+                fc(l2, None, l2["q"], l2["sx"], l2["t"], l2["y"], 0, False, None)
+
+            def fused_relu():
+                fc(l1, l1["x"], None, None, None, y1, 1, True, None)
+                quant2(False)
+                fc(l2, None, l2["q"], l2["sx"], l2["t"], l2["y"], 0, False, None)
+
+            def unfused():
+                fc(l1, l1["x"], None, None, None, y1, 1, False, None)
+                torch.relu_(y1)
+                quant2(False)
+                fc(l2, None, l2["q"], l2["sx"], l2["t"], l2["y"], 0, False, None)
+
+            def timed3(fn, n=4):
+                res = []
+                e0_, e1_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                for b in range(3):
+                    e0_.record(B.stream)
+                    for _ in range(n):
+                        fn()
+                    e1_.record(B.stream)
+                    torch.cuda.synchronize()
+                    res.append(e0_.elapsed_time(e1_) * 1e3 / n)
+                return statistics.median(res[1:])
+            # interleaved, so that all three see the same clocks
+            runs_ = {"u": [], "r": [], "f": []}
+            for rep_ in range(3):
+                for key_, fn_ in (("u", unfused), ("r", fused_relu), ("f", fused)):
+                    runs_[key_].append(timed3(fn_, n=2))
+            tu_, tr_, tf_ = (statistics.median(runs_[k_]) for k_ in ("u", "r", "f"))
+            fl_ = flops(Mmax, shapes[0].N, shapes[0].K, RANK) + flops(Mmax, shapes[1].N, shapes[1].K, RANK)
+            mlp_chain = {"what": "fc1 -> ReLU -> fc2 at M = %d, bf16 between the layers, FP32 out: separate ReLU pass; "
+                                 "ReLU in fc1's epilogue; ReLU and the token maxima in fc1's epilogue with the "
+                                 "one-pass quantizer" % Mmax,
+                         "unfused_us": round(tu_, 1), "relu_fused_us": round(tr_, 1), "relu_and_maxima_fused_us": round(tf_, 1),
+                         "unfused_tflops": round(fl_ / (tu_ * 1e-6) / 1e12, 1),
+                         "relu_fused_tflops": round(fl_ / (tr_ * 1e-6) / 1e12, 1),
+                         "relu_and_maxima_fused_tflops": round(fl_ / (tf_ * 1e-6) / 1e12, 1)}
+            del l1, l2, y1, am1
         wl7 = synth.WORKLOADS["llama7b"]  # unconstrained scales (per-group FP32 promotion) at 2048 tokens
         for shape in wl7.shapes:
             for md, lay in EXTRA_LLAMA7B:
@@ -631,7 +702,7 @@ def run_ours(args):
                           "around n = 6-20 back-to-back launches (rotated weight copies), divided by n, median of 3 "
                           "batches; layer_us = one zq_w4a8_linear call on raw x; quant_us / gemm_us = the quantizer "
                           "kernel alone and the GEMM alone on pre-quantized activations",
-            "sweep": table, "extra_rows": extra_rows, "lorc_factors_ms": lorc_ms}
+            "sweep": table, "extra_rows": extra_rows, "lorc_factors_ms": lorc_ms, "mlp_chain": mlp_chain}
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(wl)
     print(json.dumps(line))

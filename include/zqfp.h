@@ -181,7 +181,9 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
  *   y_absmax  device float [M] or NULL: receives, per token, the maximum of |y| over all N outputs, of the
  *             values as they are stored (after relu; after the rounding to bf16 when ydt is bf16).  The call
  *             clears the array first (on the stream) and the epilogues add in with atomic maxima.
- * With these maxima the next layer's quantizer needs no reduction: zq_quantize_act_fp8_scaled below.
+ * With these maxima the next layer's quantizer needs no reduction: zq_quantize_act_fp8_scaled below.  (The
+ * ReLU costs nothing; the maxima cost a warp reduction and an atomic per token, warp and tile, which pays only
+ * for narrow outputs of long rows.)
  * Output tiles shared by several CTAs take the partial-sum route through the workspace here (as for a bf16 y):
  * nobody adds into y, because the final value must be known to the CTA that forms the maximum.
  * Everything else (arguments, workspace, errors) as zq_w4a8_linear.

@@ -195,13 +195,12 @@ __device__ __forceinline__ void finalize(const Params& p, const float* v, int m0
     // here (a channel beyond N comes with store_ok == false and counts as zero).
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
-      float a = p.ydt == ZQ_OUT_F32 ? fabsf(out[c]) : fabsf(__bfloat162float(__float2bfloat16_rn(out[c])));
-      if (!store_ok) a = 0.0f;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, o));
+      const float a = p.ydt == ZQ_OUT_F32 ? fabsf(out[c]) : fabsf(__bfloat162float(__float2bfloat16_rn(out[c])));
+      // non-negative floats order like their bit patterns: one warp-wide integer maximum per token
+      const unsigned int bits = __reduce_max_sync(0xFFFFFFFFu, store_ok ? __float_as_uint(a) : 0u);
       const int m = m0 + c0 + c;
-      if ((threadIdx.x & 31) == 0 && m < p.M && a > 0.0f)
-        atomicMax(reinterpret_cast<unsigned int*>(p.y_amax) + m, __float_as_uint(a));
+      if ((threadIdx.x & 31) == 0 && m < p.M && bits != 0u)
+        atomicMax(reinterpret_cast<unsigned int*>(p.y_amax) + m, bits);
     }
   }
   if (!store_ok) return;
