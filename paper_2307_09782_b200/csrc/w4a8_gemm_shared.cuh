@@ -191,17 +191,36 @@ __device__ __forceinline__ void finalize(const Params& p, const float* v, int m0
   }
   if (p.y_amax != nullptr && !add) {
     // Per-token max |y| over this warp's 32 channels, of the values as they are stored (rounding to bf16 is
-    // monotone, so it commutes with the maximum); one atomic max per token and warp.  Every lane of the warp is
-    // here (a channel beyond N comes with store_ok == false and counts as zero).
+    // monotone, so it commutes with the maximum).  Non-negative floats order like their bit patterns: one
+    // warp-wide integer maximum per token; lane c keeps token c's.  The running maxima settle after the first few
+    // channel tiles, so each lane first looks at what is there (a stale value only costs a redundant atomic) and
+    // adds its token's maximum in only if it is larger.  Every lane of the warp is here (a channel beyond N comes
+    // with store_ok == false and counts as zero).
+    static_assert(NC <= 32, "one lane per token of the step");
+    const int lane = threadIdx.x & 31;
+    const int m_mine = m0 + c0 + lane;
+    unsigned int* slot = reinterpret_cast<unsigned int*>(p.y_amax) + m_mine;
+    const bool mine_ok = lane < NC && m_mine < p.M;
+    const unsigned int seen = mine_ok ? __ldcg(slot) : 0xFFFFFFFFu;
+    unsigned int mine = 0u;
+    if (p.ydt == ZQ_OUT_F32) {
+      const unsigned int keep = store_ok ? 0x7FFFFFFFu : 0u;  // drops the sign
 #pragma unroll
-    for (int c = 0; c < NC; ++c) {
-      const float a = p.ydt == ZQ_OUT_F32 ? fabsf(out[c]) : fabsf(__bfloat162float(__float2bfloat16_rn(out[c])));
-      // non-negative floats order like their bit patterns: one warp-wide integer maximum per token
-      const unsigned int bits = __reduce_max_sync(0xFFFFFFFFu, store_ok ? __float_as_uint(a) : 0u);
-      const int m = m0 + c0 + c;
-      if ((threadIdx.x & 31) == 0 && m < p.M && bits != 0u)
-        atomicMax(reinterpret_cast<unsigned int*>(p.y_amax) + m, bits);
+      for (int c = 0; c < NC; ++c) {
+        const unsigned int bits = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(out[c]) & keep);
+        if (lane == c) mine = bits;
+      }
+    } else {
+      // the bf16 value's magnitude is the upper half of its FP32 pattern
+      const unsigned int keep = store_ok ? 0x7FFFu : 0u;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) {
+        const unsigned int h = __bfloat16_as_ushort(__float2bfloat16_rn(out[c]));
+        const unsigned int bits = __reduce_max_sync(0xFFFFFFFFu, h & keep);
+        if (lane == c) mine = bits << 16;
+      }
     }
+    if (mine_ok && mine > seen) atomicMax(slot, mine);
   }
   if (!store_ok) return;
   const int64_t base = static_cast<int64_t>(m0 + c0) * p.ldy + n;
