@@ -156,7 +156,9 @@ def oracle_sample_step(wl, state=None, M_s=8):
 def base_config(args, shapes, Ms, mode):
     return {"workload": WORKLOAD if not args.case else f"case {args.case}",
             "layers": [f"{s.K}->{s.N}" for s in shapes], "M": Ms, "group": GROUP, "mode": mode,
-            "weight_layout": args.layout, "lorc_rank": RANK}
+            "weight_layout": args.layout, "lorc_rank": RANK,
+            "launches": ("cooperative where CTAs share output tiles (library default)" if args.cooperative else
+                         "plain: zq_set_exclusive_device(1), the bench has the device to itself")}
 
 
 def cpu_baseline(wl):
@@ -372,6 +374,7 @@ def run_ours(args):
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     B = Bench(dev, rank)
+    binding.set_exclusive_device(not args.cooperative)  # one process, one stream of kernels per GPU
 
     wl = synth.WORKLOADS[WORKLOAD]
     Ms = sorted(wl.Ms, reverse=True)
@@ -733,6 +736,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the rows outside the timed step")
     ap.add_argument("--no-sweep-table", action="store_true", help="skip the per-shape table")
+    ap.add_argument("--cooperative", action="store_true",
+                    help="keep the library's default cooperative launches (the bench has the device to itself and "
+                         "says so to the library, which then launches plainly: about 3.5 us less per shared-tile launch)")
     ap.add_argument("--layout", default="mx", choices=["cast", "mx"],
                     help="weight layout: the kernel casts FP4 to FP8 (cast) or the tensor core does (mx)")
     ap.add_argument("--case", default=None, metavar="K,N,M[,MODE]",

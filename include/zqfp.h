@@ -175,6 +175,19 @@ int zq_w4a8_linear(const uint8_t* q, const float* sx, const void* x_bf16, int64_
                    size_t workspace_bytes, void* stream);
 
 /*
+ * Not an operation of the paper: a promise about how the library is used.  Launches whose CTAs hand shared output
+ * tiles over to one another (few tokens: the K range of a tile is split between CTAs; the kernel that quantizes
+ * its activations itself) need every CTA of the grid running at the same time.  By default they are cooperative
+ * launches, which guarantee it and cost about 3.5 us each.  After zq_set_exclusive_device(1) the caller promises
+ * that no other kernel (of any stream or process) runs on the device while such a call executes; the launches
+ * are then plain ones, whose grids of at most one CTA per SM are resident as soon as the kernel ahead in the
+ * stream has drained.  If the promise is broken, CTAs may wait for CTAs that cannot start: the waits are bounded
+ * and the call ends with ZQ_ERR_DEVICE_TIMEOUT in the workspace status, not with a hang.
+ * Process-wide; returns the previous setting.
+ */
+int zq_set_exclusive_device(int on);
+
+/*
  * Fusion on the output side of the layer (Section 3: the next layer quantizes this layer's output token-wise
  * to FP8, Appendix A): zq_w4a8_linear with two additions.
  *   relu      non-zero: y = max(y, 0) before the store (the MLP non-linearity of the OPT family).

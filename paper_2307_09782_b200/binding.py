@@ -27,7 +27,7 @@ EXPORTS = [
     "zq_w4a8_linear_workspace_bytes", "zq_workspace_init", "zq_w4a8_linear",
     "zq_w4a8_linear_host_workspace_bytes", "zq_w4a8_linear_host", "zq_device_status", "zq_launch_count",
     "zq_w4a8_linear_noalloc_max_scratch_bytes", "zq_w4a8_linear_noalloc", "zq_w4a8_linear_noalloc_status", "zq_w4a8_linear_plan", "zq_selftest_bounded_wait", "zq_lorc_workspace_bytes", "zq_lorc_factors",
-    "zq_w4a8_linear_fused_out", "zq_quantize_act_fp8_scaled",
+    "zq_w4a8_linear_fused_out", "zq_quantize_act_fp8_scaled", "zq_set_exclusive_device",
 ]
 PLAN_FIELDS = ("bm", "m_tiles", "n_tiles", "ctas", "stream", "persist", "splits", "kb_per_split", "base", "rem",
                "tail_pos0", "m_group", "partial_floats", "sms", "pair")
@@ -91,8 +91,15 @@ def lib() -> C.CDLL:
         L.zq_w4a8_linear_fused_out.argtypes = L.zq_w4a8_linear.argtypes + [ci, vp]
         L.zq_quantize_act_fp8_scaled.restype = ci
         L.zq_quantize_act_fp8_scaled.argtypes = [vp, i64, i64, i64, vp, vp, vp, vp, ci, vp, vp]
+        L.zq_set_exclusive_device.restype = ci
+        L.zq_set_exclusive_device.argtypes = [ci]
         _lib = L
     return _lib
+
+
+def set_exclusive_device(on: bool) -> bool:
+    """``zq_set_exclusive_device``: promise that nothing else runs on the device; returns the previous setting."""
+    return bool(lib().zq_set_exclusive_device(1 if on else 0))
 
 
 def status_string(status: int) -> str:

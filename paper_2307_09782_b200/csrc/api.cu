@@ -9,6 +9,8 @@ namespace zq {
 
 static std::atomic<int64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+static std::atomic<int> g_exclusive{0};
+bool exclusive_device() { return g_exclusive.load(std::memory_order_relaxed) != 0; }
 
 int check_device_sm100() {
   int dev = 0, major = 0;
@@ -123,6 +125,8 @@ const char* zq_status_string(int status) {
 }
 
 int64_t zq_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int zq_set_exclusive_device(int on) { return g_exclusive.exchange(on ? 1 : 0, std::memory_order_relaxed); }
 
 namespace {
 int quantize_act(const void* x, int64_t M, int64_t K, int64_t ldx, const float* absmax, bool scaled, uint8_t* q,

@@ -1200,8 +1200,12 @@ int launch_mx_cfg(const GemmArgs& a, const GemmPlan& plan, const Params& p, cuda
       pc.handover = 1;
     }
     void* args[3] = {&tm_w, &tm_q, &pc};
-    // chained to the kernel ahead (see pdl_wait); if the two launch attributes are refused together, cooperative alone
-    if (launch_chained(w4a8_mx_gemm_kernel<BM, W8, FUSEQ, NONE>, grid, dim3(C::kThreads), C::kSmemBytes, st, true, tm_w, tm_q, pc) ==
+    // chained to the kernel ahead (see pdl_wait); if the two launch attributes are refused together, cooperative alone.
+    // The cooperative attribute is what guarantees that all CTAs of the grid (one per SM at most) run at the same
+    // time; it costs about 3.5 us per launch (the launch waits for the whole device to be free).  A caller that
+    // has promised the device to this library alone (zq_set_exclusive_device) gets a plain launch: with nothing
+    // else running, a grid of at most one CTA per SM is resident as soon as the kernel ahead has drained.
+    if (launch_chained(w4a8_mx_gemm_kernel<BM, W8, FUSEQ, NONE>, grid, dim3(C::kThreads), C::kSmemBytes, st, !exclusive_device(), tm_w, tm_q, pc) ==
         cudaSuccess) {
       count_launch();
       return ZQ_OK;

@@ -133,6 +133,7 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout, bool a
 int launch_w4a8_gemm(const GemmArgs& a, cudaStream_t st);           // ZQ_WEIGHTS_CAST
 int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st);        // ZQ_WEIGHTS_MX
 int sm_count();
+bool exclusive_device();  // see zq_set_exclusive_device
 constexpr int kErrDetailSelfTest = 100;  // status detail written by zq_selftest_bounded_wait
 
 #ifdef __CUDACC__

@@ -157,3 +157,18 @@ def test_interleaved_with_larger_calls_on_one_workspace():
         y = binding.w4a8_linear(pw, x=x[:M], U=Ud, V=Vd, workspace=ws)
         assert binding.device_status(ws) == (0, 0)
         assert np.abs(host(y).astype(np.float64) - y_o[:M]).max() <= TOL_REL * np.abs(y_o[:M]).max(), M
+
+
+@pytest.mark.parametrize("M,N,K,r", [(8, 128 * 40, 1024, 8), (1, 128 * 224, 896, 8), (16, 256, 8192, 8), (40, 128 * 30, 1024, 8),
+                                     (500, 640, 2048, 8)])
+def test_plain_launches_on_an_exclusive_device(M, N, K, r):
+    """After zq_set_exclusive_device(1) the launches whose CTAs hand tiles over to one another are plain ones
+    instead of cooperative ones: same results, and the default comes back afterwards."""
+    x_bits, W, U, V = _layer(600 + M, M, N, K, r)
+    was = binding.set_exclusive_device(True)
+    try:
+        assert binding.set_exclusive_device(True) is True
+        _check(x_bits, W, U, V, calls=3)
+    finally:
+        binding.set_exclusive_device(was)
+    assert binding.set_exclusive_device(was) == was
