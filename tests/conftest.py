@@ -21,3 +21,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _launch_mode():
+    """ZQFP_TEST_EXCLUSIVE_DEVICE=1 runs the whole suite with the plain launches of zq_set_exclusive_device(1)
+    (the test process has the GPU to itself); the default is the library's default, cooperative launches."""
+    if os.environ.get("ZQFP_TEST_EXCLUSIVE_DEVICE") == "1":
+        from paper_2307_09782_b200 import binding
+        binding.set_exclusive_device(True)
+    yield
