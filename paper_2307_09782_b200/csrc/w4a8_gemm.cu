@@ -32,6 +32,7 @@
 //                and the epilogue
 // Ring depths NP and NA are multiples of NG, so a P or A stage is always handled by the same widen
 // group; that group then sees every round of the stage's barriers, which a parity wait needs.
+#include <cstdlib>
 #include "w4a8_gemm_shared.cuh"
 
 namespace zq {
@@ -650,36 +651,33 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout, bool a
   const int kblocks = static_cast<int>(K / kBlockK);
   if (tiles <= 0 || kblocks <= 0) return pl;  // nothing to do: an empty plan (ctas == 0)
   if (wide && allow_pair && bm >= 128 && pl.n_tiles % 2 == 0 && sm_count() >= 2 && tiles <= kWsMaxTiles) {
-    // CTA pairs: the two CTAs of a cluster share each token tile (128, 192 or 224 tokens, two accumulators) and
+    // CTA pairs: the two CTAs of a cluster share each token tile (128 or 176 ... 224 tokens, two accumulators) and
     // take two neighbouring channel tiles.  Work is counted in units of one K block of one pair position
     // (token tile x channel-tile pair) and partitioned among the pairs like the single CTAs' below: whole
     // positions in whole rounds where there are at least four rounds, the rest (or everything) dealt out as
     // contiguous unit ranges.  Taken when its padded token columns are at most 15 % more than the single
     // CTAs' (the pairs run about 20 % faster).
     const int64_t pairs = sm_count() / 2, np = pl.n_tiles / 2;
-    int best_bm = 0;
-    int64_t best_cols = 0;
-    for (const int cand : {224, 192, 128}) {  // wider tiles move fewer shared-memory bytes per flop: worth 5 % of padding
-      if (cand == 128 && M > 128) continue;   // 128-token tiles: one row of them only
-      const int64_t cols = ((M + cand - 1) / cand) * cand;
-      if (best_bm == 0 || cols * 21 < best_cols * 20) {
-        best_bm = cand;
-        best_cols = cols;
-      }
-    }
-    if (best_cols * 100 <= static_cast<int64_t>(pl.m_tiles) * bm * 115) {
+    // The token tile: the width with the least estimated time = rounds the pairs need (whole rounds count in
+    // full when the last one is left uneven) x what a round costs (16 KB of codes per K block and CTA plus 64
+    // bytes per token: shared-memory bytes, the bound of this kernel).
+    GemmPlan best{};
+    double best_cost = 0.0;
+    for (const int cand : {224, 208, 192, 176, 128}) {
+      if (cand == 128 && M > 128) continue;  // 128-token tiles: one row of them only
       GemmPlan pp{};
       pp.pair = 1;
-      pp.bm = best_bm;
-      pp.m_tiles = static_cast<int>(best_cols / best_bm);
+      pp.bm = cand;
+      pp.m_tiles = static_cast<int>((M + cand - 1) / cand);
       pp.n_tiles = pl.n_tiles;
       pp.splits = 1;
       pp.kb_per_split = kblocks;
       const int64_t positions = pp.m_tiles * np, punits = positions * kblocks;
       if (pp.m_tiles > 1) {
-        const int64_t fit = (int64_t(32) << 20) / (static_cast<int64_t>(best_bm) * K);
+        const int64_t fit = (int64_t(32) << 20) / (static_cast<int64_t>(cand) * K);
         pp.m_group = static_cast<int>(fit < 1 ? 1 : (fit > 8 ? 8 : fit));
       }
+      double rounds;
       if (positions >= 4 * pairs) {
         pp.persist = 1;
         pp.ctas = static_cast<int>(2 * pairs);
@@ -688,18 +686,28 @@ GemmPlan plan_gemm(int64_t M, int64_t N, int64_t K, int mode, int layout, bool a
         pp.tail_pos0 = static_cast<int>(positions - tail);
         pp.base = static_cast<int>(tail * kblocks / pairs);
         pp.rem = static_cast<int>(tail * kblocks % pairs);
-        return pp;
-      }
-      if (punits >= 8 && punits < (int64_t(1) << 30)) {
+        rounds = tail > 0 || positions % pairs == 0 ? static_cast<double>(positions) / pairs
+                                                    : static_cast<double>((positions + pairs - 1) / pairs);
+      } else if (punits >= 8 && punits < (int64_t(1) << 30)) {
         int64_t g = pairs < punits / 4 ? pairs : punits / 4;
         if (g < 1) g = 1;
         pp.stream = 1;
         pp.ctas = static_cast<int>(2 * g);
         pp.base = static_cast<int>(punits / g);
         pp.rem = static_cast<int>(punits % g);
-        return pp;
+        rounds = static_cast<double>(positions) / g;
+      } else {
+        continue;
+      }
+      const double cost = rounds * (256 + cand);
+      if (best.pair == 0 || cost < best_cost) {
+        best = pp;
+        best_cost = cost;
       }
     }
+    // taken when its padded token columns are at most 15 % more than the single CTAs' (the pairs run about 20 % faster)
+    if (best.pair && static_cast<int64_t>(best.m_tiles) * best.bm * 100 <= static_cast<int64_t>(pl.m_tiles) * bm * 115)
+      return best;
   }
   // CTAs per SM the kernel family is sized for at this tile
   // (the block-scaled kernel: always one; its launches with shared tiles are cooperative, and a cooperative

@@ -830,7 +830,7 @@ struct PairCfg {
   static constexpr int kNumBars = 2 * NS + 2 * NB + 1;
   static constexpr int offMisc = offBars + kNumBars * 8;
   static constexpr int kSmemBytes = offMisc + 32;
-  static_assert(BM % 32 == 0 && BM >= 64 && BM <= 224, "token tile of the pair: two accumulators");
+  static_assert(BM % 16 == 0 && BM >= 64 && BM <= 224, "token tile of the pair: two accumulators");
   static_assert(kTokBytes % 1024 == 0, "token stages must start on a swizzle atom");
   static_assert(NS >= 4, "pipeline depth");
   static_assert(kColsUsed <= kTmemCols, "tensor memory");
@@ -1292,7 +1292,9 @@ int launch_w4a8_mx_gemm(const GemmArgs& a, cudaStream_t st) {
       const bool w8p = a.layout == ZQ_WEIGHTS_MX_FP8;
       switch (plan.bm) {
         case 128: e = w8p ? launch_pair_cfg<128, true>(a, plan, pp, st) : launch_pair_cfg<128, false>(a, plan, pp, st); break;
+        case 176: e = w8p ? launch_pair_cfg<176, true>(a, plan, pp, st) : launch_pair_cfg<176, false>(a, plan, pp, st); break;
         case 192: e = w8p ? launch_pair_cfg<192, true>(a, plan, pp, st) : launch_pair_cfg<192, false>(a, plan, pp, st); break;
+        case 208: e = w8p ? launch_pair_cfg<208, true>(a, plan, pp, st) : launch_pair_cfg<208, false>(a, plan, pp, st); break;
         case 224: e = w8p ? launch_pair_cfg<224, true>(a, plan, pp, st) : launch_pair_cfg<224, false>(a, plan, pp, st); break;
       }
     }

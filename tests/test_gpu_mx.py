@@ -109,19 +109,22 @@ def test_linear_persistent_whole_tiles(M):
 
 @pytest.mark.parametrize("M,N,K,r,mode,layout,out_dtype", [
     (1120, 128 * 120, 512, 8, "M2", MX, torch.bfloat16),           # 224-token tiles, bf16 y
-    (1000, 128 * 120 - 37, 384, 8, "M1", MX, torch.float32),       # 192-token tiles, ragged last channel tile
+    (1000, 128 * 120 - 37, 384, 8, "M1", MX, torch.float32),       # 208-token tiles, ragged last channel tile
     (1100, 128 * 120, 256, 0, "M2", MX, torch.float32),            # no LoRC
     (1120, 128 * 120, 256, 16, "M2", MX, torch.float32),           # a rank the epilogue reads through the cache
     (896, 128 * 148, 256, 8, "M2", MX, torch.float32),             # four whole rounds of 74 pairs
+    (528, 128 * 200, 256, 8, "M2", MX, torch.float32),             # three tiles of 176 tokens
+    (1040, 128 * 120, 384, 8, "M1", MX, torch.bfloat16),           # five tiles of 208 tokens
 ])
 def test_linear_cta_pairs(M, N, K, r, mode, layout, out_dtype):
     """Many tokens and an even number of channel tiles: two CTAs share each token tile (one MMA of 256 channels
     over both CTAs' tensor memory), whole tiles only."""
     pl = binding.linear_plan(M, N, K, mode, layout)
-    assert pl["pair"] == 1 and pl["bm"] in (192, 224)
+    assert pl["pair"] == 1 and pl["bm"] in (176, 192, 208, 224)
     x_bits, W, U, V = _layer(91 + r, M, N, K, r)
     bm = pl["bm"]
-    rows = sorted({0, bm // 2 - 1, bm // 2, bm - 1, bm, bm + bm // 2, 2 * bm - 1, 3 * bm + 5, M - bm // 2 - 1, M - 2, M - 1})
+    rows = sorted({min(v, M - 1) for v in (0, bm // 2 - 1, bm // 2, bm - 1, bm, bm + bm // 2, 2 * bm - 1, 3 * bm + 5,
+                                           M - bm // 2 - 1, M - 2, M - 1)})
     check_linear(x_bits, W, U, V, 128, mode, layout=layout, rows=rows, out_dtype=out_dtype)
 
 

@@ -120,7 +120,7 @@ def test_plan_tile_choices_of_the_block_scaled_kernel():
     # one row of tiles up to 256 tokens, then 192 / 224 (two accumulators) or 256 (long rows, many tiles)
     assert [binding.linear_plan(M, 28672, 7168, "M2", "mx")["bm"] for M in (1, 16, 17, 64, 100, 192, 256)] == \
         [16, 16, 32, 64, 128, 192, 256]
-    assert binding.linear_plan(512, 28672 + 128, 7168, "M2", "mx")["bm"] == 192
+    assert binding.linear_plan(512, 28672 + 128, 7168, "M2", "mx")["bm"] == 192   # odd channel-tile count: single CTAs
     assert binding.linear_plan(8192, 28672, 7168, "M2", "mx")["bm"] == 224
     # many tokens, an even number of channel tiles: CTA pairs on whole tiles, the tile width with the fewest
     # rounds x width (37 x 28 pair positions of 224 tokens are 14 whole rounds of 74 pairs)
@@ -128,11 +128,13 @@ def test_plan_tile_choices_of_the_block_scaled_kernel():
     if p["sms"] == 148:
         assert p["pair"] == 1 and p["persist"] == 1 and p["bm"] == 224 and p["ctas"] == 148 and p["partial_floats"] == 0
         assert p["tail_pos0"] == 37 * 28                      # 14 whole rounds, nothing left to deal out
-        p = binding.linear_plan(2048, 7168, 28672, "M2", "mx")     # 11 x 28 positions: 4 rounds, 12 positions dealt out
-        assert p["pair"] == 1 and p["persist"] == 1 and p["bm"] == 192 and p["tail_pos0"] == 4 * 74
-        assert p["base"] * 74 + p["rem"] == 12 * 224
-        p = binding.linear_plan(512, 7168, 28672, "M2", "mx")      # 3 x 28 positions: fewer than four rounds, all dealt out
-        assert p["pair"] == 1 and p["stream"] == 1 and p["bm"] == 192 and p["base"] * 74 + p["rem"] == 84 * 224
+        p = binding.linear_plan(4096, 6656, 17920, "M2", "mx")     # 20 x 26 positions of 208 tokens: 7 rounds, 2 positions dealt out
+        assert p["pair"] == 1 and p["persist"] == 1 and p["bm"] == 208 and p["tail_pos0"] == 7 * 74
+        assert p["base"] * 74 + p["rem"] == 2 * 140
+        p = binding.linear_plan(2048, 7168, 28672, "M2", "mx")     # 10 x 28 positions: fewer than four rounds, all dealt out
+        assert p["pair"] == 1 and p["stream"] == 1 and p["bm"] == 208 and p["base"] * 74 + p["rem"] == 280 * 224
+        p = binding.linear_plan(512, 7168, 28672, "M2", "mx")      # three tiles of 176 tokens instead of 192
+        assert p["pair"] == 1 and p["stream"] == 1 and p["bm"] == 176 and p["base"] * 74 + p["rem"] == 84 * 224
     # an odd number of channel tiles: single CTAs, whole rounds of whole tiles and a dealt-out last round
     p = binding.linear_plan(8192, 7168 + 128, 28672, "M2", "mx")
     assert p["pair"] == 0 and p["persist"] == 1 and p["bm"] == 256
