@@ -32,7 +32,6 @@
 //                and the epilogue
 // Ring depths NP and NA are multiples of NG, so a P or A stage is always handled by the same widen
 // group; that group then sees every round of the stage's barriers, which a parity wait needs.
-#include <cstdlib>
 #include "w4a8_gemm_shared.cuh"
 
 namespace zq {
