@@ -39,7 +39,7 @@ WORKLOAD = "opt30b"
 GROUP, MODE, RANK = 128, "M2", 8
 NOMINAL_FP8_TFLOPS = 4500.0  # public dense FP8 figure of the part, for context
 # DRAM bytes per launch from the ncu captures summarised under profiles/ (null when the kernel changed since)
-DOMINANT_TRAFFIC = 1980e6  # mean of the two M = 8192 launches (1573 MB and 2388 MB)
+DOMINANT_TRAFFIC = 1760e6  # mean of the two M = 8192 launches (1516 MB and 2003 MB)
 DECODE_TRAFFIC = 114.5e6   # 7168 -> 28672 at 8 tokens
 # LLaMA-7B-shaped rows outside the timed step: (scale mode, weight layout)
 EXTRA_LLAMA7B = (("none", "cast"), ("none", "mx"), ("M2", "mx"))
