@@ -704,7 +704,9 @@ def run_ours(args):
             "sweep_note": "per-shape rows: each (layer, M) timed by itself after the timed region and a 1.5 s pause: one event pair "
                           "around n = 6-20 back-to-back launches (rotated weight copies), divided by n, median of 3 "
                           "batches; layer_us = one zq_w4a8_linear call on raw x; quant_us / gemm_us = the quantizer "
-                          "kernel alone and the GEMM alone on pre-quantized activations",
+                          "kernel alone and the GEMM alone on pre-quantized activations; the table is taken at the clocks "
+                          "the power cap leaves after the timed region (in a fresh process the shapes up to 2048 tokens "
+                          "read 1.2-1.6 x faster, e.g. the GEMMs at 512 tokens 93 us)",
             "sweep": table, "extra_rows": extra_rows, "lorc_factors_ms": lorc_ms, "mlp_chain": mlp_chain}
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(wl)
